@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of the paged decode-attention step (RoPE + KV append -> split-KV attention -> merge).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A "step" is one pass of the whole hot path over one batch of synthetic requests.  The headline
+workload is ``long_context`` (the largest single-GPU configuration: 4 requests x 131072 cached
+tokens, 2.1 GB of K/V read per step, far larger than L2, so no cache flush is needed between steps).
+``value`` is achieved KV-read bandwidth = algorithmic K/V bytes of the step / device time per step,
+with all inputs resident in HBM.  ``e2e`` is the same metric through ``ac_decode_step_host`` with the
+step's inputs in pinned host memory and the result read back to the host inside the timed region.
+The other four workloads are reported under ``workloads`` (us per call through a captured CUDA graph,
+L2 flushed between calls for the ones that fit in L2).  With N > 1 every rank runs an independent
+replica on its own GPU (the path has no exchange step); value is the sum over ranks.
+
+``--impl reference`` times the CPU oracle, as it stands, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2606_07665_b200 import workloads as W  # noqa: E402
+
+METRIC = "paged decode-attention KV-read bandwidth (us per call in ms_per_step)"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+L2_FLUSH_BYTES = 512 << 20
+
+
+# ---------------------------------------------------------------------------------------------
+# helpers
+# ---------------------------------------------------------------------------------------------
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def ncu_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch from the committed ncu summary (profiles/dram_traffic.json), or None."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
+            return json.load(f)[kernel][workload]["dram_bytes_per_launch"]
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    return rank, local, world
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle timing (reported baseline; also the --impl reference arm)
+# ---------------------------------------------------------------------------------------------
+
+def oracle_sample_seconds(w, budget_s: float = 12.0):
+    """Times the oracle on (request, KV head) pairs of ``w`` until about ``budget_s`` of CPU work.
+
+    Each sampled pair runs the oracle's own routines on views restricted to that request and KV
+    head: rotation + append of the new token, then attention of the group's query heads over all
+    cached pages.  Returns (KV bytes covered, seconds, description).
+    """
+    from oracle import paged_decode_oracle as O
+    G = w.Hq // w.Hkv
+    pairs = [(b, h) for b in range(w.B) for h in range(w.Hkv) if w.context_lens[b] >= 0]
+    rng = np.random.default_rng(0)
+    rng.shuffle(pairs)
+    t_total, bytes_total, n_done = 0.0, 0, 0
+    for b, h in pairs:
+        used = w.block_table[b, :(int(w.context_lens[b]) + w.page_size) // w.page_size]
+        remap = np.arange(used.size, dtype=np.int32)[None, :]
+        kc = w.k_cache[used][:, :, h:h + 1, :]           # the sample's own pages (copy = gather cost excluded)
+        vc = w.v_cache[used][:, :, h:h + 1, :]
+        t0 = time.perf_counter()
+        q_rot, k_after, v_after = O.oracle_rope_kv_append(
+            w.q[b:b + 1, h * G:(h + 1) * G], w.k_new[b:b + 1, h:h + 1], w.v_new[b:b + 1, h:h + 1], kc, vc,
+            remap, w.context_lens[b:b + 1], w.rope_cos, w.rope_sin, w.page_size)
+        O.oracle_paged_decode_attn(q_rot, k_after, v_after, remap, w.context_lens[b:b + 1], w.page_size)
+        t_total += time.perf_counter() - t0
+        bytes_total += (int(w.context_lens[b]) + 1) * w.d * 2 * 2
+        n_done += 1
+        if t_total >= budget_s:
+            break
+    desc = (f"{n_done} of {len(pairs)} (request, KV head) pairs of {w.name}: rotation+append and "
+            f"attention of the {G} query heads of each pair, fp64 numpy")
+    return bytes_total, t_total, desc
+
+
+def cpu_threads_used() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0))
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    w = W.NAMED[args.workload]()
+    per_step_budget = max(1.0, min(15.0, 120.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample_seconds(w, per_step_budget)
+    tot_b, tot_t, desc = 0, 0.0, ""
+    for _ in range(args.steps):
+        b, t, desc = oracle_sample_seconds(w, per_step_budget)
+        tot_b += b
+        tot_t += t
+    gbs = tot_b / tot_t / 1e9
+    cores = cpu_threads_used()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": w.kv_bytes / (gbs * 1e9) * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "head_dim": w.d,
+                   "page_size": w.page_size, "seed": w.seed,
+                   "note": "ms_per_step is the sample's rate extrapolated to the whole step"},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------------------------
+
+def time_headline(st, steps, warmup, torch):
+    """K steps back to back; CUDA events around the whole region and around each attention launch."""
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        st.step(stream)
+    torch.cuda.synchronize()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for i in range(steps):
+        st.rope_kv_append(stream)
+        ev[i][0].record(stream)
+        st.attention(stream)
+        ev[i][1].record(stream)
+        st.merge(stream)
+    t1.record(stream)
+    torch.cuda.synchronize()
+    total_ms = t0.elapsed_time(t1)
+    attn_ms = [a.elapsed_time(b) for a, b in ev]
+    return total_ms / steps, sum(attn_ms) / len(attn_ms)
+
+
+def time_e2e(st, steps, warmup, torch):
+    from paper_2606_07665_b200 import binding as ac
+    w = st.w
+
+    def pinned(a):
+        return torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+
+    h_q, h_k, h_v = pinned(w.q), pinned(w.k_new), pinned(w.v_new)
+    h_bt, h_len = pinned(w.block_table), pinned(w.context_lens)
+    h_out = torch.empty((w.B, w.Hq, w.d), dtype=torch.int16).pin_memory()
+    q_stage = torch.empty_like(st.q_in)
+    stream = torch.cuda.current_stream()
+
+    def one():
+        ac.ac_decode_step_host(h_q, h_k, h_v, h_bt, h_len, h_out, q_stage, st.k_new, st.v_new,
+                               st.block_table, st.context_lens, st.out, st.k_cache, st.v_cache,
+                               st.stride_page, st.stride_token, st.stride_head, w.max_pages_per_seq,
+                               st.rope_cos, st.rope_sin, w.max_position, 0.0, st.num_splits,
+                               st.workspace if st.num_splits > 1 else None, st.workspace_bytes,
+                               st.B, st.Hq, st.Hkv, st.d, st.ps, st.num_pages, st.max_context_len,
+                               st.status_flag, stream)
+
+    for _ in range(warmup):
+        one()
+    torch.cuda.synchronize()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for _ in range(steps):
+        one()
+    t1.record(stream)
+    torch.cuda.synchronize()
+    h2d = sum(t.numel() * t.element_size() for t in (h_q, h_k, h_v, h_bt, h_len))
+    d2h = h_out.numel() * h_out.element_size()
+    return t0.elapsed_time(t1) / steps, h2d, d2h
+
+
+def time_graph_calls(st, torch, reps, flush):
+    """us per call of the captured step; with ``flush`` a buffer larger than L2 is overwritten
+    between calls and each call gets its own event pair."""
+    graph = st.capture()
+    for _ in range(5):
+        graph.replay()
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+    if not flush:
+        t0 = torch.cuda.Event(enable_timing=True)
+        t1 = torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        t1.record(stream)
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1) / reps * 1e3, None
+    junk = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=st.device)
+    times = []
+    for i in range(reps):
+        junk.fill_(i & 0xFF)
+        a = torch.cuda.Event(enable_timing=True)
+        b = torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        graph.replay()
+        b.record(stream)
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b) * 1e3)
+    return statistics.median(times), min(times)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2606_07665_b200 import binding as ac
+    from paper_2606_07665_b200 import build, runner
+
+    rank, local, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    build.build()
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(device))
+    ac.ac_init(local)
+    peak, peak_kind = measured_peak()
+
+    w = W.NAMED[args.workload]()
+    st = runner.DecodeStep(w, device=device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        sampler.start()
+    ms_step, ms_attn = time_headline(st, args.steps, args.warmup, torch)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_e2e, h2d, d2h = time_e2e(st, args.steps, args.warmup, torch)
+    barrier()
+    flag = int(st.status_flag.item())
+
+    t = torch.tensor([ms_step, ms_attn, ms_e2e], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step, ms_attn, ms_e2e = t.tolist()
+
+    if rank == 0:
+        kv = w.kv_bytes
+        value = world * kv / (ms_step * 1e-3) / 1e9
+        e2e_value = world * kv / (ms_e2e * 1e-3) / 1e9
+        attn_gbs = kv / (ms_attn * 1e-3) / 1e9
+        others = []
+        if not args.only_headline:
+            del st
+            torch.cuda.empty_cache()
+            for name in ("tiny", "single_request", "continuous_batching") + tuple(
+                    f"graph_sweep_b{b}" for b in W.GRAPH_SWEEP_BATCHES):
+                ww = W.NAMED[name]()
+                s2 = runner.DecodeStep(ww, device=device)
+                fits_l2 = ww.kv_bytes < 3 * (126 << 20)
+                warm_us, _ = time_graph_calls(s2, torch, 200, flush=False)
+                cold_us, cold_min = time_graph_calls(s2, torch, 30, flush=True) if fits_l2 else (warm_us, None)
+                others.append({
+                    "workload": name, "B": ww.B, "kv_mb": round(ww.kv_bytes / 1e6, 3),
+                    "num_splits": s2.num_splits, "us_per_call": round(cold_us, 2),
+                    "us_per_call_l2_warm": round(warm_us, 2),
+                    "kv_gbs": round(ww.kv_bytes / cold_us / 1e3, 1),
+                    "frac_of_hbm_peak": round(ww.kv_bytes / cold_us / 1e3 / peak, 4),
+                    "l2": "flushed between calls" if fits_l2 else "inputs larger than L2",
+                    "via": "cuda graph replay"})
+                del s2, ww
+                torch.cuda.empty_cache()
+            cpu_bytes, cpu_s, cpu_desc = oracle_sample_seconds(w, 12.0)
+            cpu = {"value": cpu_bytes / cpu_s / 1e9, "unit": UNIT, "cores": cpu_threads_used(),
+                   "kind": "oracle", "sample": cpu_desc}
+        else:
+            cpu = None
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "head_dim": w.d,
+                       "page_size": w.page_size, "context_len": int(w.context_lens.max()),
+                       "num_pages": w.num_pages, "seed": w.seed, "num_splits": runner_splits(w, ac),
+                       "kv_bytes_per_step": kv, "l2": "inputs larger than L2 (no flush)",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "us_per_call": ms_step * 1e3,
+            "frac_of_hbm_peak": value / world / peak,
+            "roofline": {"bound": "hbm", "achieved": attn_gbs, "peak": peak, "unit": "GB/s",
+                         "frac": attn_gbs / peak, "peak_kind": peak_kind,
+                         "kernel": "paged_decode_attn_kernel",
+                         "traffic": ncu_traffic("paged_decode_attn_kernel", w.name)},
+            "cpu_baseline": cpu,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
+            "gpu_launches": args.steps * (3 if runner_splits(w, ac) > 1 else 2),
+            "clocks": clocks, "status_flag": flag, "workloads": others,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def runner_splits(w, ac):
+    return ac.ac_decode_plan(w.B, w.Hq, w.Hkv, w.d, w.page_size, w.max_context_len, ac.ac_sm_count())[0]
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", default="long_context", choices=sorted(W.NAMED))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--only-headline", action="store_true",
+                    help="skip the other workloads and the CPU baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args)
+    else:
+        args.steps = 1000 if args.steps is None else args.steps
+        args.warmup = 10 if args.warmup is None else max(3, args.warmup)
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

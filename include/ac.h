@@ -1,0 +1,181 @@
+/*
+ * ac.h -- C ABI of the B200 (sm_100a) paged decode-attention library (libac.so).
+ *
+ * One decode step of one attention layer, for a batch of requests that each contribute ONE new
+ * token, over a paged KV cache:
+ *
+ *   ac_rope_kv_append      rotary embedding of the new q and k, then the new k/v are written into
+ *                          their cache page through the block table
+ *   ac_paged_decode_attn   grouped-query attention of each request's query token over all of its
+ *                          cached pages, one CTA per (request, KV head, KV split), online softmax;
+ *                          emits per-split partial results (or the final output when 1 split)
+ *   ac_splitkv_merge       log-sum-exp merge of the per-split partial results
+ *
+ * Source of each operation (the paper gives them in prose only): Method, "Principle-Driven LLM
+ * Kernel Generator", kernel families (iii) "standalone RoPE kernel" and (iv) "paged decode
+ * attention ... online-softmax kernel over paged KV with fused cross-CTA merging"; Method, "Kernel
+ * Customization and Multi-Request Adaptation": the kv_append scatter kernel ("writes the new K/V
+ * vectors", attention then runs "with the sequence length advanced by one"), the paged KV cache
+ * allocated at block granularity, sequence lengths kept on the GPU, and decode steps replayed as
+ * bucketed CUDA Graphs (one graph per batch-size bucket).
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer owned by the caller unless its name ends in _host or
+ *     _out.  The library never allocates or frees device memory, never synchronises and never reads
+ *     device memory on the host: each call only validates its arguments and enqueues work on
+ *     `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream).  The three kernel
+ *     calls may therefore be recorded in a CUDA Graph; ac_init must have been called before capture.
+ *   - Tensors q/k/v/cache/out are bf16 (16-bit patterns); rope tables and partials are fp32;
+ *     block_table and context_lens are int32.  The innermost dimension (head_dim) is contiguous.
+ *   - Return value: AC_OK (0) or an ac_status > 0.  On any non-zero return nothing was launched.
+ *     The library never throws, aborts or exits.
+ *   - Supported: head_dim d in {64, 128}; page_size a multiple of 16, <= 256; Hq % Hkv == 0 and
+ *     Hq / Hkv <= 16; all base pointers 16-byte aligned; cache strides multiples of 8 elements, and
+ *     of stride_token / stride_head the larger one a multiple of the smaller one.
+ *   - Rows with context_lens[b] < 0 are inactive (batch padding up to a graph bucket): nothing is
+ *     written to the cache for them and their output row is +0.
+ *   - Query head hq reads KV head hq / (Hq / Hkv).
+ */
+#ifndef AC_H_
+#define AC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    AC_OK = 0,
+    AC_ERR_NULL = 1,        /* a required pointer is NULL */
+    AC_ERR_SHAPE = 2,       /* a size is non-positive or inconsistent */
+    AC_ERR_UNSUPPORTED = 3, /* outside the supported set listed above */
+    AC_ERR_ALIGN = 4,       /* pointer or stride alignment */
+    AC_ERR_WORKSPACE = 5,   /* workspace too small for num_splits */
+    AC_ERR_CUDA = 6,        /* a CUDA call failed; see ac_last_cuda_error() */
+    AC_ERR_NOT_INIT = 7     /* ac_init has not succeeded on the current device */
+} ac_status;
+
+/* Bits the kernels OR into the optional device word `status_flag` (never cleared by the library). */
+#define AC_FLAG_PAGE_OOB 1     /* a block-table entry used for the append was outside [0, num_pages) */
+#define AC_FLAG_POSITION_OOB 2 /* context_lens[b] >= max_position or its page index >= max_pages_per_seq */
+#define AC_FLAG_WAIT_TIMEOUT 4 /* a bounded wait on a shared-memory barrier gave up */
+
+/* Once per device, outside any stream capture, with no other call of this library running on that
+ * device: reads the device properties, resolves the driver's tensor-map encoder and sets the
+ * dynamic shared-memory limits of every kernel instantiation.  device < 0 means the current device.
+ * Idempotent. */
+int ac_init(int device);
+
+/* Static, never-freed description of a status code. */
+const char* ac_status_string(int status);
+
+/* cudaError_t (or CUresult, for tensor-map encoding) recorded by the last AC_ERR_CUDA on this thread. */
+int ac_last_cuda_error(void);
+
+/* Number of SMs of the device ac_init saw last; 0 before any ac_init. */
+int ac_sm_count(void);
+
+/* Split plan (host only, pure, needs no GPU).  Chooses how many KV splits the attention kernel
+ * should use so that B * Hkv * num_splits CTAs fill `sm_count` SMs (<= 0: the count seen by
+ * ac_init, or 148 if none) several times over, without making splits shorter than a few hundred
+ * tokens.  max_context_len = the largest number of tokens any row attends over in this bucket
+ * (cached + new).  Outputs: *num_splits_out >= 1, *split_tokens_out = tokens per split (a multiple
+ * of 64; split s of row b covers tokens [s*split_tokens, min((s+1)*split_tokens, n_b)) ), and
+ * *workspace_bytes_out = bytes of fp32 workspace the attention + merge calls need for that plan
+ * (0 when num_splits == 1).  The paper's kernel merges across CTAs inside the attention kernel and
+ * does not state how it sizes the split; this heuristic is this library's own. */
+int ac_decode_plan(int B, int Hq, int Hkv, int d, int page_size, int max_context_len, int sm_count,
+                   int* num_splits_out, int* split_tokens_out, size_t* workspace_bytes_out);
+
+/* Tokens per split the attention kernel uses for a given (max_context_len, num_splits): the smallest
+ * multiple of 64 whose num_splits-fold covers max_context_len.  Host only, pure. */
+int ac_split_tokens(int max_context_len, int num_splits);
+
+/* Workspace bytes for (B, Hq, d, num_splits): partial_o fp32 [B,Hq,num_splits,d] followed by
+ * partial_lse fp32 [B,Hq,num_splits]; 0 when num_splits == 1.  Host only, pure. */
+size_t ac_workspace_bytes(int B, int Hq, int d, int num_splits);
+
+/* A1 + A2: RoPE on the new q/k and KV append (families (iii) "standalone RoPE kernel" and the
+ * kv_append scatter kernel of "Kernel Customization and Multi-Request Adaptation").
+ *
+ * For every active row b, with p = context_lens[b] (the position of the new token, 0-based):
+ *   q_out[b,h,:]  = rope(q_in[b,h,:], p)   for all Hq heads   (q_out may alias q_in)
+ *   k_cache[page, slot, h, :] = rope(k_new[b,h,:], p),  v_cache[page, slot, h, :] = v_new[b,h,:]
+ *   for all Hkv heads, page = block_table[b, p / page_size], slot = p % page_size.
+ * rope pairs element i with i + d/2 (i < d/2):  (x_i, x_{i+d/2}) -> (x_i c - x_{i+d/2} s,
+ * x_{i+d/2} c + x_i s) with c = rope_cos[p, i], s = rope_sin[p, i].  Each result is the
+ * round-to-nearest-even bf16 of the real value (products exact, one fp64 addition, one rounding), so
+ * cache contents are reproducible bit for bit.  v is copied verbatim.
+ *
+ * Layout: q_in/q_out [B,Hq,d], k_new/v_new [B,Hkv,d] dense; cache element (page, slot, head, j) at
+ * page*stride_page + slot*stride_token + head*stride_head + j (strides in elements);
+ * block_table [B, max_pages_per_seq]; rope_cos/rope_sin [max_position, d/2].
+ * A row whose position or page id is out of range writes nothing and sets status_flag bits (if
+ * status_flag != NULL).  Two rows appending into the same slot is a caller error (not detected). */
+int ac_rope_kv_append(const void* q_in, void* q_out, const void* k_new, const void* v_new,
+                      void* k_cache, void* v_cache,
+                      int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                      const int32_t* block_table, int max_pages_per_seq,
+                      const int32_t* context_lens,
+                      const float* rope_cos, const float* rope_sin, int max_position,
+                      int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                      int32_t* status_flag, void* stream);
+
+/* A4: paged decode attention, family (iv).  Row b attends over tokens 0 .. n_b - 1 with
+ * n_b = context_lens[b] + new_tokens (new_tokens = 1 right after ac_rope_kv_append, 0 to attend
+ * over the cached tokens only); token t lives in page block_table[b, t / page_size], slot
+ * t % page_size.  For query head hq:  out = softmax(scale * q_rot[b,hq,:] . K[t,:]) V  over those
+ * tokens (bf16 operands, fp32 accumulation, fp32 softmax); softmax_scale <= 0 means 1/sqrt(d).
+ *
+ * Grid: one CTA per (request, KV head, split) holding the whole group of Hq/Hkv query heads.
+ * num_splits == 1: the final bf16 result is written to out [B,Hq,d]; workspace may be NULL.
+ * num_splits  > 1: out is not touched; split s writes its own normalised result to
+ *   partial_o  = (float*)workspace                      [B,Hq,num_splits,d]
+ *   partial_lse = partial_o + B*Hq*num_splits*d          [B,Hq,num_splits]  natural-log
+ * log-sum-exp of the scaled scores; a split with no tokens writes lse = -inf and leaves its
+ * partial_o untouched.  workspace_bytes must be >= ac_workspace_bytes(B,Hq,d,num_splits).
+ * max_context_len must be >= every n_b (tokens beyond num_splits*split_tokens are not visited).
+ * Contents of cache slots at or past n_b, of unreferenced pages and of unused block-table entries
+ * never influence the result.  A page id outside [0, num_pages) reads as zeros. */
+int ac_paged_decode_attn(const void* q_rot, const void* k_cache, const void* v_cache,
+                         int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                         const int32_t* block_table, int max_pages_per_seq,
+                         const int32_t* context_lens, int new_tokens, float softmax_scale,
+                         int num_splits, void* workspace, size_t workspace_bytes, void* out,
+                         int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                         int max_context_len, int32_t* status_flag, void* stream);
+
+/* A5: merge of the split partials ("cross-CTA merging" of family (iv), here as its own kernel):
+ *   M = max_s lse_s,  w_s = exp(lse_s - M),  out[b,hq,:] = sum_s w_s partial_o[b,hq,s,:] / sum_s w_s
+ * rounded to bf16.  Splits with lse = -inf are skipped (their partial_o is not read); a row whose
+ * splits are all empty, or with context_lens[b] < 0 (context_lens may be NULL), gets +0.
+ * workspace has the layout written by ac_paged_decode_attn for the same B, Hq, d, num_splits. */
+int ac_splitkv_merge(const void* workspace, int num_splits, const int32_t* context_lens, void* out,
+                     int B, int Hq, int d, void* stream);
+
+/* The whole step from HOST buffers (for callers that hold the step's inputs on the host, and for
+ * end-to-end timing): copies q/k_new/v_new/block_table/context_lens from the *_host buffers (pinned
+ * memory recommended) into the caller's device buffers of the same name, enqueues the three
+ * kernels with a plan from ac_decode_plan's rule given (max_context_len, num_splits), and copies the
+ * bf16 result from out into out_host.  Everything is asynchronous on `stream`; the caller
+ * synchronises the stream before reading out_host.  The KV cache pools and rope tables stay on the
+ * device (they are the layer's resident state, not a per-step input).  No paper counterpart. */
+int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* v_new_host,
+                        const int32_t* block_table_host, const int32_t* context_lens_host,
+                        void* out_host,
+                        void* q, void* k_new, void* v_new, int32_t* block_table,
+                        int32_t* context_lens, void* out,
+                        void* k_cache, void* v_cache,
+                        int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                        int max_pages_per_seq,
+                        const float* rope_cos, const float* rope_sin, int max_position,
+                        float softmax_scale, int num_splits, void* workspace, size_t workspace_bytes,
+                        int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                        int max_context_len, int32_t* status_flag, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AC_H_ */

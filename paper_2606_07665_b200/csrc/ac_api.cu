@@ -1,0 +1,365 @@
+// The C ABI of libac: argument validation, the split plan, tensor-map construction and the launches.
+#include <math.h>
+#include <stdlib.h>
+
+#include "ac_internal.h"
+
+namespace ac {
+
+namespace {
+
+DeviceState g_devices[kMaxDevices];
+thread_local int t_last_cuda_error = 0;
+int g_last_sm_count = 0;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode_tiled = nullptr;
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct Shape {
+    int B, Hq, Hkv, d, page_size, num_pages;
+};
+
+int check_shape(const Shape& s) {
+    if (s.B <= 0 || s.Hq <= 0 || s.Hkv <= 0 || s.d <= 0 || s.page_size <= 0 || s.num_pages <= 0)
+        return AC_ERR_SHAPE;
+    if (s.Hq % s.Hkv != 0) return AC_ERR_SHAPE;
+    if (s.d != 64 && s.d != 128) return AC_ERR_UNSUPPORTED;
+    if (s.page_size % 16 != 0 || s.page_size > 256) return AC_ERR_UNSUPPORTED;
+    if (s.Hq / s.Hkv > 16) return AC_ERR_UNSUPPORTED;
+    if (s.B > 65535 || s.Hq > 65535) return AC_ERR_UNSUPPORTED;
+    return AC_OK;
+}
+
+int check_strides(const Shape& s, int64_t stride_page, int64_t stride_token, int64_t stride_head) {
+    if (stride_page <= 0 || stride_token <= 0 || stride_head <= 0) return AC_ERR_SHAPE;
+    if (stride_page % 8 || stride_token % 8 || stride_head % 8) return AC_ERR_ALIGN;
+    if (stride_token < s.d && stride_head < s.d) return AC_ERR_SHAPE;
+    const int64_t lo = stride_token < stride_head ? stride_token : stride_head;
+    const int64_t hi = stride_token < stride_head ? stride_head : stride_token;
+    if (lo < s.d) return AC_ERR_SHAPE;
+    if (hi % lo != 0 || stride_page % hi != 0) return AC_ERR_UNSUPPORTED;
+    return AC_OK;
+}
+
+int current_ready_device(int* device_out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail_cuda(static_cast<int>(e));
+    if (dev < 0 || dev >= kMaxDevices || !g_devices[dev].ready) return AC_ERR_NOT_INIT;
+    *device_out = dev;
+    return AC_OK;
+}
+
+// 4-D view of one cache pool for 16-token x 64-element box loads.  Dimensions are ordered by
+// increasing stride: head_dim, then head and token-in-page (whichever has the smaller stride first),
+// then page.
+int make_cache_map(CUtensorMap* map, const void* base, const Shape& s, int64_t stride_page,
+                   int64_t stride_token, int64_t stride_head, bool* head_before_token) {
+    const bool head_first = stride_head <= stride_token;
+    *head_before_token = head_first;
+    cuuint64_t dims[4];
+    cuuint64_t strides[3];
+    cuuint32_t box[4];
+    cuuint32_t elem_strides[4] = {1, 1, 1, 1};
+    dims[0] = static_cast<cuuint64_t>(s.d);
+    box[0] = 64;
+    if (head_first) {
+        dims[1] = s.Hkv;        strides[0] = static_cast<cuuint64_t>(stride_head) * 2;   box[1] = 1;
+        dims[2] = s.page_size;  strides[1] = static_cast<cuuint64_t>(stride_token) * 2;  box[2] = 16;
+    } else {
+        dims[1] = s.page_size;  strides[0] = static_cast<cuuint64_t>(stride_token) * 2;  box[1] = 16;
+        dims[2] = s.Hkv;        strides[1] = static_cast<cuuint64_t>(stride_head) * 2;   box[2] = 1;
+    }
+    dims[3] = s.num_pages;
+    strides[2] = static_cast<cuuint64_t>(stride_page) * 2;
+    box[3] = 1;
+    CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
+                                strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
+    return AC_OK;
+}
+
+}  // namespace
+
+DeviceState& device_state(int device) { return g_devices[device]; }
+
+int fail_cuda(int code) {
+    t_last_cuda_error = code;
+    return AC_ERR_CUDA;
+}
+
+int split_tokens_for(int max_context_len, int num_splits) {
+    if (max_context_len < 1) max_context_len = 1;
+    if (num_splits < 1) num_splits = 1;
+    const long long per = (static_cast<long long>(max_context_len) + num_splits - 1) / num_splits;
+    const long long rounded = (per + 63) / 64 * 64;
+    return static_cast<int>(rounded > 0x7fffffc0ll ? 0x7fffffc0ll : rounded);
+}
+
+}  // namespace ac
+
+using namespace ac;
+
+extern "C" {
+
+int ac_init(int device) {
+    cudaError_t e;
+    if (device < 0) {
+        e = cudaGetDevice(&device);
+        if (e != cudaSuccess) return fail_cuda(static_cast<int>(e));
+    }
+    if (device >= kMaxDevices) return AC_ERR_UNSUPPORTED;
+    int prev = -1;
+    e = cudaGetDevice(&prev);
+    if (e != cudaSuccess) return fail_cuda(static_cast<int>(e));
+    if (prev != device) {
+        e = cudaSetDevice(device);
+        if (e != cudaSuccess) return fail_cuda(static_cast<int>(e));
+    }
+    int status = AC_OK;
+    DeviceState st;
+    int major = 0;
+    do {
+        if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device)) != cudaSuccess ||
+            (e = cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess ||
+            (e = cudaDeviceGetAttribute(&st.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device)) != cudaSuccess) {
+            status = fail_cuda(static_cast<int>(e));
+            break;
+        }
+        if (major != 10) {          // the kernels are built for sm_100a only
+            status = AC_ERR_UNSUPPORTED;
+            break;
+        }
+        if (g_encode_tiled == nullptr) {
+            void* fn = nullptr;
+            cudaDriverEntryPointQueryResult qres;
+            e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+            if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess) {
+                status = fail_cuda(static_cast<int>(e != cudaSuccess ? e : cudaErrorSymbolNotFound));
+                break;
+            }
+            g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+        }
+        e = attn_set_attributes(st.smem_optin);
+        if (e != cudaSuccess) {
+            status = fail_cuda(static_cast<int>(e));
+            break;
+        }
+        st.ready = true;
+        g_devices[device] = st;
+        g_last_sm_count = st.sm_count;
+    } while (false);
+    if (prev != device) cudaSetDevice(prev);
+    return status;
+}
+
+const char* ac_status_string(int status) {
+    switch (status) {
+        case AC_OK: return "ok";
+        case AC_ERR_NULL: return "a required pointer is NULL";
+        case AC_ERR_SHAPE: return "a size or stride is non-positive or inconsistent";
+        case AC_ERR_UNSUPPORTED: return "shape, layout or device outside the supported set";
+        case AC_ERR_ALIGN: return "pointer or stride not aligned to 16 bytes";
+        case AC_ERR_WORKSPACE: return "workspace missing or too small for num_splits";
+        case AC_ERR_CUDA: return "a CUDA call failed (see ac_last_cuda_error)";
+        case AC_ERR_NOT_INIT: return "ac_init has not succeeded on the current device";
+        default: return "unknown status";
+    }
+}
+
+int ac_last_cuda_error(void) { return t_last_cuda_error; }
+
+int ac_sm_count(void) { return g_last_sm_count; }
+
+int ac_split_tokens(int max_context_len, int num_splits) {
+    return split_tokens_for(max_context_len, num_splits);
+}
+
+size_t ac_workspace_bytes(int B, int Hq, int d, int num_splits) {
+    if (B <= 0 || Hq <= 0 || d <= 0 || num_splits <= 1) return 0;
+    return static_cast<size_t>(B) * Hq * num_splits * (static_cast<size_t>(d) + 1) * sizeof(float);
+}
+
+int ac_decode_plan(int B, int Hq, int Hkv, int d, int page_size, int max_context_len, int sm_count,
+                   int* num_splits_out, int* split_tokens_out, size_t* workspace_bytes_out) {
+    if (num_splits_out == nullptr || split_tokens_out == nullptr || workspace_bytes_out == nullptr)
+        return AC_ERR_NULL;
+    Shape s{B, Hq, Hkv, d, page_size, 1};
+    int st = check_shape(s);
+    if (st != AC_OK) return st;
+    if (max_context_len <= 0) return AC_ERR_SHAPE;
+    if (sm_count <= 0) sm_count = g_last_sm_count > 0 ? g_last_sm_count : 148;
+
+    // Two CTAs are resident per SM.  Aim for about four waves of CTAs so the tail of the last wave
+    // stays small, but keep every split at least kMinSplitTokens long so the per-CTA prologue
+    // (barrier set-up, first loads in flight) and the partial-result traffic stay a small fraction.
+    const long long kMinSplitTokens = 256;
+    const long long target_ctas = static_cast<long long>(sm_count) * 2 * 4;
+    const long long base_ctas = static_cast<long long>(B) * Hkv;
+    long long want = (target_ctas + base_ctas - 1) / base_ctas;
+    long long cap = static_cast<long long>(max_context_len) / kMinSplitTokens;
+    if (cap < 1) cap = 1;
+    long long S = want < cap ? want : cap;
+    if (S < 1) S = 1;
+    if (S > 65535) S = 65535;
+    int chunk = split_tokens_for(max_context_len, static_cast<int>(S));
+    // Drop splits that the rounding of the chunk length made empty for every row.
+    S = (static_cast<long long>(max_context_len) + chunk - 1) / chunk;
+    *num_splits_out = static_cast<int>(S);
+    *split_tokens_out = split_tokens_for(max_context_len, static_cast<int>(S));
+    *workspace_bytes_out = ac_workspace_bytes(B, Hq, d, static_cast<int>(S));
+    return AC_OK;
+}
+
+int ac_rope_kv_append(const void* q_in, void* q_out, const void* k_new, const void* v_new,
+                      void* k_cache, void* v_cache, int64_t stride_page, int64_t stride_token,
+                      int64_t stride_head, const int32_t* block_table, int max_pages_per_seq,
+                      const int32_t* context_lens, const float* rope_cos, const float* rope_sin,
+                      int max_position, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                      int32_t* status_flag, void* stream) {
+    if (!q_in || !q_out || !k_new || !v_new || !k_cache || !v_cache || !block_table || !context_lens ||
+        !rope_cos || !rope_sin)
+        return AC_ERR_NULL;
+    Shape s{B, Hq, Hkv, d, page_size, num_pages};
+    int st = check_shape(s);
+    if (st != AC_OK) return st;
+    if (max_pages_per_seq <= 0 || max_position <= 0) return AC_ERR_SHAPE;
+    st = check_strides(s, stride_page, stride_token, stride_head);
+    if (st != AC_OK) return st;
+    if (!aligned16(q_in) || !aligned16(q_out) || !aligned16(k_new) || !aligned16(v_new) ||
+        !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(rope_cos) || !aligned16(rope_sin))
+        return AC_ERR_ALIGN;
+    int dev;
+    st = current_ready_device(&dev);
+    if (st != AC_OK) return st;
+    cudaError_t e = launch_rope_kv_append(q_in, q_out, k_new, v_new, k_cache, v_cache, stride_page,
+                                          stride_token, stride_head, block_table, max_pages_per_seq,
+                                          context_lens, rope_cos, rope_sin, max_position, B, Hq, Hkv, d,
+                                          page_size, num_pages, status_flag,
+                                          static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
+}
+
+int ac_paged_decode_attn(const void* q_rot, const void* k_cache, const void* v_cache,
+                         int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                         const int32_t* block_table, int max_pages_per_seq,
+                         const int32_t* context_lens, int new_tokens, float softmax_scale,
+                         int num_splits, void* workspace, size_t workspace_bytes, void* out, int B,
+                         int Hq, int Hkv, int d, int page_size, int num_pages, int max_context_len,
+                         int32_t* status_flag, void* stream) {
+    if (!q_rot || !k_cache || !v_cache || !block_table || !context_lens) return AC_ERR_NULL;
+    Shape s{B, Hq, Hkv, d, page_size, num_pages};
+    int st = check_shape(s);
+    if (st != AC_OK) return st;
+    if (max_pages_per_seq <= 0 || max_context_len <= 0 || num_splits <= 0) return AC_ERR_SHAPE;
+    if (new_tokens != 0 && new_tokens != 1) return AC_ERR_UNSUPPORTED;
+    if (num_splits > 65535) return AC_ERR_UNSUPPORTED;
+    st = check_strides(s, stride_page, stride_token, stride_head);
+    if (st != AC_OK) return st;
+    if (!aligned16(q_rot) || !aligned16(k_cache) || !aligned16(v_cache)) return AC_ERR_ALIGN;
+    float* partial_o = nullptr;
+    float* partial_lse = nullptr;
+    if (num_splits == 1) {
+        if (!out) return AC_ERR_NULL;
+        if (!aligned16(out)) return AC_ERR_ALIGN;
+    } else {
+        if (!workspace || workspace_bytes < ac_workspace_bytes(B, Hq, d, num_splits)) return AC_ERR_WORKSPACE;
+        if (!aligned16(workspace)) return AC_ERR_ALIGN;
+        partial_o = static_cast<float*>(workspace);
+        partial_lse = partial_o + static_cast<size_t>(B) * Hq * num_splits * d;
+    }
+    int dev;
+    st = current_ready_device(&dev);
+    if (st != AC_OK) return st;
+    CUtensorMap k_map, v_map;
+    bool head_first = true;
+    st = make_cache_map(&k_map, k_cache, s, stride_page, stride_token, stride_head, &head_first);
+    if (st != AC_OK) return st;
+    st = make_cache_map(&v_map, v_cache, s, stride_page, stride_token, stride_head, &head_first);
+    if (st != AC_OK) return st;
+    const float scale = softmax_scale > 0.0f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d));
+    const int split_tokens = split_tokens_for(max_context_len, num_splits);
+    cudaError_t e = launch_paged_decode_attn(k_map, v_map, head_first, q_rot, block_table,
+                                             max_pages_per_seq, context_lens, new_tokens, scale,
+                                             num_splits, split_tokens, partial_o, partial_lse, out, B,
+                                             Hq, Hkv, d, page_size, status_flag,
+                                             static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
+}
+
+int ac_splitkv_merge(const void* workspace, int num_splits, const int32_t* context_lens, void* out,
+                     int B, int Hq, int d, void* stream) {
+    if (!workspace || !out) return AC_ERR_NULL;
+    if (B <= 0 || Hq <= 0 || num_splits <= 0) return AC_ERR_SHAPE;
+    if (d != 64 && d != 128) return AC_ERR_UNSUPPORTED;
+    if (B > 65535) return AC_ERR_UNSUPPORTED;
+    if (!aligned16(workspace) || !aligned16(out)) return AC_ERR_ALIGN;
+    int dev;
+    int st = current_ready_device(&dev);
+    if (st != AC_OK) return st;
+    const float* partial_o = static_cast<const float*>(workspace);
+    const float* partial_lse = partial_o + static_cast<size_t>(B) * Hq * num_splits * d;
+    cudaError_t e = launch_splitkv_merge(partial_o, partial_lse, num_splits, context_lens, out, B, Hq, d,
+                                         static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
+}
+
+int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* v_new_host,
+                        const int32_t* block_table_host, const int32_t* context_lens_host,
+                        void* out_host, void* q, void* k_new, void* v_new, int32_t* block_table,
+                        int32_t* context_lens, void* out, void* k_cache, void* v_cache,
+                        int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                        int max_pages_per_seq, const float* rope_cos, const float* rope_sin,
+                        int max_position, float softmax_scale, int num_splits, void* workspace,
+                        size_t workspace_bytes, int B, int Hq, int Hkv, int d, int page_size,
+                        int num_pages, int max_context_len, int32_t* status_flag, void* stream) {
+    if (!q_host || !k_new_host || !v_new_host || !block_table_host || !context_lens_host || !out_host ||
+        !q || !k_new || !v_new || !block_table || !context_lens || !out)
+        return AC_ERR_NULL;
+    Shape s{B, Hq, Hkv, d, page_size, num_pages};
+    int st = check_shape(s);
+    if (st != AC_OK) return st;
+    if (max_pages_per_seq <= 0) return AC_ERR_SHAPE;
+    if (num_splits > 1 && (!workspace || workspace_bytes < ac_workspace_bytes(B, Hq, d, num_splits)))
+        return AC_ERR_WORKSPACE;
+    int dev;
+    st = current_ready_device(&dev);
+    if (st != AC_OK) return st;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const size_t q_bytes = static_cast<size_t>(B) * Hq * d * 2;
+    const size_t kv_bytes = static_cast<size_t>(B) * Hkv * d * 2;
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(q, q_host, q_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(k_new, k_new_host, kv_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(v_new, v_new_host, kv_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(block_table, block_table_host,
+                             static_cast<size_t>(B) * max_pages_per_seq * sizeof(int32_t),
+                             cudaMemcpyHostToDevice, cs)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(context_lens, context_lens_host, static_cast<size_t>(B) * sizeof(int32_t),
+                             cudaMemcpyHostToDevice, cs)) != cudaSuccess)
+        return fail_cuda(static_cast<int>(e));
+    st = ac_rope_kv_append(q, q, k_new, v_new, k_cache, v_cache, stride_page, stride_token, stride_head,
+                           block_table, max_pages_per_seq, context_lens, rope_cos, rope_sin,
+                           max_position, B, Hq, Hkv, d, page_size, num_pages, status_flag, stream);
+    if (st != AC_OK) return st;
+    st = ac_paged_decode_attn(q, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
+                              max_pages_per_seq, context_lens, 1, softmax_scale, num_splits, workspace,
+                              workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages,
+                              max_context_len, status_flag, stream);
+    if (st != AC_OK) return st;
+    if (num_splits > 1) {
+        st = ac_splitkv_merge(workspace, num_splits, context_lens, out, B, Hq, d, stream);
+        if (st != AC_OK) return st;
+    }
+    e = cudaMemcpyAsync(out_host, out, q_bytes, cudaMemcpyDeviceToHost, cs);
+    return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
+}
+
+}  // extern "C"

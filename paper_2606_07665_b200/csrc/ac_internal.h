@@ -1,0 +1,58 @@
+// Host-side declarations shared by the translation units of libac (not part of the public ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "ac.h"
+
+namespace ac {
+
+constexpr int kMaxDevices = 64;
+
+struct DeviceState {
+    bool ready = false;
+    int sm_count = 0;
+    int smem_optin = 0;
+};
+
+// Filled by ac_init; indexed by CUDA device ordinal.
+DeviceState& device_state(int device);
+
+// Records the CUDA error of the calling thread's last failure and returns AC_ERR_CUDA.
+int fail_cuda(int code);
+
+// Tokens per split for (max_context_len, num_splits): smallest multiple of 64 that covers it.
+int split_tokens_for(int max_context_len, int num_splits);
+
+struct CacheView {
+    const void* k_cache;
+    const void* v_cache;
+    int64_t stride_page, stride_token, stride_head;   // elements
+    int num_pages, page_size, Hkv, d;
+};
+
+// Per-kernel launchers; each validates nothing (the ABI layer did) and returns a cudaError_t.
+cudaError_t attn_set_attributes(int smem_optin);
+cudaError_t launch_rope_kv_append(const void* q_in, void* q_out, const void* k_new, const void* v_new,
+                                  void* k_cache, void* v_cache, int64_t stride_page,
+                                  int64_t stride_token, int64_t stride_head,
+                                  const int32_t* block_table, int max_pages_per_seq,
+                                  const int32_t* context_lens, const float* rope_cos,
+                                  const float* rope_sin, int max_position, int B, int Hq, int Hkv,
+                                  int d, int page_size, int num_pages, int32_t* status_flag,
+                                  cudaStream_t stream);
+cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap& v_map,
+                                     bool head_before_token, const void* q_rot,
+                                     const int32_t* block_table, int max_pages_per_seq,
+                                     const int32_t* context_lens, int new_tokens, float scale,
+                                     int num_splits, int split_tokens, float* partial_o,
+                                     float* partial_lse, void* out, int B, int Hq, int Hkv, int d,
+                                     int page_size, int32_t* status_flag, cudaStream_t stream);
+cudaError_t launch_splitkv_merge(const float* partial_o, const float* partial_lse, int num_splits,
+                                 const int32_t* context_lens, void* out, int B, int Hq, int d,
+                                 cudaStream_t stream);
+
+}  // namespace ac

@@ -1,0 +1,415 @@
+// A4: single-token decode attention over a paged KV cache, one CTA per (request, KV head, split).
+//
+// Data movement.  The K and V pools are described to the TMA unit as 4-D tensors
+// (head_dim, {head, token-in-page} ordered by stride, page).  A work tile is 16 consecutive tokens of
+// one KV head inside one page: head_dim/64 box loads of [16 tokens x 64 elements] for K and the same
+// for V, written to shared memory with the 128-byte swizzle so that ldmatrix reads are free of bank
+// conflicts.  Every warp runs its own ring of STAGES tiles with one mbarrier per stage and takes
+// tiles warp, warp+WARPS, ... of the CTA's token range; there is no CTA-wide synchronisation in the
+// main loop.  The physical page id of a tile is fetched from the block table one tile ahead of the
+// TMA issue that needs it.  KV bytes are read once, so the loads carry an evict-first L2 policy.
+//
+// Arithmetic.  The Hq/Hkv query heads of the group are the rows of a 16-row MMA tile (rows >= group
+// size are zero).  S = Q K^T and O += P V use the bf16 m16n8k16 warp MMA with fp32 accumulators; the
+// accumulator layout of S is the A-operand layout of the second product, so P never leaves
+// registers.  Softmax is the online form (running max and sum per row, in the exp2 domain) with
+// warp-shuffle reductions across the four lanes that share a row.  At the end the warps' partial
+// (max, sum, O) are combined through shared memory and the CTA writes either the final bf16 row
+// (one split) or its normalised fp32 partial plus the natural-log log-sum-exp (several splits).
+//
+// With a group of 4-8 query rows the path needs G flop per KV byte; at HBM speed that exceeds what
+// the fp32 pipes deliver for G >= 7, which is why the products run on the tensor pipe even though
+// the kernel is bound by HBM bandwidth.
+#include <math.h>
+
+#include "ac_device.cuh"
+#include "ac_internal.h"
+
+namespace ac {
+namespace {
+
+using namespace acdev;
+
+constexpr int WARPS = 4;
+constexpr int THREADS = WARPS * 32;
+constexpr int STAGES = 3;
+constexpr int TILE = 16;                      // tokens per stage
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr float LN2 = 0.6931471805599453f;
+
+template <int D>
+struct Smem {
+    static constexpr int HALVES = D / 64;                 // 64-element (128-byte) column blocks
+    static constexpr int HALF_BYTES = TILE * 128;         // one swizzled [16 x 128 B] block
+    static constexpr int K_BYTES = HALVES * HALF_BYTES;   // K tile; V tile has the same size
+    static constexpr int STAGE_BYTES = 2 * K_BYTES;
+    static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
+    static constexpr int BAR_OFFSET = WARPS * RING_BYTES;
+    static constexpr int TOTAL = BAR_OFFSET + WARPS * STAGES * 8 + 1024;   // + alignment slack
+};
+
+struct AttnParams {
+    const uint16_t* q;            // [B, Hq, D] bf16, already rotated
+    const int32_t* block_table;   // [B, max_pages_per_seq]
+    const int32_t* context_lens;  // [B]
+    float* partial_o;             // [B, Hq, S, D]   (S > 1)
+    float* partial_lse;           // [B, Hq, S]      (S > 1)
+    uint16_t* out;                // [B, Hq, D] bf16 (S == 1)
+    int32_t* status_flag;
+    float scale_log2;             // softmax scale * log2(e)
+    int max_pages_per_seq;
+    int new_tokens;
+    int num_splits;
+    int split_tokens;
+    int Hq, Hkv, page_size;
+    int head_before_token;        // order of the two middle tensor-map coordinates
+};
+
+template <int D, bool WIDE>
+__global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
+    const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
+    const AttnParams p) {
+    using L = Smem<D>;
+    constexpr int ROWS = WIDE ? 2 : 1;          // row blocks of 8 query heads held per thread
+    constexpr int KSTEPS = D / 16;
+    constexpr int NTILES = D / 8;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_addr(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_addr(smem_raw));
+
+    const int h = blockIdx.x;
+    const int split = blockIdx.y;
+    const int b = blockIdx.z;
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int G = p.Hq / p.Hkv;
+    const int S = p.num_splits;
+
+    const int ctx = p.context_lens[b];
+    int n_tokens = ctx < 0 ? 0 : ctx + p.new_tokens;
+    n_tokens = min(n_tokens, p.max_pages_per_seq * p.page_size);
+    const int tok_begin = split * p.split_tokens;
+    const int tok_end = min(tok_begin + p.split_tokens, n_tokens);
+
+    if (tok_begin >= tok_end) {
+        // Nothing to attend over in this split.
+        if (S > 1) {
+            if (threadIdx.x < G)
+                p.partial_lse[(static_cast<size_t>(b) * p.Hq + h * G + threadIdx.x) * S + split] = -INFINITY;
+        } else {
+            uint16_t* o = p.out + (static_cast<size_t>(b) * p.Hq + h * G) * D;
+            for (int e = threadIdx.x; e < G * D; e += THREADS) o[e] = 0;
+        }
+        return;
+    }
+
+    const uint32_t ring = smem_base + warp * L::RING_BYTES;
+    const uint32_t bars = smem_base + L::BAR_OFFSET + warp * STAGES * 8;
+    if (lane == 0) {
+        tma_prefetch_descriptor(&k_map);
+        tma_prefetch_descriptor(&v_map);
+#pragma unroll
+        for (int s = 0; s < STAGES; ++s) mbar_init(bars + s * 8, 1);
+        mbar_init_fence();
+    }
+    __syncwarp();
+
+    const int tile_begin = tok_begin / TILE;
+    const int n_tiles = (tok_end - tok_begin + TILE - 1) / TILE;
+    const int n_my = n_tiles > warp ? (n_tiles - warp + WARPS - 1) / WARPS : 0;
+    const int32_t* bt_row = p.block_table + static_cast<size_t>(b) * p.max_pages_per_seq;
+    const uint64_t policy = l2_policy_evict_first();
+
+    auto tile_token0 = [&](int j) { return (tile_begin + warp + j * WARPS) * TILE; };
+    auto load_page_id = [&](int j) { return bt_row[tile_token0(j) / p.page_size]; };
+    auto issue = [&](int j, int page) {      // lane 0 only
+        const int tok0 = tile_token0(j);
+        const int slot = tok0 % p.page_size;
+        const int stage = j % STAGES;
+        const uint32_t bar = bars + stage * 8;
+        const uint32_t dst = ring + stage * L::STAGE_BYTES;
+        const int c1 = p.head_before_token ? h : slot;
+        const int c2 = p.head_before_token ? slot : h;
+        mbar_arrive_expect_tx(bar, L::STAGE_BYTES);
+#pragma unroll
+        for (int hf = 0; hf < L::HALVES; ++hf)
+            tma_load_4d(dst + hf * L::HALF_BYTES, &k_map, bar, hf * 64, c1, c2, page, policy);
+#pragma unroll
+        for (int hf = 0; hf < L::HALVES; ++hf)
+            tma_load_4d(dst + L::K_BYTES + hf * L::HALF_BYTES, &v_map, bar, hf * 64, c1, c2, page, policy);
+    };
+
+    // ---- prologue: fill the ring -------------------------------------------------------------
+    int issued = 0;
+    int page_next = n_my > 0 ? load_page_id(0) : 0;
+    for (; issued < STAGES && issued < n_my; ++issued) {
+        const int page = page_next;
+        page_next = issued + 1 < n_my ? load_page_id(issued + 1) : 0;
+        if (lane == 0) issue(issued, page);
+    }
+
+    // ---- query fragments (A operand of Q K^T), rows = heads of the group ---------------------------
+    const int g = lane >> 2;
+    const int t = lane & 3;
+    uint32_t qa[KSTEPS][2 * ROWS];
+    {
+        const uint16_t* qrow0 = p.q + (static_cast<size_t>(b) * p.Hq + h * G + g) * D;
+        const bool v0 = g < G;
+        const bool v1 = WIDE && (g + 8 < G);
+#pragma unroll
+        for (int kk = 0; kk < KSTEPS; ++kk) {
+            const int col = kk * 16 + 2 * t;
+            qa[kk][0] = v0 ? *reinterpret_cast<const uint32_t*>(qrow0 + col) : 0u;
+            qa[kk][ROWS] = v0 ? *reinterpret_cast<const uint32_t*>(qrow0 + col + 8) : 0u;
+            if (WIDE) {
+                qa[kk][1] = v1 ? *reinterpret_cast<const uint32_t*>(qrow0 + 8 * D + col) : 0u;
+                qa[kk][ROWS + 1] = v1 ? *reinterpret_cast<const uint32_t*>(qrow0 + 8 * D + col + 8) : 0u;
+            }
+        }
+    }
+    // qa[kk] = {a0 (row g, k lo), [a1 (row g+8, k lo)], a2 (row g, k hi), [a3 (row g+8, k hi)]}
+
+    float o[NTILES][2 * ROWS];
+#pragma unroll
+    for (int nt = 0; nt < NTILES; ++nt)
+#pragma unroll
+        for (int e = 0; e < 2 * ROWS; ++e) o[nt][e] = 0.0f;
+    float m_run[ROWS], l_run[ROWS];
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+        m_run[r] = -INFINITY;
+        l_run[r] = 0.0f;
+    }
+
+    // lane-dependent parts of the ldmatrix addresses (row r of matrix mi; 128-byte rows, swizzled)
+    const int mi = lane >> 3;
+    const int r8 = lane & 7;
+    const uint32_t k_row_off = ((mi >> 1) * 8 + r8) * 128;     // K: matrices 0,1 -> tokens 0-7; 2,3 -> 8-15
+    const int k_chunk_lo = mi & 1;                              //    matrices 0,2 -> k lo; 1,3 -> k hi
+    const uint32_t v_row_off = ((mi & 1) * 8 + r8) * 128;      // V: matrices 0,2 -> tokens 0-7; 1,3 -> 8-15
+    const int v_chunk_lo = mi >> 1;                             //    matrices 0,1 -> n-tile even; 2,3 -> odd
+
+    bool timed_out = false;
+    int j = 0;
+    for (; j < n_my; ++j) {
+        const int stage = j % STAGES;
+        const uint32_t kbase = ring + stage * L::STAGE_BYTES;
+        const uint32_t vbase = kbase + L::K_BYTES;
+        if (!mbar_wait_bounded(bars + stage * 8, (j / STAGES) & 1)) {
+            timed_out = true;
+            break;
+        }
+        const int tok0 = tile_token0(j);
+        const int n_valid = tok_end - tok0;                    // >= 1; < 16 only on the last tile
+
+        // ---- S = Q K^T for 16 tokens -------------------------------------------------------
+        float s[2][4];
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) s[nt][e] = 0.0f;
+#pragma unroll
+        for (int kk = 0; kk < KSTEPS; ++kk) {
+            const int dc = 2 * kk + k_chunk_lo;                // 16-byte column chunk of head_dim
+            const uint32_t addr = kbase + (dc >> 3) * L::HALF_BYTES + k_row_off + (((dc & 7) ^ r8) << 4);
+            uint32_t b00, b01, b10, b11;
+            ldmatrix_x4(b00, b01, b10, b11, addr);
+            if (WIDE) {
+                mma_bf16_16816(s[0][0], s[0][1], s[0][2], s[0][3], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b00, b01);
+                mma_bf16_16816(s[1][0], s[1][1], s[1][2], s[1][3], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b10, b11);
+            } else {
+                mma_bf16_16816_top(s[0][0], s[0][1], qa[kk][0], qa[kk][1], b00, b01);
+                mma_bf16_16816_top(s[1][0], s[1][1], qa[kk][0], qa[kk][1], b10, b11);
+            }
+        }
+
+        if (n_valid < TILE) {
+            // Slots past the request's length hold arbitrary bits: mask their scores and clear their
+            // V rows (0 * NaN would poison the product).
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (nt * 8 + 2 * t + (e & 1) >= n_valid) s[nt][e] = -INFINITY;
+            const int chunks_per_row = L::HALVES * 8;
+            for (int idx = lane; idx < (TILE - n_valid) * chunks_per_row; idx += 32) {
+                const int row = n_valid + idx / chunks_per_row;
+                const int rem = idx % chunks_per_row;
+                uint4* dstz = reinterpret_cast<uint4*>(smem_gen + (vbase - smem_base) +
+                                                       (rem >> 3) * L::HALF_BYTES + row * 128 + (rem & 7) * 16);
+                *dstz = make_uint4(0u, 0u, 0u, 0u);
+            }
+            __syncwarp();
+        }
+
+        // ---- online softmax (exp2 domain) --------------------------------------------------
+        uint32_t pa[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r) {
+            float mx = fmaxf(fmaxf(s[0][2 * r], s[0][2 * r + 1]), fmaxf(s[1][2 * r], s[1][2 * r + 1]));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m_run[r], mx * p.scale_log2);
+            const float alpha = exp2f(m_run[r] - m_new);
+            m_run[r] = m_new;
+            const float p00 = exp2f(fmaf(s[0][2 * r], p.scale_log2, -m_new));
+            const float p01 = exp2f(fmaf(s[0][2 * r + 1], p.scale_log2, -m_new));
+            const float p10 = exp2f(fmaf(s[1][2 * r], p.scale_log2, -m_new));
+            const float p11 = exp2f(fmaf(s[1][2 * r + 1], p.scale_log2, -m_new));
+            l_run[r] = fmaf(l_run[r], alpha, (p00 + p01) + (p10 + p11));
+            pa[r] = pack_bf16x2(p00, p01);          // a0 / a1: tokens 2t, 2t+1
+            pa[2 + r] = pack_bf16x2(p10, p11);      // a2 / a3: tokens 2t+8, 2t+9
+            if (alpha != 1.0f) {
+#pragma unroll
+                for (int nt = 0; nt < NTILES; ++nt) {
+                    o[nt][2 * r] *= alpha;
+                    o[nt][2 * r + 1] *= alpha;
+                }
+            }
+        }
+
+        // ---- O += P V ----------------------------------------------------------------------
+#pragma unroll
+        for (int jj = 0; jj < NTILES / 2; ++jj) {
+            const int dc = 2 * jj + v_chunk_lo;
+            const uint32_t addr = vbase + (dc >> 3) * L::HALF_BYTES + v_row_off + (((dc & 7) ^ r8) << 4);
+            uint32_t b00, b01, b10, b11;
+            ldmatrix_x4_trans(b00, b01, b10, b11, addr);
+            if (WIDE) {
+                mma_bf16_16816(o[2 * jj][0], o[2 * jj][1], o[2 * jj][2], o[2 * jj][3], pa[0], pa[1], pa[2], pa[3], b00, b01);
+                mma_bf16_16816(o[2 * jj + 1][0], o[2 * jj + 1][1], o[2 * jj + 1][2], o[2 * jj + 1][3], pa[0], pa[1], pa[2], pa[3], b10, b11);
+            } else {
+                mma_bf16_16816_top(o[2 * jj][0], o[2 * jj][1], pa[0], pa[2], b00, b01);
+                mma_bf16_16816_top(o[2 * jj + 1][0], o[2 * jj + 1][1], pa[0], pa[2], b10, b11);
+            }
+        }
+
+        // ---- refill this stage -----------------------------------------------------------------
+        __syncwarp();
+        if (issued < n_my) {
+            const int page = page_next;
+            page_next = issued + 1 < n_my ? load_page_id(issued + 1) : 0;
+            if (lane == 0) issue(issued, page);
+            ++issued;
+        }
+    }
+
+    if (timed_out) {
+        // Record the failure, then give the copies still in flight a bounded chance to land before
+        // this CTA's shared memory is released.
+        if (lane == 0 && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_WAIT_TIMEOUT);
+        for (int jj = j; jj < issued; ++jj) mbar_wait_bounded(bars + (jj % STAGES) * 8, (jj / STAGES) & 1);
+    }
+
+    // ---- combine the warps' partial results through shared memory ----------------------------------
+    // Each warp reuses the start of its own ring (all of its loads have completed).
+    constexpr int WROWS = 8 * ROWS;
+    float* wo = reinterpret_cast<float*>(smem_gen + warp * L::RING_BYTES);     // [WROWS][D]
+    float* wm = wo + WROWS * D;                                                 // [WROWS]
+    float* wl = wm + WROWS;                                                     // [WROWS]
+    static_assert((WROWS * D + 2 * WROWS) * 4 <= L::RING_BYTES, "merge scratch must fit in a ring");
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+        float l = l_run[r];
+        l += __shfl_xor_sync(0xffffffffu, l, 1);
+        l += __shfl_xor_sync(0xffffffffu, l, 2);
+        const int row = g + 8 * r;
+        if (t == 0) {
+            wm[row] = m_run[r];
+            wl[row] = l;
+        }
+#pragma unroll
+        for (int nt = 0; nt < NTILES; ++nt)
+            *reinterpret_cast<float2*>(wo + row * D + nt * 8 + 2 * t) = make_float2(o[nt][2 * r], o[nt][2 * r + 1]);
+    }
+    __syncthreads();
+
+    for (int e = threadIdx.x; e < G * D; e += THREADS) {
+        const int row = e / D;
+        const int col = e - row * D;
+        float mw[WARPS];
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) {
+            mw[w] = reinterpret_cast<const float*>(smem_gen + w * L::RING_BYTES)[WROWS * D + row];
+            M = fmaxf(M, mw[w]);
+        }
+        float num = 0.0f, den = 0.0f;
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) {
+            const float* base = reinterpret_cast<const float*>(smem_gen + w * L::RING_BYTES);
+            const float wgt = exp2f(mw[w] - M);                 // 0 for a warp that saw no tile
+            num = fmaf(wgt, base[row * D + col], num);
+            den = fmaf(wgt, base[WROWS * D + WROWS + row], den);
+        }
+        const float val = num / den;
+        const size_t hq = static_cast<size_t>(b) * p.Hq + h * G + row;
+        if (S == 1) {
+            p.out[hq * D + col] = static_cast<uint16_t>(pack_bf16x2(val, 0.0f) & 0xFFFFu);
+        } else {
+            p.partial_o[(hq * S + split) * D + col] = val;
+            if (col == 0) p.partial_lse[hq * S + split] = (M + log2f(den)) * LN2;
+        }
+    }
+}
+
+template <int D, bool WIDE>
+cudaError_t launch_one(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnParams& p, int B,
+                       cudaStream_t stream) {
+    dim3 grid(p.Hkv, p.num_splits, B);
+    paged_decode_attn_kernel<D, WIDE><<<grid, THREADS, Smem<D>::TOTAL, stream>>>(k_map, v_map, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t attn_set_attributes(int smem_optin) {
+    if (Smem<128>::TOTAL > smem_optin) return cudaErrorInvalidConfiguration;
+    cudaError_t e;
+#define AC_SET(D_, W_)                                                                             \
+    e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_>,                                     \
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D_>::TOTAL);        \
+    if (e != cudaSuccess) return e;
+    AC_SET(128, false)
+    AC_SET(128, true)
+    AC_SET(64, false)
+    AC_SET(64, true)
+#undef AC_SET
+    return cudaSuccess;
+}
+
+cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap& v_map,
+                                     bool head_before_token, const void* q_rot,
+                                     const int32_t* block_table, int max_pages_per_seq,
+                                     const int32_t* context_lens, int new_tokens, float scale,
+                                     int num_splits, int split_tokens, float* partial_o,
+                                     float* partial_lse, void* out, int B, int Hq, int Hkv, int d,
+                                     int page_size, int32_t* status_flag, cudaStream_t stream) {
+    AttnParams p;
+    p.q = static_cast<const uint16_t*>(q_rot);
+    p.block_table = block_table;
+    p.context_lens = context_lens;
+    p.partial_o = partial_o;
+    p.partial_lse = partial_lse;
+    p.out = static_cast<uint16_t*>(out);
+    p.status_flag = status_flag;
+    p.scale_log2 = scale * LOG2E;
+    p.max_pages_per_seq = max_pages_per_seq;
+    p.new_tokens = new_tokens;
+    p.num_splits = num_splits;
+    p.split_tokens = split_tokens;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.page_size = page_size;
+    p.head_before_token = head_before_token ? 1 : 0;
+    const bool wide = Hq / Hkv > 8;
+    if (d == 128) {
+        return wide ? launch_one<128, true>(k_map, v_map, p, B, stream)
+                    : launch_one<128, false>(k_map, v_map, p, B, stream);
+    }
+    return wide ? launch_one<64, true>(k_map, v_map, p, B, stream)
+                : launch_one<64, false>(k_map, v_map, p, B, stream);
+}
+
+}  // namespace ac

@@ -1,0 +1,138 @@
+"""Device-side staging of a workload and the launch sequence of one decode step.
+
+Only plumbing: torch tensors for device memory, the split plan from the library, and the three
+C-ABI calls in order.  Every arithmetic step runs inside libac's kernels.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as ac
+
+
+def _dev_u16(a: np.ndarray, device) -> torch.Tensor:
+    """uint16 bf16 bit patterns -> device int16 tensor (same bits)."""
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(device)
+
+
+def bits_of(t: torch.Tensor) -> np.ndarray:
+    """Device int16 tensor -> host uint16 bit patterns."""
+    return t.detach().cpu().numpy().view(np.uint16)
+
+
+class DecodeStep:
+    """Holds one workload on the device and enqueues RoPE+append -> attention -> merge.
+
+    ``layout`` is "token_major" ([page, slot, head, d], the default) or "head_major"
+    ([page, head, slot, d]); the kernels see only the strides.
+    """
+
+    def __init__(self, w, device="cuda:0", num_splits: int | None = None, layout: str = "token_major",
+                 max_context_len: int | None = None):
+        self.w = w
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        ac.ac_init(self.device.index if self.device.index is not None else -1)
+        self.B, self.Hq, self.Hkv, self.d, self.ps = w.B, w.Hq, w.Hkv, w.d, w.page_size
+        self.num_pages = w.num_pages
+        self.layout = layout
+        kc, vc = w.k_cache, w.v_cache
+        if layout == "head_major":
+            kc = np.ascontiguousarray(kc.transpose(0, 2, 1, 3))
+            vc = np.ascontiguousarray(vc.transpose(0, 2, 1, 3))
+            self.stride_page = self.Hkv * self.ps * self.d
+            self.stride_head = self.ps * self.d
+            self.stride_token = self.d
+        elif layout == "token_major":
+            self.stride_page = self.ps * self.Hkv * self.d
+            self.stride_token = self.Hkv * self.d
+            self.stride_head = self.d
+        else:
+            raise ValueError(layout)
+        self.k_cache = _dev_u16(kc, self.device)
+        self.v_cache = _dev_u16(vc, self.device)
+        self.q_in = _dev_u16(w.q, self.device)
+        self.q_rot = self.q_in.clone()          # rows the kernel skips (inactive) keep their input
+        self.k_new = _dev_u16(w.k_new, self.device)
+        self.v_new = _dev_u16(w.v_new, self.device)
+        self.block_table = torch.from_numpy(w.block_table).to(self.device)
+        self.context_lens = torch.from_numpy(w.context_lens).to(self.device)
+        self.rope_cos = torch.from_numpy(w.rope_cos).to(self.device)
+        self.rope_sin = torch.from_numpy(w.rope_sin).to(self.device)
+        self.out = torch.zeros((self.B, self.Hq, self.d), dtype=torch.int16, device=self.device)
+        self.status_flag = torch.zeros(1, dtype=torch.int32, device=self.device)
+        self.max_context_len = int(max_context_len) if max_context_len else w.max_context_len
+        self.set_splits(num_splits)
+
+    def set_splits(self, num_splits: int | None) -> None:
+        if num_splits is None:
+            num_splits, _, _ = ac.ac_decode_plan(self.B, self.Hq, self.Hkv, self.d, self.ps,
+                                                 self.max_context_len, ac.ac_sm_count())
+        self.num_splits = int(num_splits)
+        self.split_tokens = ac.ac_split_tokens(self.max_context_len, self.num_splits)
+        self.workspace_bytes = ac.ac_workspace_bytes(self.B, self.Hq, self.d, self.num_splits)
+        self.workspace = (torch.empty(max(self.workspace_bytes, 16) // 4, dtype=torch.float32,
+                                      device=self.device))
+
+    # -- the three calls -----------------------------------------------------------------------
+    def rope_kv_append(self, stream=None) -> None:
+        ac.ac_rope_kv_append(self.q_in, self.q_rot, self.k_new, self.v_new, self.k_cache, self.v_cache,
+                             self.stride_page, self.stride_token, self.stride_head, self.block_table,
+                             self.w.max_pages_per_seq, self.context_lens, self.rope_cos, self.rope_sin,
+                             self.w.max_position, self.B, self.Hq, self.Hkv, self.d, self.ps,
+                             self.num_pages, self.status_flag, stream)
+
+    def attention(self, stream=None, new_tokens: int = 1, q=None) -> None:
+        ac.ac_paged_decode_attn(self.q_rot if q is None else q, self.k_cache, self.v_cache,
+                                self.stride_page, self.stride_token, self.stride_head, self.block_table,
+                                self.w.max_pages_per_seq, self.context_lens, new_tokens, 0.0,
+                                self.num_splits, self.workspace if self.num_splits > 1 else None,
+                                self.workspace_bytes, self.out, self.B, self.Hq, self.Hkv, self.d,
+                                self.ps, self.num_pages, self.max_context_len, self.status_flag, stream)
+
+    def merge(self, stream=None) -> None:
+        if self.num_splits > 1:
+            ac.ac_splitkv_merge(self.workspace, self.num_splits, self.context_lens, self.out, self.B,
+                                self.Hq, self.d, stream)
+
+    def step(self, stream=None) -> None:
+        self.rope_kv_append(stream)
+        self.attention(stream)
+        self.merge(stream)
+
+    @property
+    def launches_per_step(self) -> int:
+        return 3 if self.num_splits > 1 else 2
+
+    def capture(self) -> torch.cuda.CUDAGraph:
+        """Record one step into a CUDA graph (one graph per batch-size bucket in a serving loop)."""
+        side = torch.cuda.Stream(device=self.device)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            self.step(side)                      # warm-up outside capture
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            self.step(side)
+        return graph
+
+    # -- results -------------------------------------------------------------------------------
+    def cache_bits(self):
+        k, v = bits_of(self.k_cache), bits_of(self.v_cache)
+        if self.layout == "head_major":
+            k = k.reshape(self.num_pages, self.Hkv, self.ps, self.d).transpose(0, 2, 1, 3)
+            v = v.reshape(self.num_pages, self.Hkv, self.ps, self.d).transpose(0, 2, 1, 3)
+        return k, v
+
+    def out_f64(self) -> np.ndarray:
+        b = bits_of(self.out)
+        return (b.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+    def partials(self):
+        n = self.B * self.Hq * self.num_splits
+        ws = self.workspace.detach().cpu().numpy()
+        po = ws[:n * self.d].reshape(self.B, self.Hq, self.num_splits, self.d)
+        pl = ws[n * self.d:n * self.d + n].reshape(self.B, self.Hq, self.num_splits)
+        return po, pl

@@ -1,0 +1,364 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Cache writes and rotated q are compared bit for bit; attention outputs within the stated
+tolerances (max abs <= 2e-2, mean abs <= 2e-3, plus a scale-aware bound)."""
+import numpy as np
+import pytest
+
+from oracle import paged_decode_oracle as O
+from paper_2606_07665_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS = 2e-2
+MEAN_ABS = 2e-3
+# Scale-aware bound per output element, from the kernel's arithmetic: the final rounding to bf16
+# costs at most half a bf16 spacing, 2^-8 * |ref|; rounding the softmax weights to bf16 before the
+# P.V product perturbs each weight by at most 2^-8 relative with random sign, which moves an output
+# by a few times 2^-8/sqrt(3) * rms of its row in the worst element; fp32 accumulation is far below.
+ROUND_REL = 2.0 ** -8
+ROW_RMS_REL = 1e-2
+
+
+@pytest.fixture(scope="module")
+def rt():
+    import torch
+    from paper_2606_07665_b200 import binding, build, runner
+    build.build()
+    binding.ac_init(0)
+    torch.cuda.set_device(0)
+    return runner
+
+
+def check_out(got, ref, what=""):
+    """got, ref: [..., d]; rows are the last axis."""
+    err = np.abs(got - ref)
+    assert np.isfinite(got).all(), what
+    assert err.max() <= MAX_ABS, (what, err.max())
+    assert err.mean() <= MEAN_ABS, (what, err.mean())
+    row_rms = np.sqrt(np.mean(ref ** 2, axis=-1, keepdims=True))
+    bound = ROUND_REL * np.abs(ref) + ROW_RMS_REL * row_rms
+    worst = float((err / np.maximum(bound, 1e-30)).max()) if err.size else 0.0
+    assert (err <= bound).all(), (what, "worst err/bound", worst)
+    return worst
+
+
+def run_and_compare(rt, w, num_splits=None, layout="token_major", check_cache=True):
+    import torch
+    q_rot, k_after, v_after, out_ref = O.oracle_decode_step(w)
+    st = rt.DecodeStep(w, num_splits=num_splits, layout=layout)
+    st.step()
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) == 0
+    if check_cache:
+        assert np.array_equal(rt.bits_of(st.q_rot), q_rot), "rotated q differs"
+        k_gpu, v_gpu = st.cache_bits()
+        assert np.array_equal(k_gpu, k_after), "K pool differs"
+        assert np.array_equal(v_gpu, v_after), "V pool differs"
+    worst = check_out(st.out_f64(), out_ref, f"{w.name} S={st.num_splits} {layout}")
+    print(f"[parity] {w.name} S={st.num_splits} {layout}: worst err/bound = {worst:.3f}")
+    return st, out_ref
+
+
+def small(seed, **kw):
+    base = dict(B=3, Hq=8, Hkv=2, d=128, page_size=16, num_pages=96, context_lens=[200, 37, 333],
+                rope_base=10000.0)
+    base.update(kw)
+    return W.make_workload("small", seed, **base)
+
+
+# ---------------------------------------------------------------------------------------------
+# RoPE + append: bit-exact
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("kw", [
+    dict(),
+    dict(d=64, Hq=6, Hkv=3, context_lens=[15, 16, 17]),                     # around a page boundary
+    dict(context_lens=[0, 1, 31], page_size=32, num_pages=16),
+    dict(B=5, Hq=28, Hkv=4, page_size=32, num_pages=64, context_lens=[100, 64, 0, 255, 31], inactive_rows=(1, 3)),
+    dict(B=2, Hq=32, Hkv=2, context_lens=[500, 77], rope_base=500000.0),
+])
+def test_rope_append_bit_exact(rt, kw):
+    run_and_compare(rt, small(31, **kw))
+
+
+def test_rope_append_bit_exact_with_far_position_angles(rt):
+    # Short contexts keep the pool small; table row p is replaced by the row of a far position
+    # (100000..131071, base 500000: tiny sines, many near-cancellations).  Both sides read this table.
+    rng = np.random.default_rng(7)
+    w = W.make_workload("rope_far", 32, B=64, Hq=32, Hkv=8, d=128, page_size=16, num_pages=400,
+                        context_lens=rng.integers(0, 60, size=64).tolist(), rope_base=500000.0)
+    cos, sin = W.rope_table(131072, 128, 500000.0)
+    far = rng.integers(100000, 131072, size=w.max_position)
+    w.rope_cos = np.ascontiguousarray(cos[far])
+    w.rope_sin = np.ascontiguousarray(sin[far])
+    run_and_compare(rt, w)
+
+
+def test_rope_constructed_near_tie(rt):
+    # x = (1 + 2^-7, 1), c = 1, s = -(2^-8)(1 + 2^-20): exact result just above a bf16 tie
+    import torch
+    w = small(33, B=1, Hq=2, Hkv=2, d=64, context_lens=[5], num_pages=8)
+    w.q[:] = 0x3F80
+    w.q[0, :, :32] = 0x3F81
+    w.k_new[:] = w.q[0]
+    w.rope_cos[:] = 1.0
+    w.rope_sin[:] = np.float32(-(2.0 ** -8) * (1 + 2.0 ** -20))
+    st, _ = run_and_compare(rt, w)
+    assert (rt.bits_of(st.q_rot)[0, :, :32] == 0x3F82).all()
+
+
+def test_append_flags_out_of_range_and_writes_nothing(rt):
+    import torch
+    w = small(34, B=2, context_lens=[40, 50], num_pages=32)
+    st = rt.DecodeStep(w)
+    bt = w.block_table.copy()
+    bt[0, 40 // 16] = 10_000                  # page id outside the pool
+    st.block_table.copy_(torch.from_numpy(bt))
+    lens = w.context_lens.copy()
+    lens[1] = w.max_position + 5               # position outside the rope table
+    st.context_lens.copy_(torch.from_numpy(lens))
+    before_k, before_v = st.cache_bits()
+    st.rope_kv_append()
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) == 3
+    after_k, after_v = st.cache_bits()
+    assert np.array_equal(before_k, after_k) and np.array_equal(before_v, after_v)
+
+
+# ---------------------------------------------------------------------------------------------
+# attention: small shapes spanning several tiles, ragged tails, every group size and layout
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("kw", [
+    dict(),
+    dict(Hq=4, Hkv=4),                                                       # G = 1
+    dict(Hq=28, Hkv=4, page_size=32, num_pages=48),                          # G = 7
+    dict(Hq=16, Hkv=2),                                                      # G = 8
+    dict(Hq=32, Hkv=2),                                                      # G = 16 (two row blocks)
+    dict(Hq=24, Hkv=2, d=64),                                                # G = 12, d = 64
+    dict(d=64, Hq=8, Hkv=2, page_size=64, num_pages=24),
+    dict(context_lens=[0, 15, 16], num_pages=16),                            # one token; tile edges
+    dict(context_lens=[63, 64, 65]),
+    dict(B=4, context_lens=[1000, 3, 511, 700], num_pages=200, inactive_rows=(2,)),
+])
+@pytest.mark.parametrize("splits", [1, 3])
+def test_attention_small(rt, kw, splits):
+    run_and_compare(rt, small(41, **kw), num_splits=splits)
+
+
+@pytest.mark.parametrize("splits", [1, 2, 5, 16])
+def test_attention_split_sweep_and_partials(rt, splits):
+    import torch
+    w = small(42, B=2, context_lens=[900, 257], num_pages=128)
+    st, out_ref = run_and_compare(rt, w, num_splits=splits)
+    if splits > 1:
+        # the workspace format is part of the ABI: compare each split's partial with the oracle's
+        q_rot, k_after, v_after, _ = O.oracle_decode_step(w)
+        starts = [[s * st.split_tokens for s in range(splits + 1)]] * w.B
+        po_ref, pl_ref = O.oracle_split_partials(q_rot, k_after, v_after, w.block_table, w.context_lens,
+                                                 w.page_size, starts)
+        po, pl = st.partials()
+        empty = ~np.isfinite(pl_ref)
+        assert np.array_equal(np.isneginf(pl), empty)
+        assert np.abs(pl[~empty] - pl_ref[~empty]).max() < 2e-2
+        assert np.abs(po[~empty] - po_ref[~empty]).max() < 2e-2
+
+
+def test_merge_kernel_alone_against_oracle(rt):
+    import torch
+    from paper_2606_07665_b200 import binding as ac
+    rng = np.random.default_rng(5)
+    B, Hq, S, d = 3, 5, 7, 128
+    po = rng.standard_normal((B, Hq, S, d)).astype(np.float32)
+    pl = (rng.standard_normal((B, Hq, S)) * 5).astype(np.float32)
+    pl[0, 0, :] = -np.inf                          # a row with nothing to merge
+    pl[1, 2, 3] = -np.inf
+    po[1, 2, 3] = np.nan                           # partial of an empty split must not be read
+    pl[2, 1, :] = [-np.inf] * 6 + [1.5]
+    ws = torch.from_numpy(np.concatenate([po.ravel(), pl.ravel()])).cuda()
+    lens = torch.tensor([5, 5, 5], dtype=torch.int32).cuda()
+    out = torch.full((B, Hq, d), 0x7FC0, dtype=torch.int16).cuda()
+    ac.ac_splitkv_merge(ws, S, lens, out, B, Hq, d)
+    torch.cuda.synchronize()
+    ref, _ = O.oracle_splitkv_merge(np.where(np.isnan(po), 0.0, po), pl)
+    got = W.bf16_bits_to_f32(rt.bits_of(out)).astype(np.float64)
+    assert np.abs(got - ref).max() <= 2.0 ** -8 * max(1.0, np.abs(ref).max())
+    assert (rt.bits_of(out)[0, 0] == 0).all()
+    lens[1] = -1
+    ac.ac_splitkv_merge(ws, S, lens, out, B, Hq, d)
+    torch.cuda.synchronize()
+    assert (rt.bits_of(out)[1] == 0).all()
+
+
+@pytest.mark.parametrize("splits", [1, 4])
+def test_attention_head_major_layout(rt, splits):
+    run_and_compare(rt, small(43, Hq=16, Hkv=4, context_lens=[300, 45, 129]), num_splits=splits,
+                    layout="head_major")
+
+
+def test_single_token_context_returns_v_bits(rt):
+    import torch
+    w = small(44, context_lens=[0, 0, 0], num_pages=8)
+    st, _ = run_and_compare(rt, w, num_splits=1)
+    G = w.Hq // w.Hkv
+    got = rt.bits_of(st.out)
+    for hq in range(w.Hq):
+        assert np.array_equal(got[:, hq], w.v_new[:, hq // G])
+
+
+def test_page_permutation_gives_bit_identical_output(rt):
+    import torch
+    w = small(45, context_lens=[700, 123, 64], num_pages=128)
+    st1, _ = run_and_compare(rt, w, num_splits=3)
+    out1 = rt.bits_of(st1.out).copy()
+    perm = np.random.default_rng(9).permutation(w.num_pages)
+    w2 = W.make_workload("small", 45, B=3, Hq=8, Hkv=2, d=128, page_size=16, num_pages=128,
+                         context_lens=[700, 123, 64], rope_base=10000.0)
+    k2 = np.empty_like(w2.k_cache); v2 = np.empty_like(w2.v_cache)
+    k2[perm] = w2.k_cache; v2[perm] = w2.v_cache
+    w2.k_cache, w2.v_cache = k2, v2
+    w2.block_table = perm[w2.block_table].astype(np.int32)
+    st2 = rt.DecodeStep(w2, num_splits=3)
+    st2.step()
+    torch.cuda.synchronize()
+    assert np.array_equal(out1, rt.bits_of(st2.out))
+
+
+def test_attention_without_new_token_and_deterministic(rt):
+    import torch
+    w = small(46, context_lens=[310, 48, 129], num_pages=64)
+    q_rot, k_after, v_after, _ = O.oracle_decode_step(w)
+    ref = O.oracle_paged_decode_attn(q_rot, w.k_cache, w.v_cache, w.block_table, w.context_lens,
+                                     w.page_size, new_tokens=0)
+    st = rt.DecodeStep(w, num_splits=2)
+    q_dev = torch.from_numpy(q_rot.view(np.int16)).cuda()
+    st.attention(new_tokens=0, q=q_dev)
+    st.merge()
+    torch.cuda.synchronize()
+    check_out(st.out_f64(), ref, "new_tokens=0")
+    first = rt.bits_of(st.out).copy()
+    for _ in range(3):
+        st.attention(new_tokens=0, q=q_dev)
+        st.merge()
+    torch.cuda.synchronize()
+    assert np.array_equal(first, rt.bits_of(st.out))
+
+
+def test_graph_replay_equals_eager_and_tracks_updated_lengths(rt):
+    import torch
+
+    def make():
+        w = small(47, B=4, Hq=28, Hkv=4, page_size=32, num_pages=96, context_lens=[600, 31, 32, 257],
+                  inactive_rows=(1,))
+        w.rope_cos, w.rope_sin = W.rope_table(w.max_position + 4, w.d, w.rope_base)   # room to advance
+        return w
+
+    w = make()
+    st, out_ref = run_and_compare(rt, w, num_splits=2)
+    eager = rt.bits_of(st.out).copy()
+    k_eager, v_eager = st.cache_bits()
+    st2 = rt.DecodeStep(w, num_splits=2, max_context_len=w.max_context_len + 4)
+    graph = st2.capture()
+    # capture ran one eager warm-up step on the same buffers; restore the caches and replay
+    fresh = rt.DecodeStep(w, num_splits=2)
+    st2.k_cache.copy_(fresh.k_cache); st2.v_cache.copy_(fresh.v_cache); st2.out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    check_out(st2.out_f64(), out_ref, "graph replay")
+    k2, v2 = st2.cache_bits()
+    assert np.array_equal(k2, k_eager) and np.array_equal(v2, v_eager)
+    # identical launch configuration replayed eagerly gives identical bits
+    st2.k_cache.copy_(fresh.k_cache); st2.v_cache.copy_(fresh.v_cache)
+    st2.step()
+    torch.cuda.synchronize()
+    eager2 = rt.bits_of(st2.out).copy()
+    st2.k_cache.copy_(fresh.k_cache); st2.v_cache.copy_(fresh.v_cache); st2.out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert np.array_equal(rt.bits_of(st2.out), eager2)
+    # same graph, device-side lengths advanced by one token per active row: still matches the oracle
+    w_next = make()
+    _, k_after, v_after, _ = O.oracle_decode_step(w_next)
+    w_next.k_cache, w_next.v_cache = k_after, v_after
+    w_next.context_lens = np.where(w_next.context_lens >= 0, w_next.context_lens + 1, -1).astype(np.int32)
+    _, _, _, out_next = O.oracle_decode_step(w_next)
+    st2.context_lens.copy_(torch.from_numpy(w_next.context_lens))
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(st2.status_flag.item()) == 0
+    check_out(st2.out_f64(), out_next, "replay with advanced lengths")
+
+
+def test_peaked_scores(rt):
+    w = W.make_workload("peaked", 48, B=2, Hq=16, Hkv=2, d=128, page_size=16, num_pages=300,
+                        context_lens=[2000, 1500], rope_base=500000.0, peak_fraction=0.01)
+    run_and_compare(rt, w, num_splits=4)
+    run_and_compare(rt, w, num_splits=1, check_cache=False)
+
+
+# ---------------------------------------------------------------------------------------------
+# the five benchmark workloads, in the launch configuration the benchmark uses (planned splits)
+# ---------------------------------------------------------------------------------------------
+
+def test_workload_tiny(rt):
+    run_and_compare(rt, W.tiny())
+
+
+def test_workload_single_request(rt):
+    run_and_compare(rt, W.single_request())
+
+
+@pytest.mark.parametrize("batch", W.GRAPH_SWEEP_BATCHES)
+def test_workload_graph_sweep(rt, batch):
+    import torch
+    w = W.graph_sweep(batch)
+    st, out_ref = run_and_compare(rt, w)
+    graph = st.capture()
+    graph.replay()
+    torch.cuda.synchronize()
+    check_out(st.out_f64(), out_ref, "graph replay")
+
+
+def test_workload_continuous_batching(rt):
+    run_and_compare(rt, W.continuous_batching())
+
+
+def test_workload_long_context_sampled_heads(rt):
+    import torch
+    w = W.long_context()
+    st = rt.DecodeStep(w)
+    st.step()
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) == 0
+    # bit-exact append: compare the rotated q and the appended slots, and that nothing else moved
+    q_rot = np.empty_like(w.q)
+    for b in range(w.B):
+        p = int(w.context_lens[b])
+        q_rot[b] = O.rope_rotate_bf16(w.q[b], w.rope_cos[p], w.rope_sin[p])
+    assert np.array_equal(rt.bits_of(st.q_rot), q_rot)
+    k_gpu, v_gpu = st.cache_bits()
+    k_ref, v_ref = w.k_cache, w.v_cache                # patched in place below
+    for b in range(w.B):
+        p = int(w.context_lens[b])
+        pg, sl = int(w.block_table[b, p // w.page_size]), p % w.page_size
+        k_ref[pg, sl] = O.rope_rotate_bf16(w.k_new[b], w.rope_cos[p], w.rope_sin[p])
+        v_ref[pg, sl] = w.v_new[b]
+    assert np.array_equal(k_gpu, k_ref) and np.array_equal(v_gpu, v_ref)
+    # attention on a sample of (request, KV head) pairs, all query heads of the group
+    got = st.out_f64()
+    G = w.Hq // w.Hkv
+    scale = 1.0 / np.sqrt(w.d)
+    gots, refs = [], []
+    for b, h in ((0, 0), (1, 3), (2, 5), (3, 7)):
+        n = int(w.context_lens[b]) + 1
+        K = O.gather_kv(k_ref, w.block_table[b], n, w.page_size, h)
+        V = O.gather_kv(v_ref, w.block_table[b], n, w.page_size, h)
+        for g in range(G):
+            hq = h * G + g
+            s = (K @ O.bf16_to_f64(q_rot[b, hq])) * scale
+            pw = np.exp(s - s.max())
+            ref = pw @ V / pw.sum()
+            refs.append(ref)
+            gots.append(got[b, hq])
+    check_out(np.array(gots), np.array(refs), "long_context sampled heads")
+    assert np.isfinite(got).all()
