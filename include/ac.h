@@ -54,7 +54,8 @@ typedef enum {
     AC_ERR_ALIGN = 4,       /* pointer or stride alignment */
     AC_ERR_WORKSPACE = 5,   /* workspace too small for num_splits */
     AC_ERR_CUDA = 6,        /* a CUDA call failed; see ac_last_cuda_error() */
-    AC_ERR_NOT_INIT = 7     /* ac_init has not succeeded on the current device */
+    AC_ERR_NOT_INIT = 7,    /* ac_init has not succeeded on the current device */
+    AC_ERR_SCRATCH_LIMIT = 8 /* ac_paged_decode_attn_static_scratch: partials exceed AC_STATIC_SCRATCH_BYTES */
 } ac_status;
 
 /* Bits the kernels OR into the optional device word `status_flag` (never cleared by the library). */
@@ -174,6 +175,49 @@ int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* 
                         float softmax_scale, int num_splits, void* workspace, size_t workspace_bytes,
                         int B, int Hq, int Hkv, int d, int page_size, int num_pages,
                         int max_context_len, int32_t* status_flag, void* stream);
+
+/* Size of the library's built-in partial-result array (bytes), held by every GPU that loads the
+ * library until the process exits. */
+#define AC_STATIC_SCRATCH_BYTES (8u << 20)
+
+/* Split-KV attention and merge in one call, for callers that cannot allocate device memory.  (The
+ * paper has no counterpart to this entry point; it exists for the integration cases below.)
+ *
+ * ac_paged_decode_attn needs a workspace for the split partials, which normally means a cudaMalloc
+ * (or a framework allocation) somewhere in the caller.  That is not always possible: an engine that
+ * gave all remaining HBM to its KV-cache pool at start-up has nothing left to ask for; code running
+ * under a host framework that forbids allocation in the serving loop, or that must not take the
+ * driver's allocation lock, cannot call cudaMalloc at all; and a stateless step function has nowhere
+ * to keep a buffer from one call to the next.  This entry point calls no cudaMalloc, cudaFree or
+ * any allocating routine: the partials go into a fixed array inside the library image, of
+ * AC_STATIC_SCRATCH_BYTES bytes per GPU.
+ *
+ * Arguments are those of ac_paged_decode_attn without workspace/workspace_bytes; the caller still
+ * passes every input and the output.  The call runs the attention kernel with num_splits splits
+ * (use ac_decode_plan to choose) and then the merge, both on `stream`, and always writes the final
+ * bf16 rows to out [B,Hq,d].
+ *
+ * Limits and rules
+ *   - B * Hq * num_splits * (d + 1) * 4 bytes must not exceed AC_STATIC_SCRATCH_BYTES, otherwise
+ *     AC_ERR_SCRATCH_LIMIT is returned and nothing is launched.  Lower num_splits, or use
+ *     ac_paged_decode_attn with your own workspace.
+ *   - ac_init must have succeeded on the current device.  The first call on each device also looks
+ *     up the array's device address (once; later calls reuse it): make that first call outside any
+ *     stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call wrote.
+ *     Nothing needs clearing between calls (each call overwrites the log-sum-exp slot of every split
+ *     it uses before reading it, and never reads the partial of a split marked empty), but two calls
+ *     whose kernels overlap on the GPU -- different streams, or different host threads without
+ *     ordering between their streams -- would write the same bytes and corrupt each other.  Order
+ *     them on one stream or with events.
+ *   - Errors are otherwise those of ac_paged_decode_attn and ac_splitkv_merge. */
+int ac_paged_decode_attn_static_scratch(const void* q_rot, const void* k_cache, const void* v_cache,
+                                        int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                                        const int32_t* block_table, int max_pages_per_seq,
+                                        const int32_t* context_lens, int new_tokens,
+                                        float softmax_scale, int num_splits, void* out, int B, int Hq,
+                                        int Hkv, int d, int page_size, int num_pages,
+                                        int max_context_len, int32_t* status_flag, void* stream);
 
 #ifdef __cplusplus
 }

@@ -15,14 +15,16 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libac.so")
 _lib = None
 
 STATUS_NAMES = {0: "AC_OK", 1: "AC_ERR_NULL", 2: "AC_ERR_SHAPE", 3: "AC_ERR_UNSUPPORTED",
-                4: "AC_ERR_ALIGN", 5: "AC_ERR_WORKSPACE", 6: "AC_ERR_CUDA", 7: "AC_ERR_NOT_INIT"}
+                4: "AC_ERR_ALIGN", 5: "AC_ERR_WORKSPACE", 6: "AC_ERR_CUDA", 7: "AC_ERR_NOT_INIT",
+                8: "AC_ERR_SCRATCH_LIMIT"}
 AC_FLAG_PAGE_OOB = 1
 AC_FLAG_POSITION_OOB = 2
 AC_FLAG_WAIT_TIMEOUT = 4
 
 EXPORTS = ("ac_init", "ac_status_string", "ac_last_cuda_error", "ac_sm_count", "ac_decode_plan",
            "ac_split_tokens", "ac_workspace_bytes", "ac_rope_kv_append", "ac_paged_decode_attn",
-           "ac_splitkv_merge", "ac_decode_step_host")
+           "ac_splitkv_merge", "ac_decode_step_host", "ac_paged_decode_attn_static_scratch")
+AC_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class AcError(RuntimeError):
@@ -72,6 +74,10 @@ def lib():
                                           [c_int, c_void_p, c_void_p, c_int, c_float, c_int, c_void_p,
                                            c_size_t] + [c_int] * 7 + [c_void_p, c_void_p])
         L.ac_decode_step_host.restype = c_int
+        L.ac_paged_decode_attn_static_scratch.argtypes = ([c_void_p] * 3 + [c_int64] * 3 + [c_void_p, c_int,
+                                                          c_void_p, c_int, c_float, c_int, c_void_p] +
+                                                          [c_int] * 7 + [c_void_p, c_void_p])
+        L.ac_paged_decode_attn_static_scratch.restype = c_int
         _lib = L
     return _lib
 
@@ -164,3 +170,16 @@ def ac_decode_step_host(q_host, k_new_host, v_new_host, block_table_host, contex
                                      num_splits, _ptr(workspace), workspace_bytes, B, Hq, Hkv, d,
                                      page_size, num_pages, max_context_len, _ptr(status_flag),
                                      _stream(stream)), "ac_decode_step_host")
+
+
+def ac_paged_decode_attn_static_scratch(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head,
+                                        block_table, max_pages_per_seq, context_lens, new_tokens,
+                                        softmax_scale, num_splits, out, B, Hq, Hkv, d, page_size,
+                                        num_pages, max_context_len, status_flag=None, stream=None):
+    """Attention + merge with the split partials in the library's built-in array (no workspace
+    argument, no allocation anywhere in the call); see include/ac.h for the size limit and rules."""
+    _check(lib().ac_paged_decode_attn_static_scratch(
+        _ptr(q_rot), _ptr(k_cache), _ptr(v_cache), stride_page, stride_token, stride_head,
+        _ptr(block_table), max_pages_per_seq, _ptr(context_lens), new_tokens, softmax_scale, num_splits,
+        _ptr(out), B, Hq, Hkv, d, page_size, num_pages, max_context_len, _ptr(status_flag),
+        _stream(stream)), "ac_paged_decode_attn_static_scratch")

@@ -12,7 +12,8 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libac.so")
-SOURCES = ["ac_api.cu", "rope_kv_append.cu", "paged_decode_attn.cu", "splitkv_merge.cu"]
+SOURCES = ["ac_api.cu", "rope_kv_append.cu", "paged_decode_attn.cu", "splitkv_merge.cu",
+           "attn_static_scratch.cu"]
 HEADERS = [os.path.join(CSRC, "ac_device.cuh"), os.path.join(CSRC, "ac_internal.h"),
            os.path.join(ROOT, "include", "ac.h")]
 

@@ -170,6 +170,9 @@ const char* ac_status_string(int status) {
         case AC_ERR_WORKSPACE: return "workspace missing or too small for num_splits";
         case AC_ERR_CUDA: return "a CUDA call failed (see ac_last_cuda_error)";
         case AC_ERR_NOT_INIT: return "ac_init has not succeeded on the current device";
+        case AC_ERR_SCRATCH_LIMIT:
+            return "partials for this B, Hq, d, num_splits exceed the library's built-in scratch "
+                   "(AC_STATIC_SCRATCH_BYTES); use fewer splits or ac_paged_decode_attn with a workspace";
         default: return "unknown status";
     }
 }
