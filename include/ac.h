@@ -79,9 +79,11 @@ int ac_last_cuda_error(void);
 int ac_sm_count(void);
 
 /* Split plan (host only, pure, needs no GPU).  Chooses how many KV splits the attention kernel
- * should use so that B * Hkv * num_splits CTAs fill `sm_count` SMs (<= 0: the count seen by
- * ac_init, or 148 if none) several times over, without making splits shorter than a few hundred
- * tokens.  max_context_len = the largest number of tokens any row attends over in this bucket
+ * should use for `sm_count` SMs (<= 0: the count seen by ac_init, or 148 if none): none when the
+ * (request, KV head) pairs alone fill the GPU and contexts are short, chunks of at most 2560 tokens
+ * when contexts are long, and otherwise the split count with the smallest estimated time from a
+ * small cost model (bandwidth of one CTA, waves of CTAs, partial-result traffic); splits are never
+ * shorter than 256 tokens.  max_context_len = the largest number of tokens any row attends over in this bucket
  * (cached + new).  Outputs: *num_splits_out >= 1, *split_tokens_out = tokens per split (a multiple
  * of 64; split s of row b covers tokens [s*split_tokens, min((s+1)*split_tokens, n_b)) ), and
  * *workspace_bytes_out = bytes of fp32 workspace the attention + merge calls need for that plan
@@ -148,6 +150,30 @@ int ac_paged_decode_attn(const void* q_rot, const void* k_cache, const void* v_c
                          int B, int Hq, int Hkv, int d, int page_size, int num_pages,
                          int max_context_len, int32_t* status_flag, void* stream);
 
+/* A4 + A5 in one launch: the same attention kernel, but the CTA that finishes last for a (request,
+ * KV head) merges that pair's split partials itself and writes the final bf16 rows to out [B,Hq,d]
+ * (the "fused cross-CTA merging" of family (iv); Supplementary Implementation Notes: "a fused
+ * fence-based merge that removes a separate reduction kernel").  Each CTA publishes its partial,
+ * fences, and takes a ticket from a per-(request, KV head) arrival counter; the holder of the last
+ * ticket merges and resets the counter.  No CTA ever waits for another.
+ *
+ * Arguments as ac_paged_decode_attn, except: out is always written; for num_splits > 1 the workspace
+ * must hold ac_fused_workspace_bytes(B,Hq,Hkv,d,num_splits) bytes = the partials followed by int32
+ * arrival counters [B,Hkv], and the counters must be ZERO on entry.  A launch that completes leaves
+ * them zero, so call ac_fused_workspace_reset once after allocating the workspace (and again after
+ * any launch that did not complete).  Results differ from the separate merge only in rounding order
+ * of the fp32 combination; for fixed inputs and num_splits they are deterministic. */
+size_t ac_fused_workspace_bytes(int B, int Hq, int Hkv, int d, int num_splits);
+int ac_fused_workspace_reset(void* workspace, size_t workspace_bytes, int B, int Hq, int Hkv, int d,
+                             int num_splits, void* stream);
+int ac_paged_decode_attn_fused_merge(const void* q_rot, const void* k_cache, const void* v_cache,
+                                     int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                                     const int32_t* block_table, int max_pages_per_seq,
+                                     const int32_t* context_lens, int new_tokens, float softmax_scale,
+                                     int num_splits, void* workspace, size_t workspace_bytes, void* out,
+                                     int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                                     int max_context_len, int32_t* status_flag, void* stream);
+
 /* A5: merge of the split partials ("cross-CTA merging" of family (iv), here as its own kernel):
  *   M = max_s lse_s,  w_s = exp(lse_s - M),  out[b,hq,:] = sum_s w_s partial_o[b,hq,s,:] / sum_s w_s
  * rounded to bf16.  Splits with lse = -inf are skipped (their partial_o is not read); a row whose
@@ -158,9 +184,9 @@ int ac_splitkv_merge(const void* workspace, int num_splits, const int32_t* conte
 
 /* The whole step from HOST buffers (for callers that hold the step's inputs on the host, and for
  * end-to-end timing): copies q/k_new/v_new/block_table/context_lens from the *_host buffers (pinned
- * memory recommended) into the caller's device buffers of the same name, enqueues the three
- * kernels with a plan from ac_decode_plan's rule given (max_context_len, num_splits), and copies the
- * bf16 result from out into out_host.  Everything is asynchronous on `stream`; the caller
+ * memory recommended) into the caller's device buffers of the same name, resets the arrival
+ * counters, enqueues ac_rope_kv_append and ac_paged_decode_attn_fused_merge for the given num_splits
+ * (workspace_bytes >= ac_fused_workspace_bytes), and copies the bf16 result from out into out_host.  Everything is asynchronous on `stream`; the caller
  * synchronises the stream before reading out_host.  The KV cache pools and rope tables stay on the
  * device (they are the layer's resident state, not a per-step input).  No paper counterpart. */
 int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* v_new_host,

@@ -36,7 +36,7 @@ def up_to_date() -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and up_to_date():
         return LIB_PATH
-    cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+    cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-diag-suppress", "550",
            "-shared", "-Xcompiler", "-fPIC", "-cudart", "static",
            "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", LIB_PATH]
     if verbose:

@@ -200,16 +200,41 @@ int ac_decode_plan(int B, int Hq, int Hkv, int d, int page_size, int max_context
     if (max_context_len <= 0) return AC_ERR_SHAPE;
     if (sm_count <= 0) sm_count = g_last_sm_count > 0 ? g_last_sm_count : 148;
 
-    // Two CTAs are resident per SM.  Aim for about four waves of CTAs so the tail of the last wave
-    // stays small, but keep every split at least kMinSplitTokens long so the per-CTA prologue
-    // (barrier set-up, first loads in flight) and the partial-result traffic stay a small fraction.
-    const long long kMinSplitTokens = 256;
-    const long long target_ctas = static_cast<long long>(sm_count) * 2 * 4;
-    const long long base_ctas = static_cast<long long>(B) * Hkv;
-    long long want = (target_ctas + base_ctas - 1) / base_ctas;
-    long long cap = static_cast<long long>(max_context_len) / kMinSplitTokens;
-    if (cap < 1) cap = 1;
-    long long S = want < cap ? want : cap;
+    // Two CTAs are resident per SM ("slots").  Measured on B200: one CTA streams at most ~35 GB/s
+    // (its ring holds 96 KB against ~2.5 us of load latency), a wave of CTAs costs ~3 us of
+    // ramp-up/epilogue that overlaps poorly, and every extra split adds partial-result traffic.
+    //  * At least one wave of (request, KV head) pairs: do not split, unless contexts are long --
+    //    then cut them into chunks of at most 2560 tokens so that ragged batches balance.
+    //  * Fewer pairs than slots: scan the split counts and take the one with the smallest
+    //    estimated time, all rows assumed at max_context_len.
+    const double slots = 2.0 * sm_count;
+    const double hbm = 6.5e12 * sm_count / 148.0;      // bytes/s the whole GPU streams
+    const double cta_rate = 33e9;                       // bytes/s one CTA streams on its own
+    const double wave_cost = 3e-6;
+    const long long pairs = static_cast<long long>(B) * Hkv;
+    long long S = 1;
+    if (pairs >= static_cast<long long>(slots)) {
+        S = (static_cast<long long>(max_context_len) + 2559) / 2560;
+    } else {
+        const int s_max = max_context_len / 256 > 1 ? max_context_len / 256 : 1;
+        double best = 0.0;
+        for (int cand = 1; cand <= s_max && cand <= 4096; ++cand) {
+            const int chunk = split_tokens_for(max_context_len, cand);
+            if (static_cast<long long>(chunk) * (cand - 1) >= max_context_len) continue;   // empty split
+            const double n = static_cast<double>(pairs) * cand;
+            const double c = static_cast<double>(chunk) * d * 4.0;          // K+V bytes of one CTA
+            const double waves = ceil(n / slots);
+            const double last = n - (waves - 1.0) * slots;
+            double t = (waves - 1.0) * slots * c / hbm;
+            const double t_last_bw = last * c / hbm, t_last_cta = c / cta_rate;
+            t += (t_last_bw > t_last_cta ? t_last_bw : t_last_cta) + waves * wave_cost;
+            if (cand > 1) t += 2.0 * B * Hq * cand * (d + 1.0) * 4.0 / hbm + 1e-6;
+            if (best == 0.0 || t < best) {
+                best = t;
+                S = cand;
+            }
+        }
+    }
     if (S < 1) S = 1;
     if (S > 65535) S = 65535;
     int chunk = split_tokens_for(max_context_len, static_cast<int>(S));
@@ -250,13 +275,12 @@ int ac_rope_kv_append(const void* q_in, void* q_out, const void* k_new, const vo
     return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
 }
 
-int ac_paged_decode_attn(const void* q_rot, const void* k_cache, const void* v_cache,
-                         int64_t stride_page, int64_t stride_token, int64_t stride_head,
-                         const int32_t* block_table, int max_pages_per_seq,
-                         const int32_t* context_lens, int new_tokens, float softmax_scale,
-                         int num_splits, void* workspace, size_t workspace_bytes, void* out, int B,
-                         int Hq, int Hkv, int d, int page_size, int num_pages, int max_context_len,
-                         int32_t* status_flag, void* stream) {
+static int attn_common(const void* q_rot, const void* k_cache, const void* v_cache, int64_t stride_page,
+                       int64_t stride_token, int64_t stride_head, const int32_t* block_table,
+                       int max_pages_per_seq, const int32_t* context_lens, int new_tokens,
+                       float softmax_scale, int num_splits, void* workspace, size_t workspace_bytes,
+                       void* out, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                       int max_context_len, int32_t* status_flag, void* stream, bool fused_merge) {
     if (!q_rot || !k_cache || !v_cache || !block_table || !context_lens) return AC_ERR_NULL;
     Shape s{B, Hq, Hkv, d, page_size, num_pages};
     int st = check_shape(s);
@@ -269,14 +293,20 @@ int ac_paged_decode_attn(const void* q_rot, const void* k_cache, const void* v_c
     if (!aligned16(q_rot) || !aligned16(k_cache) || !aligned16(v_cache)) return AC_ERR_ALIGN;
     float* partial_o = nullptr;
     float* partial_lse = nullptr;
-    if (num_splits == 1) {
+    int32_t* arrivals = nullptr;
+    if (num_splits == 1 || fused_merge) {
         if (!out) return AC_ERR_NULL;
         if (!aligned16(out)) return AC_ERR_ALIGN;
-    } else {
-        if (!workspace || workspace_bytes < ac_workspace_bytes(B, Hq, d, num_splits)) return AC_ERR_WORKSPACE;
+    }
+    if (num_splits > 1) {
+        const size_t need = fused_merge ? ac_fused_workspace_bytes(B, Hq, Hkv, d, num_splits)
+                                        : ac_workspace_bytes(B, Hq, d, num_splits);
+        if (!workspace || workspace_bytes < need) return AC_ERR_WORKSPACE;
         if (!aligned16(workspace)) return AC_ERR_ALIGN;
         partial_o = static_cast<float*>(workspace);
         partial_lse = partial_o + static_cast<size_t>(B) * Hq * num_splits * d;
+        if (fused_merge)
+            arrivals = reinterpret_cast<int32_t*>(partial_lse + static_cast<size_t>(B) * Hq * num_splits);
     }
     int dev;
     st = current_ready_device(&dev);
@@ -291,10 +321,53 @@ int ac_paged_decode_attn(const void* q_rot, const void* k_cache, const void* v_c
     const int split_tokens = split_tokens_for(max_context_len, num_splits);
     cudaError_t e = launch_paged_decode_attn(k_map, v_map, head_first, q_rot, block_table,
                                              max_pages_per_seq, context_lens, new_tokens, scale,
-                                             num_splits, split_tokens, partial_o, partial_lse, out, B,
-                                             Hq, Hkv, d, page_size, status_flag,
+                                             num_splits, split_tokens, partial_o, partial_lse, arrivals,
+                                             out, B, Hq, Hkv, d, page_size, status_flag,
                                              static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
+}
+
+size_t ac_fused_workspace_bytes(int B, int Hq, int Hkv, int d, int num_splits) {
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || d <= 0 || num_splits <= 1) return 0;
+    return ac_workspace_bytes(B, Hq, d, num_splits) + static_cast<size_t>(B) * Hkv * sizeof(int32_t);
+}
+
+int ac_fused_workspace_reset(void* workspace, size_t workspace_bytes, int B, int Hq, int Hkv, int d,
+                             int num_splits, void* stream) {
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || d <= 0 || num_splits <= 0) return AC_ERR_SHAPE;
+    if (num_splits == 1) return AC_OK;                       // nothing to reset
+    if (!workspace || workspace_bytes < ac_fused_workspace_bytes(B, Hq, Hkv, d, num_splits))
+        return AC_ERR_WORKSPACE;
+    char* counters = static_cast<char*>(workspace) + ac_workspace_bytes(B, Hq, d, num_splits);
+    cudaError_t e = cudaMemsetAsync(counters, 0, static_cast<size_t>(B) * Hkv * sizeof(int32_t),
+                                    static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
+}
+
+int ac_paged_decode_attn(const void* q_rot, const void* k_cache, const void* v_cache,
+                         int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                         const int32_t* block_table, int max_pages_per_seq,
+                         const int32_t* context_lens, int new_tokens, float softmax_scale,
+                         int num_splits, void* workspace, size_t workspace_bytes, void* out, int B,
+                         int Hq, int Hkv, int d, int page_size, int num_pages, int max_context_len,
+                         int32_t* status_flag, void* stream) {
+    return attn_common(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
+                       max_pages_per_seq, context_lens, new_tokens, softmax_scale, num_splits, workspace,
+                       workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages, max_context_len,
+                       status_flag, stream, false);
+}
+
+int ac_paged_decode_attn_fused_merge(const void* q_rot, const void* k_cache, const void* v_cache,
+                                     int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                                     const int32_t* block_table, int max_pages_per_seq,
+                                     const int32_t* context_lens, int new_tokens, float softmax_scale,
+                                     int num_splits, void* workspace, size_t workspace_bytes, void* out,
+                                     int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                                     int max_context_len, int32_t* status_flag, void* stream) {
+    return attn_common(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
+                       max_pages_per_seq, context_lens, new_tokens, softmax_scale, num_splits, workspace,
+                       workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages, max_context_len,
+                       status_flag, stream, true);
 }
 
 int ac_splitkv_merge(const void* workspace, int num_splits, const int32_t* context_lens, void* out,
@@ -330,12 +403,15 @@ int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* 
     int st = check_shape(s);
     if (st != AC_OK) return st;
     if (max_pages_per_seq <= 0) return AC_ERR_SHAPE;
-    if (num_splits > 1 && (!workspace || workspace_bytes < ac_workspace_bytes(B, Hq, d, num_splits)))
+    if (num_splits > 1 &&
+        (!workspace || workspace_bytes < ac_fused_workspace_bytes(B, Hq, Hkv, d, num_splits)))
         return AC_ERR_WORKSPACE;
     int dev;
     st = current_ready_device(&dev);
     if (st != AC_OK) return st;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    st = ac_fused_workspace_reset(workspace, workspace_bytes, B, Hq, Hkv, d, num_splits, stream);
+    if (st != AC_OK) return st;
     const size_t q_bytes = static_cast<size_t>(B) * Hq * d * 2;
     const size_t kv_bytes = static_cast<size_t>(B) * Hkv * d * 2;
     cudaError_t e;
@@ -352,15 +428,11 @@ int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* 
                            block_table, max_pages_per_seq, context_lens, rope_cos, rope_sin,
                            max_position, B, Hq, Hkv, d, page_size, num_pages, status_flag, stream);
     if (st != AC_OK) return st;
-    st = ac_paged_decode_attn(q, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
-                              max_pages_per_seq, context_lens, 1, softmax_scale, num_splits, workspace,
-                              workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages,
-                              max_context_len, status_flag, stream);
+    st = ac_paged_decode_attn_fused_merge(q, k_cache, v_cache, stride_page, stride_token, stride_head,
+                                          block_table, max_pages_per_seq, context_lens, 1, softmax_scale,
+                                          num_splits, workspace, workspace_bytes, out, B, Hq, Hkv, d,
+                                          page_size, num_pages, max_context_len, status_flag, stream);
     if (st != AC_OK) return st;
-    if (num_splits > 1) {
-        st = ac_splitkv_merge(workspace, num_splits, context_lens, out, B, Hq, d, stream);
-        if (st != AC_OK) return st;
-    }
     e = cudaMemcpyAsync(out_host, out, q_bytes, cudaMemcpyDeviceToHost, cs);
     return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
 }

@@ -49,8 +49,9 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
                                      const int32_t* block_table, int max_pages_per_seq,
                                      const int32_t* context_lens, int new_tokens, float scale,
                                      int num_splits, int split_tokens, float* partial_o,
-                                     float* partial_lse, void* out, int B, int Hq, int Hkv, int d,
-                                     int page_size, int32_t* status_flag, cudaStream_t stream);
+                                     float* partial_lse, int32_t* arrivals, void* out, int B, int Hq,
+                                     int Hkv, int d, int page_size, int32_t* status_flag,
+                                     cudaStream_t stream);
 cudaError_t launch_splitkv_merge(const float* partial_o, const float* partial_lse, int num_splits,
                                  const int32_t* context_lens, void* out, int B, int Hq, int d,
                                  cudaStream_t stream);

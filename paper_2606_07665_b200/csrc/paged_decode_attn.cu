@@ -56,6 +56,7 @@ struct AttnParams {
     float* partial_lse;           // [B, Hq, S]      (S > 1)
     uint16_t* out;                // [B, Hq, D] bf16 (S == 1)
     int32_t* status_flag;
+    int32_t* arrivals;            // [B, Hkv] arrival counters, zero on entry (fused merge only)
     float scale_log2;             // softmax scale * log2(e)
     int max_pages_per_seq;
     int new_tokens;
@@ -63,6 +64,7 @@ struct AttnParams {
     int split_tokens;
     int Hq, Hkv, page_size;
     int head_before_token;        // order of the two middle tensor-map coordinates
+    int fused_merge;              // 1: the last CTA of a (request, KV head) merges the splits itself
 };
 
 template <int D, bool WIDE>
@@ -79,24 +81,45 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     uint8_t* smem_gen = smem_raw + (smem_base - smem_addr(smem_raw));
 
     const int h = blockIdx.x;
-    const int split = blockIdx.y;
-    const int b = blockIdx.z;
+    const int b = blockIdx.y;
+    const int split = blockIdx.z;
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int G = p.Hq / p.Hkv;
     const int S = p.num_splits;
 
+    // Everything up to the first read of q or of the slot that holds the new token is independent of
+    // the kernel that precedes this one in the stream (normally the RoPE + append kernel), so with a
+    // programmatic dependent launch it overlaps that kernel's execution.
+    const int tok_begin = split * p.split_tokens;
+    const int tile_begin = tok_begin / TILE;
+    auto tile_token0 = [&](int j) { return (tile_begin + warp + j * WARPS) * TILE; };
+    const int32_t* bt_row = p.block_table + static_cast<size_t>(b) * p.max_pages_per_seq;
+    auto load_page_id = [&](int j) {
+        const int idx = tile_token0(j) / p.page_size;
+        return idx < p.max_pages_per_seq ? bt_row[idx] : -1;
+    };
+
     const int ctx = p.context_lens[b];
+    int page_first[STAGES];                       // page ids of the first tiles, fetched alongside ctx
+#pragma unroll
+    for (int s = 0; s < STAGES; ++s) page_first[s] = load_page_id(s);
+
     int n_tokens = ctx < 0 ? 0 : ctx + p.new_tokens;
     n_tokens = min(n_tokens, p.max_pages_per_seq * p.page_size);
-    const int tok_begin = split * p.split_tokens;
     const int tok_end = min(tok_begin + p.split_tokens, n_tokens);
 
     if (tok_begin >= tok_end) {
-        // Nothing to attend over in this split.
+        // Nothing to attend over in this split.  The buffers written here may still be in use by
+        // the preceding kernel (a merge of the previous step, say), so wait for it first.
+        cudaGridDependencySynchronize();
         if (S > 1) {
-            if (threadIdx.x < G)
+            if (!p.fused_merge && threadIdx.x < G)
                 p.partial_lse[(static_cast<size_t>(b) * p.Hq + h * G + threadIdx.x) * S + split] = -INFINITY;
+            if (p.fused_merge && split == 0) {   // a row with no tokens at all: its output is +0
+                uint16_t* o = p.out + (static_cast<size_t>(b) * p.Hq + h * G) * D;
+                for (int e = threadIdx.x; e < G * D; e += THREADS) o[e] = 0;
+            }
         } else {
             uint16_t* o = p.out + (static_cast<size_t>(b) * p.Hq + h * G) * D;
             for (int e = threadIdx.x; e < G * D; e += THREADS) o[e] = 0;
@@ -115,14 +138,13 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     }
     __syncwarp();
 
-    const int tile_begin = tok_begin / TILE;
     const int n_tiles = (tok_end - tok_begin + TILE - 1) / TILE;
     const int n_my = n_tiles > warp ? (n_tiles - warp + WARPS - 1) / WARPS : 0;
-    const int32_t* bt_row = p.block_table + static_cast<size_t>(b) * p.max_pages_per_seq;
     const uint64_t policy = l2_policy_evict_first();
+    // The tile that holds the token appended by the preceding kernel (if any) must not be fetched
+    // before that kernel has completed.
+    const int new_token_tile = p.new_tokens > 0 ? ctx / TILE : -1;
 
-    auto tile_token0 = [&](int j) { return (tile_begin + warp + j * WARPS) * TILE; };
-    auto load_page_id = [&](int j) { return bt_row[tile_token0(j) / p.page_size]; };
     auto issue = [&](int j, int page) {      // lane 0 only
         const int tok0 = tile_token0(j);
         const int slot = tok0 % p.page_size;
@@ -142,12 +164,20 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
 
     // ---- prologue: fill the ring -------------------------------------------------------------
     int issued = 0;
-    int page_next = n_my > 0 ? load_page_id(0) : 0;
-    for (; issued < STAGES && issued < n_my; ++issued) {
-        const int page = page_next;
-        page_next = issued + 1 < n_my ? load_page_id(issued + 1) : 0;
-        if (lane == 0) issue(issued, page);
+    bool dependency_met = false;
+#pragma unroll
+    for (int s = 0; s < STAGES; ++s) {
+        if (s < n_my) {
+            if (!dependency_met && tile_begin + warp + s * WARPS == new_token_tile) {
+                cudaGridDependencySynchronize();
+                dependency_met = true;
+            }
+            if (lane == 0) issue(s, page_first[s]);
+            issued = s + 1;
+        }
     }
+    int page_next = issued < n_my ? load_page_id(issued) : 0;
+    if (!dependency_met) cudaGridDependencySynchronize();      // q was written by the preceding kernel
 
     // ---- query fragments (A operand of Q K^T), rows = heads of the group ---------------------------
     const int g = lane >> 2;
@@ -305,10 +335,11 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     // ---- combine the warps' partial results through shared memory ----------------------------------
     // Each warp reuses the start of its own ring (all of its loads have completed).
     constexpr int WROWS = 8 * ROWS;
-    float* wo = reinterpret_cast<float*>(smem_gen + warp * L::RING_BYTES);     // [WROWS][D]
-    float* wm = wo + WROWS * D;                                                 // [WROWS]
+    constexpr int WSTRIDE = D + 8;            // +8 floats: the 8-byte stores of a half-warp hit 32 banks
+    float* wo = reinterpret_cast<float*>(smem_gen + warp * L::RING_BYTES);     // [WROWS][WSTRIDE]
+    float* wm = wo + WROWS * WSTRIDE;                                           // [WROWS]
     float* wl = wm + WROWS;                                                     // [WROWS]
-    static_assert((WROWS * D + 2 * WROWS) * 4 <= L::RING_BYTES, "merge scratch must fit in a ring");
+    static_assert((WROWS * WSTRIDE + 2 * WROWS) * 4 <= L::RING_BYTES, "merge scratch must fit in a ring");
 #pragma unroll
     for (int r = 0; r < ROWS; ++r) {
         float l = l_run[r];
@@ -321,7 +352,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
         }
 #pragma unroll
         for (int nt = 0; nt < NTILES; ++nt)
-            *reinterpret_cast<float2*>(wo + row * D + nt * 8 + 2 * t) = make_float2(o[nt][2 * r], o[nt][2 * r + 1]);
+            *reinterpret_cast<float2*>(wo + row * WSTRIDE + nt * 8 + 2 * t) = make_float2(o[nt][2 * r], o[nt][2 * r + 1]);
     }
     __syncthreads();
 
@@ -332,7 +363,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
         float M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < WARPS; ++w) {
-            mw[w] = reinterpret_cast<const float*>(smem_gen + w * L::RING_BYTES)[WROWS * D + row];
+            mw[w] = reinterpret_cast<const float*>(smem_gen + w * L::RING_BYTES)[WROWS * WSTRIDE + row];
             M = fmaxf(M, mw[w]);
         }
         float num = 0.0f, den = 0.0f;
@@ -340,8 +371,8 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
         for (int w = 0; w < WARPS; ++w) {
             const float* base = reinterpret_cast<const float*>(smem_gen + w * L::RING_BYTES);
             const float wgt = exp2f(mw[w] - M);                 // 0 for a warp that saw no tile
-            num = fmaf(wgt, base[row * D + col], num);
-            den = fmaf(wgt, base[WROWS * D + WROWS + row], den);
+            num = fmaf(wgt, base[row * WSTRIDE + col], num);
+            den = fmaf(wgt, base[WROWS * WSTRIDE + WROWS + row], den);
         }
         const float val = num / den;
         const size_t hq = static_cast<size_t>(b) * p.Hq + h * G + row;
@@ -352,14 +383,99 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
             if (col == 0) p.partial_lse[hq * S + split] = (M + log2f(den)) * LN2;
         }
     }
+
+    if (S == 1 || !p.fused_merge) return;
+
+    // ---- fused merge: the CTA that arrives last for this (request, KV head) combines the splits ----
+    // Publish this CTA's partials, take a ticket, and let the holder of the last ticket do the merge.
+    // Nobody waits for anybody: CTAs that are not last simply exit.
+    __shared__ int s_is_last;
+    const int n_active = (n_tokens + p.split_tokens - 1) / p.split_tokens;     // splits with tokens
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int32_t* counter = p.arrivals + static_cast<size_t>(b) * p.Hkv + h;
+        const int ticket = atomicAdd(counter, 1);
+        s_is_last = ticket == n_active - 1;
+        if (s_is_last) *counter = 0;             // leave the counter ready for the next launch
+    }
+    __syncthreads();
+    if (!s_is_last) return;
+    __threadfence();
+    // The rings are idle now (every warp passed the barriers above): stage the log-sum-exps of the
+    // G rows there so that each thread reads them from shared memory, then stream the partials with
+    // four independent 16-byte loads in flight per thread.
+    constexpr int LSE_CAPACITY = L::RING_BYTES / 4;
+    float* s_lse = reinterpret_cast<float*>(smem_gen);
+    const size_t hq0 = static_cast<size_t>(b) * p.Hq + h * G;
+    const bool staged = G * n_active <= LSE_CAPACITY;
+    if (staged) {
+        for (int i = threadIdx.x; i < G * n_active; i += THREADS) {
+            const int row = i / n_active;
+            s_lse[i] = __ldcg(p.partial_lse + (hq0 + row) * S + (i - row * n_active));
+        }
+        __syncthreads();
+    }
+    constexpr int D4 = D / 4;
+    for (int e = threadIdx.x; e < G * D4; e += THREADS) {
+        const int row = e / D4;
+        const int c4 = e - row * D4;
+        const float* lse_g = p.partial_lse + (hq0 + row) * S;
+        auto lse_at = [&](int sidx) { return staged ? s_lse[row * n_active + sidx] : __ldcg(lse_g + sidx); };
+        float M = -INFINITY;
+        for (int sidx = 0; sidx < n_active; ++sidx) M = fmaxf(M, lse_at(sidx));
+        const float4* po = reinterpret_cast<const float4*>(p.partial_o + (hq0 + row) * S * D) + c4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float den = 0.0f;
+        int sidx = 0;
+        for (; sidx + 4 <= n_active; sidx += 4) {
+            float4 v[4];
+            float wgt[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = __ldcg(po + static_cast<size_t>(sidx + u) * D4);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) wgt[u] = __expf(lse_at(sidx + u) - M);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                acc.x = fmaf(wgt[u], v[u].x, acc.x);
+                acc.y = fmaf(wgt[u], v[u].y, acc.y);
+                acc.z = fmaf(wgt[u], v[u].z, acc.z);
+                acc.w = fmaf(wgt[u], v[u].w, acc.w);
+                den += wgt[u];
+            }
+        }
+        for (; sidx < n_active; ++sidx) {
+            const float4 v = __ldcg(po + static_cast<size_t>(sidx) * D4);
+            const float wgt = __expf(lse_at(sidx) - M);
+            acc.x = fmaf(wgt, v.x, acc.x);
+            acc.y = fmaf(wgt, v.y, acc.y);
+            acc.z = fmaf(wgt, v.z, acc.z);
+            acc.w = fmaf(wgt, v.w, acc.w);
+            den += wgt;
+        }
+        const float inv = 1.0f / den;
+        *reinterpret_cast<uint2*>(p.out + (hq0 + row) * D + c4 * 4) =
+            make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
+    }
 }
 
 template <int D, bool WIDE>
 cudaError_t launch_one(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnParams& p, int B,
                        cudaStream_t stream) {
-    dim3 grid(p.Hkv, p.num_splits, B);
-    paged_decode_attn_kernel<D, WIDE><<<grid, THREADS, Smem<D>::TOTAL, stream>>>(k_map, v_map, p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.Hkv, B, p.num_splits);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = Smem<D>::TOTAL;
+    cfg.stream = stream;
+    // Programmatic dependent launch: this kernel may start while the preceding kernel of the
+    // stream is still running; it calls cudaGridDependencySynchronize() before touching anything
+    // that kernel produces.
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, paged_decode_attn_kernel<D, WIDE>, k_map, v_map, p);
 }
 
 }  // namespace
@@ -384,9 +500,12 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
                                      const int32_t* block_table, int max_pages_per_seq,
                                      const int32_t* context_lens, int new_tokens, float scale,
                                      int num_splits, int split_tokens, float* partial_o,
-                                     float* partial_lse, void* out, int B, int Hq, int Hkv, int d,
-                                     int page_size, int32_t* status_flag, cudaStream_t stream) {
+                                     float* partial_lse, int32_t* arrivals, void* out, int B, int Hq,
+                                     int Hkv, int d, int page_size, int32_t* status_flag,
+                                     cudaStream_t stream) {
     AttnParams p;
+    p.arrivals = arrivals;
+    p.fused_merge = arrivals != nullptr ? 1 : 0;
     p.q = static_cast<const uint16_t*>(q_rot);
     p.block_table = block_table;
     p.context_lens = context_lens;

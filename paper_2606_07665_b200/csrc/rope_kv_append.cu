@@ -41,6 +41,9 @@ __global__ void __launch_bounds__(128) rope_kv_append_kernel(
     int max_pages_per_seq, const int32_t* __restrict__ context_lens,
     const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, int max_position, int B,
     int Hq, int Hkv, int page_size, int num_pages, int32_t* status_flag) {
+    // Let a dependent kernel (the attention launch that follows) begin its own set-up right away; it
+    // synchronises on this grid's completion before reading anything written here.
+    cudaTriggerProgrammaticLaunchCompletion();
     constexpr int HALF = D / 2;
     constexpr int THREADS_PER_VEC = HALF / 8;            // 8 (D=128) or 4 (D=64)
     const int heads = Hq + Hkv;

@@ -29,8 +29,9 @@ class DecodeStep:
     """
 
     def __init__(self, w, device="cuda:0", num_splits: int | None = None, layout: str = "token_major",
-                 max_context_len: int | None = None):
+                 max_context_len: int | None = None, fused_merge: bool = True):
         self.w = w
+        self.fused_merge = bool(fused_merge)
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         ac.ac_init(self.device.index if self.device.index is not None else -1)
@@ -71,9 +72,13 @@ class DecodeStep:
                                                  self.max_context_len, ac.ac_sm_count())
         self.num_splits = int(num_splits)
         self.split_tokens = ac.ac_split_tokens(self.max_context_len, self.num_splits)
-        self.workspace_bytes = ac.ac_workspace_bytes(self.B, self.Hq, self.d, self.num_splits)
+        # sized for either merge flavour: partials, then the fused path's arrival counters
+        self.workspace_bytes = ac.ac_fused_workspace_bytes(self.B, self.Hq, self.Hkv, self.d,
+                                                           self.num_splits)
         self.workspace = (torch.empty(max(self.workspace_bytes, 16) // 4, dtype=torch.float32,
                                       device=self.device))
+        ac.ac_fused_workspace_reset(self.workspace, self.workspace_bytes, self.B, self.Hq, self.Hkv,
+                                    self.d, self.num_splits)
 
     # -- the three calls -----------------------------------------------------------------------
     def rope_kv_append(self, stream=None) -> None:
@@ -84,7 +89,8 @@ class DecodeStep:
                              self.num_pages, self.status_flag, stream)
 
     def attention(self, stream=None, new_tokens: int = 1, q=None) -> None:
-        ac.ac_paged_decode_attn(self.q_rot if q is None else q, self.k_cache, self.v_cache,
+        fn = ac.ac_paged_decode_attn_fused_merge if self.fused_merge else ac.ac_paged_decode_attn
+        fn(self.q_rot if q is None else q, self.k_cache, self.v_cache,
                                 self.stride_page, self.stride_token, self.stride_head, self.block_table,
                                 self.w.max_pages_per_seq, self.context_lens, new_tokens, 0.0,
                                 self.num_splits, self.workspace if self.num_splits > 1 else None,
@@ -92,7 +98,7 @@ class DecodeStep:
                                 self.ps, self.num_pages, self.max_context_len, self.status_flag, stream)
 
     def merge(self, stream=None) -> None:
-        if self.num_splits > 1:
+        if self.num_splits > 1 and not self.fused_merge:
             ac.ac_splitkv_merge(self.workspace, self.num_splits, self.context_lens, self.out, self.B,
                                 self.Hq, self.d, stream)
 
@@ -103,7 +109,7 @@ class DecodeStep:
 
     @property
     def launches_per_step(self) -> int:
-        return 3 if self.num_splits > 1 else 2
+        return 3 if (self.num_splits > 1 and not self.fused_merge) else 2
 
     def capture(self) -> torch.cuda.CUDAGraph:
         """Record one step into a CUDA graph (one graph per batch-size bucket in a serving loop)."""

@@ -42,10 +42,10 @@ def check_out(got, ref, what=""):
     return worst
 
 
-def run_and_compare(rt, w, num_splits=None, layout="token_major", check_cache=True):
+def run_and_compare(rt, w, num_splits=None, layout="token_major", check_cache=True, fused=True):
     import torch
     q_rot, k_after, v_after, out_ref = O.oracle_decode_step(w)
-    st = rt.DecodeStep(w, num_splits=num_splits, layout=layout)
+    st = rt.DecodeStep(w, num_splits=num_splits, layout=layout, fused_merge=fused)
     st.step()
     torch.cuda.synchronize()
     assert int(st.status_flag.item()) == 0
@@ -54,8 +54,8 @@ def run_and_compare(rt, w, num_splits=None, layout="token_major", check_cache=Tr
         k_gpu, v_gpu = st.cache_bits()
         assert np.array_equal(k_gpu, k_after), "K pool differs"
         assert np.array_equal(v_gpu, v_after), "V pool differs"
-    worst = check_out(st.out_f64(), out_ref, f"{w.name} S={st.num_splits} {layout}")
-    print(f"[parity] {w.name} S={st.num_splits} {layout}: worst err/bound = {worst:.3f}")
+    worst = check_out(st.out_f64(), out_ref, f"{w.name} S={st.num_splits} {layout} fused={fused}")
+    print(f"[parity] {w.name} S={st.num_splits} {layout} fused={fused}: worst err/bound = {worst:.3f}")
     return st, out_ref
 
 
@@ -141,16 +141,17 @@ def test_append_flags_out_of_range_and_writes_nothing(rt):
     dict(context_lens=[63, 64, 65]),
     dict(B=4, context_lens=[1000, 3, 511, 700], num_pages=200, inactive_rows=(2,)),
 ])
-@pytest.mark.parametrize("splits", [1, 3])
-def test_attention_small(rt, kw, splits):
-    run_and_compare(rt, small(41, **kw), num_splits=splits)
+@pytest.mark.parametrize("splits,fused", [(1, True), (3, True), (3, False)])
+def test_attention_small(rt, kw, splits, fused):
+    run_and_compare(rt, small(41, **kw), num_splits=splits, fused=fused)
 
 
 @pytest.mark.parametrize("splits", [1, 2, 5, 16])
 def test_attention_split_sweep_and_partials(rt, splits):
     import torch
     w = small(42, B=2, context_lens=[900, 257], num_pages=128)
-    st, out_ref = run_and_compare(rt, w, num_splits=splits)
+    run_and_compare(rt, w, num_splits=splits, fused=True)
+    st, out_ref = run_and_compare(rt, w, num_splits=splits, fused=False)
     if splits > 1:
         # the workspace format is part of the ABI: compare each split's partial with the oracle's
         q_rot, k_after, v_after, _ = O.oracle_decode_step(w)
@@ -190,10 +191,10 @@ def test_merge_kernel_alone_against_oracle(rt):
     assert (rt.bits_of(out)[1] == 0).all()
 
 
-@pytest.mark.parametrize("splits", [1, 4])
-def test_attention_head_major_layout(rt, splits):
+@pytest.mark.parametrize("splits,fused", [(1, True), (4, True), (4, False)])
+def test_attention_head_major_layout(rt, splits, fused):
     run_and_compare(rt, small(43, Hq=16, Hkv=4, context_lens=[300, 45, 129]), num_splits=splits,
-                    layout="head_major")
+                    layout="head_major", fused=fused)
 
 
 def test_single_token_context_returns_v_bits(rt):
@@ -319,8 +320,28 @@ def test_workload_graph_sweep(rt, batch):
     check_out(st.out_f64(), out_ref, "graph replay")
 
 
-def test_workload_continuous_batching(rt):
-    run_and_compare(rt, W.continuous_batching())
+@pytest.mark.parametrize("fused", [True, False])
+def test_workload_continuous_batching(rt, fused):
+    run_and_compare(rt, W.continuous_batching(), fused=fused)
+
+
+def test_fused_merge_repeated_launches_and_row_without_tokens(rt):
+    # The arrival counters reset themselves: many launches on one workspace stay correct, also when a
+    # row has no tokens at all (its output is +0) and when most splits of a short row are empty.
+    import torch
+    w = small(49, B=4, Hq=16, Hkv=2, context_lens=[1500, 10, 700, 64], num_pages=200, inactive_rows=(3,))
+    q_rot, k_after, v_after, out_ref = O.oracle_decode_step(w)
+    st = rt.DecodeStep(w, num_splits=6, fused_merge=True)
+    st.rope_kv_append()
+    for i in range(20):
+        st.out.fill_(0x7FC0)
+        st.attention()
+        torch.cuda.synchronize()
+        check_out(st.out_f64(), out_ref, f"fused launch {i}")
+    assert (rt.bits_of(st.out)[3] == 0).all()
+    n = st.B * st.Hq * st.num_splits * (st.d + 1)
+    counters = st.workspace.view(torch.int32)[n:n + st.B * st.Hkv]
+    assert int(counters.abs().sum().item()) == 0
 
 
 def test_workload_long_context_sampled_heads(rt):

@@ -19,7 +19,7 @@ pytestmark = pytest.mark.gpu
 
 
 def _both_paths(runner, ac, torch, w, num_splits):
-    st = runner.DecodeStep(w, num_splits=num_splits)
+    st = runner.DecodeStep(w, num_splits=num_splits, fused_merge=False)
     st.rope_kv_append()
     st.attention()
     st.merge()
