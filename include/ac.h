@@ -30,8 +30,8 @@
  *   - Return value: AC_OK (0) or an ac_status > 0.  On any non-zero return nothing was launched.
  *     The library never throws, aborts or exits.
  *   - Supported: head_dim d in {64, 128}; page_size a multiple of 16, <= 256; Hq % Hkv == 0 and
- *     Hq / Hkv <= 16; all base pointers 16-byte aligned; cache strides multiples of 8 elements, and
- *     of stride_token / stride_head the larger one a multiple of the smaller one.
+ *     Hq / Hkv <= 16; all base pointers 16-byte aligned; cache strides multiples of 8 elements and
+ *     stride_token, stride_head >= d.
  *   - Rows with context_lens[b] < 0 are inactive (batch padding up to a graph bucket): nothing is
  *     written to the cache for them and their output row is +0.
  *   - Query head hq reads KV head hq / (Hq / Hkv).

@@ -38,11 +38,7 @@ int check_shape(const Shape& s) {
 int check_strides(const Shape& s, int64_t stride_page, int64_t stride_token, int64_t stride_head) {
     if (stride_page <= 0 || stride_token <= 0 || stride_head <= 0) return AC_ERR_SHAPE;
     if (stride_page % 8 || stride_token % 8 || stride_head % 8) return AC_ERR_ALIGN;
-    if (stride_token < s.d && stride_head < s.d) return AC_ERR_SHAPE;
-    const int64_t lo = stride_token < stride_head ? stride_token : stride_head;
-    const int64_t hi = stride_token < stride_head ? stride_head : stride_token;
-    if (lo < s.d) return AC_ERR_SHAPE;
-    if (hi % lo != 0 || stride_page % hi != 0) return AC_ERR_UNSUPPORTED;
+    if (stride_token < s.d || stride_head < s.d) return AC_ERR_SHAPE;
     return AC_OK;
 }
 
@@ -55,30 +51,19 @@ int current_ready_device(int* device_out) {
     return AC_OK;
 }
 
-// 4-D view of one cache pool for 16-token x 64-element box loads.  Dimensions are ordered by
-// increasing stride: head_dim, then head and token-in-page (whichever has the smaller stride first),
-// then page.
+// 5-D view of one cache pool for box loads of 16 tokens x head_dim of one head:
+// (64 elements, token-in-page, 64-element block of head_dim, head, page).  The block dimension has a
+// 128-byte stride, smaller than the token stride before it: tensor-map strides need not be ordered.
 int make_cache_map(CUtensorMap* map, const void* base, const Shape& s, int64_t stride_page,
-                   int64_t stride_token, int64_t stride_head, bool* head_before_token) {
-    const bool head_first = stride_head <= stride_token;
-    *head_before_token = head_first;
-    cuuint64_t dims[4];
-    cuuint64_t strides[3];
-    cuuint32_t box[4];
-    cuuint32_t elem_strides[4] = {1, 1, 1, 1};
-    dims[0] = static_cast<cuuint64_t>(s.d);
-    box[0] = 64;
-    if (head_first) {
-        dims[1] = s.Hkv;        strides[0] = static_cast<cuuint64_t>(stride_head) * 2;   box[1] = 1;
-        dims[2] = s.page_size;  strides[1] = static_cast<cuuint64_t>(stride_token) * 2;  box[2] = 16;
-    } else {
-        dims[1] = s.page_size;  strides[0] = static_cast<cuuint64_t>(stride_token) * 2;  box[1] = 16;
-        dims[2] = s.Hkv;        strides[1] = static_cast<cuuint64_t>(stride_head) * 2;   box[2] = 1;
-    }
-    dims[3] = s.num_pages;
-    strides[2] = static_cast<cuuint64_t>(stride_page) * 2;
-    box[3] = 1;
-    CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
+                   int64_t stride_token, int64_t stride_head) {
+    cuuint64_t dims[5] = {64, static_cast<cuuint64_t>(s.page_size), static_cast<cuuint64_t>(s.d / 64),
+                          static_cast<cuuint64_t>(s.Hkv), static_cast<cuuint64_t>(s.num_pages)};
+    cuuint64_t strides[4] = {static_cast<cuuint64_t>(stride_token) * 2, 128,
+                             static_cast<cuuint64_t>(stride_head) * 2,
+                             static_cast<cuuint64_t>(stride_page) * 2};
+    cuuint32_t box[5] = {64, 16, static_cast<cuuint32_t>(s.d / 64), 1, 1};
+    cuuint32_t elem_strides[5] = {1, 1, 1, 1, 1};
+    CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims,
                                 strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -312,14 +297,13 @@ static int attn_common(const void* q_rot, const void* k_cache, const void* v_cac
     st = current_ready_device(&dev);
     if (st != AC_OK) return st;
     CUtensorMap k_map, v_map;
-    bool head_first = true;
-    st = make_cache_map(&k_map, k_cache, s, stride_page, stride_token, stride_head, &head_first);
+    st = make_cache_map(&k_map, k_cache, s, stride_page, stride_token, stride_head);
     if (st != AC_OK) return st;
-    st = make_cache_map(&v_map, v_cache, s, stride_page, stride_token, stride_head, &head_first);
+    st = make_cache_map(&v_map, v_cache, s, stride_page, stride_token, stride_head);
     if (st != AC_OK) return st;
     const float scale = softmax_scale > 0.0f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d));
     const int split_tokens = split_tokens_for(max_context_len, num_splits);
-    cudaError_t e = launch_paged_decode_attn(k_map, v_map, head_first, q_rot, block_table,
+    cudaError_t e = launch_paged_decode_attn(k_map, v_map, q_rot, block_table,
                                              max_pages_per_seq, context_lens, new_tokens, scale,
                                              num_splits, split_tokens, partial_o, partial_lse, arrivals,
                                              out, B, Hq, Hkv, d, page_size, status_flag,

@@ -45,7 +45,7 @@ cudaError_t launch_rope_kv_append(const void* q_in, void* q_out, const void* k_n
                                   int d, int page_size, int num_pages, int32_t* status_flag,
                                   cudaStream_t stream);
 cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap& v_map,
-                                     bool head_before_token, const void* q_rot,
+                                     const void* q_rot,
                                      const int32_t* block_table, int max_pages_per_seq,
                                      const int32_t* context_lens, int new_tokens, float scale,
                                      int num_splits, int split_tokens, float* partial_o,

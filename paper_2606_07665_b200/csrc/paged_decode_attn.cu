@@ -1,10 +1,13 @@
 // A4: single-token decode attention over a paged KV cache, one CTA per (request, KV head, split).
 //
-// Data movement.  The K and V pools are described to the TMA unit as 4-D tensors
-// (head_dim, {head, token-in-page} ordered by stride, page).  A work tile is 16 consecutive tokens of
-// one KV head inside one page: head_dim/64 box loads of [16 tokens x 64 elements] for K and the same
-// for V, written to shared memory with the 128-byte swizzle so that ldmatrix reads are free of bank
-// conflicts.  Every warp runs its own ring of STAGES tiles with one mbarrier per stage and takes
+// Data movement.  The K and V pools are described to the TMA unit as 5-D tensors
+// (64 elements, token-in-page, 64-element block of head_dim, head, page).  A work tile is 16
+// consecutive tokens of one KV head inside one page: ONE box load [64 x 16 x head_dim/64] for K and
+// one for V, which lands in shared memory as head_dim/64 blocks of [16 tokens x 128 bytes] with the
+// 128-byte swizzle, so ldmatrix reads are free of bank conflicts.  (Issuing a tensor load costs the
+// issuing thread on the order of 100 ns, so the number of loads per tile matters: splitting head_dim
+// into the innermost 64 elements and an outer block index keeps the swizzle span at 128 bytes while
+// still fetching the whole 256-byte rows with one instruction.)  Every warp runs its own ring of STAGES tiles with one mbarrier per stage and takes
 // tiles warp, warp+WARPS, ... of the CTA's token range; there is no CTA-wide synchronisation in the
 // main loop.  The physical page id of a tile is fetched from the block table one tile ahead of the
 // TMA issue that needs it.  KV bytes are read once, so the loads carry an evict-first L2 policy.
@@ -63,7 +66,6 @@ struct AttnParams {
     int num_splits;
     int split_tokens;
     int Hq, Hkv, page_size;
-    int head_before_token;        // order of the two middle tensor-map coordinates
     int fused_merge;              // 1: the last CTA of a (request, KV head) merges the splits itself
 };
 
@@ -151,15 +153,9 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
         const int stage = j % STAGES;
         const uint32_t bar = bars + stage * 8;
         const uint32_t dst = ring + stage * L::STAGE_BYTES;
-        const int c1 = p.head_before_token ? h : slot;
-        const int c2 = p.head_before_token ? slot : h;
         mbar_arrive_expect_tx(bar, L::STAGE_BYTES);
-#pragma unroll
-        for (int hf = 0; hf < L::HALVES; ++hf)
-            tma_load_4d(dst + hf * L::HALF_BYTES, &k_map, bar, hf * 64, c1, c2, page, policy);
-#pragma unroll
-        for (int hf = 0; hf < L::HALVES; ++hf)
-            tma_load_4d(dst + L::K_BYTES + hf * L::HALF_BYTES, &v_map, bar, hf * 64, c1, c2, page, policy);
+        tma_load_5d(dst, &k_map, bar, 0, slot, 0, h, page, policy);
+        tma_load_5d(dst + L::K_BYTES, &v_map, bar, 0, slot, 0, h, page, policy);
     };
 
     // ---- prologue: fill the ring -------------------------------------------------------------
@@ -496,7 +492,7 @@ cudaError_t attn_set_attributes(int smem_optin) {
 }
 
 cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap& v_map,
-                                     bool head_before_token, const void* q_rot,
+                                     const void* q_rot,
                                      const int32_t* block_table, int max_pages_per_seq,
                                      const int32_t* context_lens, int new_tokens, float scale,
                                      int num_splits, int split_tokens, float* partial_o,
@@ -521,7 +517,6 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
     p.Hq = Hq;
     p.Hkv = Hkv;
     p.page_size = page_size;
-    p.head_before_token = head_before_token ? 1 : 0;
     const bool wide = Hq / Hkv > 8;
     if (d == 128) {
         return wide ? launch_one<128, true>(k_map, v_map, p, B, stream)
