@@ -33,9 +33,9 @@ namespace {
 
 using namespace acdev;
 
-constexpr int WARPS = 4;
+constexpr int WARPS = 6;
 constexpr int THREADS = WARPS * 32;
-constexpr int STAGES = 3;
+constexpr int STAGES = 2;
 constexpr int TILE = 16;                      // tokens per stage
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
