@@ -80,7 +80,7 @@ int ac_sm_count(void);
 
 /* Split plan (host only, pure, needs no GPU).  Chooses how many KV splits the attention kernel
  * should use for `sm_count` SMs (<= 0: the count seen by ac_init, or 148 if none): none when the
- * (request, KV head) pairs alone fill the GPU and contexts are short, chunks of at most 2560 tokens
+ * (request, KV head) pairs alone fill the GPU and contexts are short, chunks of at most 4096 tokens
  * when contexts are long, and otherwise the split count with the smallest estimated time from a
  * small cost model (bandwidth of one CTA, waves of CTAs, partial-result traffic); splits are never
  * shorter than 256 tokens.  max_context_len = the largest number of tokens any row attends over in this bucket

@@ -189,7 +189,7 @@ int ac_decode_plan(int B, int Hq, int Hkv, int d, int page_size, int max_context
     // (its ring holds 96 KB against ~2.5 us of load latency), a wave of CTAs costs ~3 us of
     // ramp-up/epilogue that overlaps poorly, and every extra split adds partial-result traffic.
     //  * At least one wave of (request, KV head) pairs: do not split, unless contexts are long --
-    //    then cut them into chunks of at most 2560 tokens so that ragged batches balance.
+    //    then cut them into chunks of at most 4096 tokens so that ragged batches balance.
     //  * Fewer pairs than slots: scan the split counts and take the one with the smallest
     //    estimated time, all rows assumed at max_context_len.
     const double slots = 2.0 * sm_count;
@@ -199,7 +199,7 @@ int ac_decode_plan(int B, int Hq, int Hkv, int d, int page_size, int max_context
     const long long pairs = static_cast<long long>(B) * Hkv;
     long long S = 1;
     if (pairs >= static_cast<long long>(slots)) {
-        S = (static_cast<long long>(max_context_len) + 2559) / 2560;
+        S = (static_cast<long long>(max_context_len) + 4095) / 4096;
     } else {
         const int s_max = max_context_len / 256 > 1 ? max_context_len / 256 : 1;
         double best = 0.0;

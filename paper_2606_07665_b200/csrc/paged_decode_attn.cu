@@ -23,6 +23,7 @@
 // With a group of 4-8 query rows the path needs G flop per KV byte; at HBM speed that exceeds what
 // the fp32 pipes deliver for G >= 7, which is why the products run on the tensor pipe even though
 // the kernel is bound by HBM bandwidth.
+#include <limits.h>
 #include <math.h>
 
 #include "ac_device.cuh"
@@ -37,6 +38,7 @@ constexpr int WARPS = 6;
 constexpr int THREADS = WARPS * 32;
 constexpr int STAGES = 2;
 constexpr int TILE = 16;                      // tokens per stage
+constexpr int kLongestFirstMaxBatch = 128;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 
@@ -67,6 +69,7 @@ struct AttnParams {
     int split_tokens;
     int Hq, Hkv, page_size;
     int fused_merge;              // 1: the last CTA of a (request, KV head) merges the splits itself
+    int longest_first;            // 1: grid row y serves the request with the y-th longest context
 };
 
 template <int D, bool WIDE>
@@ -83,10 +86,36 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     uint8_t* smem_gen = smem_raw + (smem_base - smem_addr(smem_raw));
 
     const int h = blockIdx.x;
-    const int b = blockIdx.y;
     const int split = blockIdx.z;
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    int b = blockIdx.y;
+    if (p.longest_first) {
+        // The hardware hands out CTAs in grid order; when the grid is several waves deep, serving
+        // the longest requests first keeps the short ones for the tail of the grid (greedy
+        // longest-processing-time order).  Every CTA derives the same ranking from context_lens:
+        // thread t counts the requests that sort before request t (longer, or equal and earlier).
+        __shared__ int s_request;
+        int* s_len = reinterpret_cast<int*>(smem_gen);            // the rings are not in use yet
+        const int B = gridDim.y;
+        const int B4 = (B + 3) & ~3;
+        for (int i = threadIdx.x; i < B4; i += THREADS) s_len[i] = i < B ? p.context_lens[i] : INT_MIN;
+        __syncthreads();
+        for (int t = threadIdx.x; t < B; t += THREADS) {
+            const int mine = s_len[t];
+            int rank = 0;
+            for (int j = 0; j < B4; j += 4) {               // padding entries never sort before anything
+                const int4 o = *reinterpret_cast<const int4*>(s_len + j);
+                rank += (o.x > mine) || (o.x == mine && j < t);
+                rank += (o.y > mine) || (o.y == mine && j + 1 < t);
+                rank += (o.z > mine) || (o.z == mine && j + 2 < t);
+                rank += (o.w > mine) || (o.w == mine && j + 3 < t);
+            }
+            if (rank == static_cast<int>(blockIdx.y)) s_request = t;
+        }
+        __syncthreads();
+        b = s_request;
+    }
     const int G = p.Hq / p.Hkv;
     const int S = p.num_splits;
 
@@ -502,6 +531,13 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
     AttnParams p;
     p.arrivals = arrivals;
     p.fused_merge = arrivals != nullptr ? 1 : 0;
+    // Worth its ~1 us per CTA only when the grid does not fit on the GPU at once, and kept to batch
+    // sizes whose ranking (B comparisons per thread) stays short.
+    int sms = 0, dev = 0;
+    cudaGetDevice(&dev);
+    sms = device_state(dev).sm_count;
+    p.longest_first = (B > 1 && B <= kLongestFirstMaxBatch &&
+                       static_cast<long long>(B) * Hkv * num_splits > 2ll * sms) ? 1 : 0;
     p.q = static_cast<const uint16_t*>(q_rot);
     p.block_table = block_table;
     p.context_lens = context_lens;

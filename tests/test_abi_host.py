@@ -61,7 +61,7 @@ def test_plan_properties(ac, B, Hq, Hkv, d, ps, maxlen):
     assert wb == ac.ac_workspace_bytes(B, Hq, d, S)
     if S > 1:
         assert st >= 256                                          # splits stay long enough to amortise set-up
-    if B * Hkv >= 148 * 2 and maxlen <= 2560:
+    if B * Hkv >= 148 * 2 and maxlen <= 4096:
         assert S == 1                                             # already enough CTAs without splitting
     if B * Hkv < 148 and maxlen >= 512:
         assert S > 1                                              # small batches are split across SMs

@@ -325,6 +325,19 @@ def test_workload_continuous_batching(rt, fused):
     run_and_compare(rt, W.continuous_batching(), fused=fused)
 
 
+@pytest.mark.parametrize("splits", [1, 2])
+def test_longest_first_row_order_with_ties_and_inactive_rows(rt, splits):
+    # 100 requests x 4 KV heads = 400+ CTAs: more than fit on the GPU at once, so the kernel serves
+    # requests in order of decreasing length.  Many equal lengths and some inactive rows: every row
+    # must still be served exactly once.
+    rng = np.random.default_rng(11)
+    lens = rng.choice([0, 15, 16, 100, 100, 100, 333, 700], size=100).tolist()
+    w = W.make_workload("lpt", 50, B=100, Hq=8, Hkv=4, d=64, page_size=16, num_pages=2600,
+                        context_lens=lens, rope_base=10000.0, inactive_rows=(0, 17, 99))
+    st, _ = run_and_compare(rt, w, num_splits=splits)
+    assert (rt.bits_of(st.out)[[0, 17, 99]] == 0).all()
+
+
 def test_fused_merge_repeated_launches_and_row_without_tokens(rt):
     # The arrival counters reset themselves: many launches on one workspace stay correct, also when a
     # row has no tokens at all (its output is +0) and when most splits of a short row are empty.
