@@ -174,6 +174,28 @@ int ac_paged_decode_attn_fused_merge(const void* q_rot, const void* k_cache, con
                                      int B, int Hq, int Hkv, int d, int page_size, int num_pages,
                                      int max_context_len, int32_t* status_flag, void* stream);
 
+/* A1 + A2 + A4 + A5 in ONE launch (the step as the paper's families (iii)/(iv) and its kv_append
+ * kernel define it, fused): every CTA rotates the query rows of its group in registers (same exact
+ * arithmetic as ac_rope_kv_append); the warp whose tile holds the new token's slot rotates k_new,
+ * writes k and v into the cache page AND into the tile it just loaded, then attention proceeds over
+ * context_lens[b] + 1 tokens and the last CTA of each (request, KV head) merges the splits.  Cache
+ * contents after the call are bit-identical to ac_rope_kv_append's; outputs equal those of the
+ * three-call sequence up to the fp32 merge order.
+ *
+ * q_in is the un-rotated query [B,Hq,d]; q_rot_out (optional, may be NULL) receives the rotated
+ * rows and must not alias q_in.  Workspace as for ac_paged_decode_attn_fused_merge (counters zero on
+ * entry when num_splits > 1).  A row whose position is outside the rope table or whose page id is
+ * outside the pool sets the status bits and appends nothing; its output is then unspecified. */
+int ac_decode_step_fused(const void* q_in, void* q_rot_out, const void* k_new, const void* v_new,
+                         void* k_cache, void* v_cache,
+                         int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                         const int32_t* block_table, int max_pages_per_seq,
+                         const int32_t* context_lens,
+                         const float* rope_cos, const float* rope_sin, int max_position,
+                         float softmax_scale, int num_splits, void* workspace, size_t workspace_bytes,
+                         void* out, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                         int max_context_len, int32_t* status_flag, void* stream);
+
 /* A5: merge of the split partials ("cross-CTA merging" of family (iv), here as its own kernel):
  *   M = max_s lse_s,  w_s = exp(lse_s - M),  out[b,hq,:] = sum_s w_s partial_o[b,hq,s,:] / sum_s w_s
  * rounded to bf16.  Splits with lse = -inf are skipped (their partial_o is not read); a row whose
@@ -185,8 +207,8 @@ int ac_splitkv_merge(const void* workspace, int num_splits, const int32_t* conte
 /* The whole step from HOST buffers (for callers that hold the step's inputs on the host, and for
  * end-to-end timing): copies q/k_new/v_new/block_table/context_lens from the *_host buffers (pinned
  * memory recommended) into the caller's device buffers of the same name, resets the arrival
- * counters, enqueues ac_rope_kv_append and ac_paged_decode_attn_fused_merge for the given num_splits
- * (workspace_bytes >= ac_fused_workspace_bytes), and copies the bf16 result from out into out_host.  Everything is asynchronous on `stream`; the caller
+ * counters, enqueues ac_decode_step_fused for the given num_splits (workspace_bytes >=
+ * ac_fused_workspace_bytes), and copies the bf16 result from out into out_host.  Everything is asynchronous on `stream`; the caller
  * synchronises the stream before reading out_host.  The KV cache pools and rope tables stay on the
  * device (they are the layer's resident state, not a per-step input).  No paper counterpart. */
 int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* v_new_host,

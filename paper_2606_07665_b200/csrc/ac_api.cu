@@ -265,7 +265,8 @@ static int attn_common(const void* q_rot, const void* k_cache, const void* v_cac
                        int max_pages_per_seq, const int32_t* context_lens, int new_tokens,
                        float softmax_scale, int num_splits, void* workspace, size_t workspace_bytes,
                        void* out, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
-                       int max_context_len, int32_t* status_flag, void* stream, bool fused_merge) {
+                       int max_context_len, int32_t* status_flag, void* stream, bool fused_merge,
+                       const FusedRopeArgs* rope = nullptr) {
     if (!q_rot || !k_cache || !v_cache || !block_table || !context_lens) return AC_ERR_NULL;
     Shape s{B, Hq, Hkv, d, page_size, num_pages};
     int st = check_shape(s);
@@ -306,7 +307,7 @@ static int attn_common(const void* q_rot, const void* k_cache, const void* v_cac
     cudaError_t e = launch_paged_decode_attn(k_map, v_map, q_rot, block_table,
                                              max_pages_per_seq, context_lens, new_tokens, scale,
                                              num_splits, split_tokens, partial_o, partial_lse, arrivals,
-                                             out, B, Hq, Hkv, d, page_size, status_flag,
+                                             out, B, Hq, Hkv, d, page_size, status_flag, rope,
                                              static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
 }
@@ -352,6 +353,38 @@ int ac_paged_decode_attn_fused_merge(const void* q_rot, const void* k_cache, con
                        max_pages_per_seq, context_lens, new_tokens, softmax_scale, num_splits, workspace,
                        workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages, max_context_len,
                        status_flag, stream, true);
+}
+
+int ac_decode_step_fused(const void* q_in, void* q_rot_out, const void* k_new, const void* v_new,
+                         void* k_cache, void* v_cache, int64_t stride_page, int64_t stride_token,
+                         int64_t stride_head, const int32_t* block_table, int max_pages_per_seq,
+                         const int32_t* context_lens, const float* rope_cos, const float* rope_sin,
+                         int max_position, float softmax_scale, int num_splits, void* workspace,
+                         size_t workspace_bytes, void* out, int B, int Hq, int Hkv, int d, int page_size,
+                         int num_pages, int max_context_len, int32_t* status_flag, void* stream) {
+    if (!q_in || !k_new || !v_new || !rope_cos || !rope_sin) return AC_ERR_NULL;
+    if (max_position <= 0) return AC_ERR_SHAPE;
+    if (q_rot_out == q_in) return AC_ERR_UNSUPPORTED;      // other CTAs still read the raw rows
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(rope_cos) || !aligned16(rope_sin) ||
+        (q_rot_out && !aligned16(q_rot_out)))
+        return AC_ERR_ALIGN;
+    FusedRopeArgs rope;
+    rope.q_rot_out = q_rot_out;
+    rope.k_new = k_new;
+    rope.v_new = v_new;
+    rope.k_cache = k_cache;
+    rope.v_cache = v_cache;
+    rope.stride_page = stride_page;
+    rope.stride_token = stride_token;
+    rope.stride_head = stride_head;
+    rope.rope_cos = rope_cos;
+    rope.rope_sin = rope_sin;
+    rope.max_position = max_position;
+    rope.num_pages = num_pages;
+    return attn_common(q_in, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
+                       max_pages_per_seq, context_lens, 1, softmax_scale, num_splits, workspace,
+                       workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages, max_context_len,
+                       status_flag, stream, true, &rope);
 }
 
 int ac_splitkv_merge(const void* workspace, int num_splits, const int32_t* context_lens, void* out,
@@ -408,14 +441,11 @@ int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* 
         (e = cudaMemcpyAsync(context_lens, context_lens_host, static_cast<size_t>(B) * sizeof(int32_t),
                              cudaMemcpyHostToDevice, cs)) != cudaSuccess)
         return fail_cuda(static_cast<int>(e));
-    st = ac_rope_kv_append(q, q, k_new, v_new, k_cache, v_cache, stride_page, stride_token, stride_head,
-                           block_table, max_pages_per_seq, context_lens, rope_cos, rope_sin,
-                           max_position, B, Hq, Hkv, d, page_size, num_pages, status_flag, stream);
-    if (st != AC_OK) return st;
-    st = ac_paged_decode_attn_fused_merge(q, k_cache, v_cache, stride_page, stride_token, stride_head,
-                                          block_table, max_pages_per_seq, context_lens, 1, softmax_scale,
-                                          num_splits, workspace, workspace_bytes, out, B, Hq, Hkv, d,
-                                          page_size, num_pages, max_context_len, status_flag, stream);
+    st = ac_decode_step_fused(q, nullptr, k_new, v_new, k_cache, v_cache, stride_page, stride_token,
+                              stride_head, block_table, max_pages_per_seq, context_lens, rope_cos,
+                              rope_sin, max_position, softmax_scale, num_splits, workspace,
+                              workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages, max_context_len,
+                              status_flag, stream);
     if (st != AC_OK) return st;
     e = cudaMemcpyAsync(out_host, out, q_bytes, cudaMemcpyDeviceToHost, cs);
     return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));

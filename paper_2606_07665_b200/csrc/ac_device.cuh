@@ -133,4 +133,33 @@ __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
     return __uint_as_float(static_cast<uint32_t>(b) << 16);
 }
 
+// ---- rotary embedding of one pair, exact then rounded once ------------------------------------
+
+// Nearest-even bf16 of an fp64 value without double rounding: fp64 -> fp32 by truncation with a
+// sticky bit (round to odd), then the usual nearest-even cut to 16 bits.
+__device__ __forceinline__ uint16_t f64_to_bf16_rne(double x) {
+    float f = __double2float_rz(x);
+    uint32_t u = __float_as_uint(f);
+    if (static_cast<double>(f) != x) u |= 1u;          // sticky bit: round to odd (NaN stays NaN)
+    if ((u & 0x7F800000u) == 0x7F800000u) {            // inf or NaN
+        return static_cast<uint16_t>((u >> 16) | ((u & 0xFFFFu) ? 0x40u : 0u));
+    }
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return static_cast<uint16_t>(u >> 16);
+}
+
+// (a, b) = (x_i, x_{i+d/2}) as bf16 bits, c/s = cos/sin of the pair's angle.  Both products are exact
+// in fp64 (8-bit x 24-bit significands); __dmul_rn/__dadd_rn keep the three operations separate.
+__device__ __forceinline__ uint16_t rope_first_half(uint16_t a, uint16_t b, float c, float s) {
+    const double ad = static_cast<double>(bf16_bits_to_float(a));
+    const double bd = static_cast<double>(bf16_bits_to_float(b));
+    return f64_to_bf16_rne(__dsub_rn(__dmul_rn(ad, static_cast<double>(c)), __dmul_rn(bd, static_cast<double>(s))));
+}
+
+__device__ __forceinline__ uint16_t rope_second_half(uint16_t a, uint16_t b, float c, float s) {
+    const double ad = static_cast<double>(bf16_bits_to_float(a));
+    const double bd = static_cast<double>(bf16_bits_to_float(b));
+    return f64_to_bf16_rne(__dadd_rn(__dmul_rn(bd, static_cast<double>(c)), __dmul_rn(ad, static_cast<double>(s))));
+}
+
 }  // namespace acdev

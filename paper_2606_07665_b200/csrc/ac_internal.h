@@ -34,6 +34,19 @@ struct CacheView {
     int num_pages, page_size, Hkv, d;
 };
 
+// Extra inputs of the fused step: the attention kernel itself rotates q/k and appends k/v.
+struct FusedRopeArgs {
+    void* q_rot_out;          // optional
+    const void* k_new;
+    const void* v_new;
+    void* k_cache;
+    void* v_cache;
+    int64_t stride_page, stride_token, stride_head;
+    const float* rope_cos;
+    const float* rope_sin;
+    int max_position, num_pages;
+};
+
 // Per-kernel launchers; each validates nothing (the ABI layer did) and returns a cudaError_t.
 cudaError_t attn_set_attributes(int smem_optin);
 cudaError_t launch_rope_kv_append(const void* q_in, void* q_out, const void* k_new, const void* v_new,
@@ -51,7 +64,7 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
                                      int num_splits, int split_tokens, float* partial_o,
                                      float* partial_lse, int32_t* arrivals, void* out, int B, int Hq,
                                      int Hkv, int d, int page_size, int32_t* status_flag,
-                                     cudaStream_t stream);
+                                     const FusedRopeArgs* rope, cudaStream_t stream);
 cudaError_t launch_splitkv_merge(const float* partial_o, const float* partial_lse, int num_splits,
                                  const int32_t* context_lens, void* out, int B, int Hq, int d,
                                  cudaStream_t stream);

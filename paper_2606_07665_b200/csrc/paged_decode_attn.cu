@@ -54,7 +54,18 @@ struct Smem {
 };
 
 struct AttnParams {
-    const uint16_t* q;            // [B, Hq, D] bf16, already rotated
+    // -- only for the fused step (ROPE = true): the kernel rotates q/k and appends k/v itself
+    uint16_t* q_rot_out;          // [B, Hq, D] rotated q, optional (must not alias q)
+    const uint16_t* k_new;        // [B, Hkv, D] un-rotated
+    const uint16_t* v_new;        // [B, Hkv, D]
+    uint16_t* k_cache;            // page pools (element strides below)
+    uint16_t* v_cache;
+    int64_t stride_page, stride_token, stride_head;
+    const float* rope_cos;        // [max_position, D/2]
+    const float* rope_sin;
+    int max_position, num_pages;
+    // -- always
+    const uint16_t* q;            // [B, Hq, D] bf16: already rotated (ROPE = false) or raw (ROPE = true)
     const int32_t* block_table;   // [B, max_pages_per_seq]
     const int32_t* context_lens;  // [B]
     float* partial_o;             // [B, Hq, S, D]   (S > 1)
@@ -72,7 +83,7 @@ struct AttnParams {
     int longest_first;            // 1: grid row y serves the request with the y-th longest context
 };
 
-template <int D, bool WIDE>
+template <int D, bool WIDE, bool ROPE>
 __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
     const AttnParams p) {
@@ -119,9 +130,15 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     const int G = p.Hq / p.Hkv;
     const int S = p.num_splits;
 
-    // Everything up to the first read of q or of the slot that holds the new token is independent of
-    // the kernel that precedes this one in the stream (normally the RoPE + append kernel), so with a
-    // programmatic dependent launch it overlaps that kernel's execution.
+    // Let the next kernel of the stream (launched with the programmatic-serialization attribute, as
+    // the kernels of this library are) become resident as soon as this grid's last CTAs are: its
+    // set-up and first loads then fill the SM slots that free up during this grid's tail.
+    cudaTriggerProgrammaticLaunchCompletion();
+
+    // Everything up to the first read of q or of a cache slot that the preceding kernel may have
+    // written is independent of that kernel, so with a programmatic dependent launch it overlaps the
+    // preceding kernel's execution.  The preceding kernel is either the RoPE + append kernel of this
+    // step (writes slot ctx) or the fused step of the previous token (wrote slot ctx - 1).
     const int tok_begin = split * p.split_tokens;
     const int tile_begin = tok_begin / TILE;
     auto tile_token0 = [&](int j) { return (tile_begin + warp + j * WARPS) * TILE; };
@@ -172,9 +189,10 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     const int n_tiles = (tok_end - tok_begin + TILE - 1) / TILE;
     const int n_my = n_tiles > warp ? (n_tiles - warp + WARPS - 1) / WARPS : 0;
     const uint64_t policy = l2_policy_evict_first();
-    // The tile that holds the token appended by the preceding kernel (if any) must not be fetched
-    // before that kernel has completed.
+    // Tiles from the one holding slot ctx - 1 onwards must not be fetched before the preceding kernel
+    // has completed; new_token_tile is where this step's own token lives.
     const int new_token_tile = p.new_tokens > 0 ? ctx / TILE : -1;
+    const int first_dependent_tile = (ctx > 0 ? ctx - 1 : 0) / TILE;
 
     auto issue = [&](int j, int page) {      // lane 0 only
         const int tok0 = tile_token0(j);
@@ -193,7 +211,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
 #pragma unroll
     for (int s = 0; s < STAGES; ++s) {
         if (s < n_my) {
-            if (!dependency_met && tile_begin + warp + s * WARPS == new_token_tile) {
+            if (!dependency_met && tile_begin + warp + s * WARPS >= first_dependent_tile) {
                 cudaGridDependencySynchronize();
                 dependency_met = true;
             }
@@ -204,11 +222,99 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     int page_next = issued < n_my ? load_page_id(issued) : 0;
     if (!dependency_met) cudaGridDependencySynchronize();      // q was written by the preceding kernel
 
+    // ---- fused step: rotate and append the new k/v early, under the latency of the first tiles ------
+    constexpr int APPEND_PAIRS = D / 64;          // rotary pairs per lane (D/2 pairs over 32 lanes)
+    uint16_t k_rot_lo[APPEND_PAIRS], k_rot_hi[APPEND_PAIRS];
+    uint2 v_new4 = make_uint2(0u, 0u);
+    int append_j = -1;                            // index of this warp's tile that holds the new slot
+    bool append_ok = false;
+    const bool rope_ok = ROPE && ctx < p.max_position;
+    if (ROPE) {
+        if (!rope_ok && threadIdx.x == 0 && p.status_flag != nullptr)
+            atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
+        const int rel = new_token_tile - tile_begin - warp;
+        if (rel >= 0 && rel % WARPS == 0 && rel / WARPS < n_my) append_j = rel / WARPS;
+        if (append_j >= 0 && rope_ok) {
+            const int page = load_page_id(append_j);
+            if (page < 0 || page >= p.num_pages) {
+                if (lane == 0 && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
+            } else {
+                append_ok = true;
+                const size_t goff = static_cast<size_t>(page) * p.stride_page +
+                                    static_cast<size_t>(ctx % p.page_size) * p.stride_token +
+                                    static_cast<size_t>(h) * p.stride_head;
+                const uint16_t* ksrc = p.k_new + (static_cast<size_t>(b) * p.Hkv + h) * D;
+                const uint16_t* vsrc = p.v_new + (static_cast<size_t>(b) * p.Hkv + h) * D;
+                const float* cos_row = p.rope_cos + static_cast<size_t>(ctx) * (D / 2);
+                const float* sin_row = p.rope_sin + static_cast<size_t>(ctx) * (D / 2);
+#pragma unroll
+                for (int u = 0; u < APPEND_PAIRS; ++u) {
+                    const int i = lane + 32 * u;
+                    const uint16_t a = ksrc[i], bb = ksrc[i + D / 2];
+                    const float c = cos_row[i], sn = sin_row[i];
+                    k_rot_lo[u] = rope_first_half(a, bb, c, sn);
+                    k_rot_hi[u] = rope_second_half(a, bb, c, sn);
+                    p.k_cache[goff + i] = k_rot_lo[u];
+                    p.k_cache[goff + i + D / 2] = k_rot_hi[u];
+                }
+                if (lane * 4 < D) {
+                    v_new4 = *reinterpret_cast<const uint2*>(vsrc + lane * 4);
+                    *reinterpret_cast<uint2*>(p.v_cache + goff + lane * 4) = v_new4;
+                }
+            }
+        }
+    }
+
     // ---- query fragments (A operand of Q K^T), rows = heads of the group ---------------------------
     const int g = lane >> 2;
     const int t = lane & 3;
     uint32_t qa[KSTEPS][2 * ROWS];
-    {
+    constexpr int QSTRIDE = D + 8;                 // padded row: fragment loads hit 32 distinct banks
+    __shared__ __align__(16) uint16_t s_q[ROPE ? 16 * QSTRIDE : 8];
+    if (ROPE) {
+        // The CTA rotates its G query rows once (pair i with i + D/2, exact then rounded, as the
+        // stand-alone kernel does) into shared memory; every warp then reads its fragments from there.
+        const uint16_t* qsrc = p.q + (static_cast<size_t>(b) * p.Hq + h * G) * D;
+        const float* cos_row = p.rope_cos + static_cast<size_t>(ctx) * (D / 2);
+        const float* sin_row = p.rope_sin + static_cast<size_t>(ctx) * (D / 2);
+        uint16_t* qdst = (p.q_rot_out != nullptr && split == 0)
+                             ? p.q_rot_out + (static_cast<size_t>(b) * p.Hq + h * G) * D : nullptr;
+        for (int idx = threadIdx.x; idx < 16 * (D / 2); idx += THREADS) {
+            const int row = idx / (D / 2);
+            const int i = idx - row * (D / 2);
+            uint16_t r0 = 0, r1 = 0;
+            if (row < G) {
+                const uint16_t a = qsrc[row * D + i], bb = qsrc[row * D + i + D / 2];
+                if (rope_ok) {
+                    const float c = cos_row[i], sn = sin_row[i];
+                    r0 = rope_first_half(a, bb, c, sn);
+                    r1 = rope_second_half(a, bb, c, sn);
+                } else {
+                    r0 = a;
+                    r1 = bb;
+                }
+                if (qdst != nullptr && rope_ok) {
+                    qdst[row * D + i] = r0;
+                    qdst[row * D + i + D / 2] = r1;
+                }
+            }
+            if (WIDE || row < 8) {
+                s_q[row * QSTRIDE + i] = r0;
+                s_q[row * QSTRIDE + i + D / 2] = r1;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < KSTEPS; ++kk) {
+            const int col = kk * 16 + 2 * t;
+            qa[kk][0] = *reinterpret_cast<const uint32_t*>(s_q + g * QSTRIDE + col);
+            qa[kk][ROWS] = *reinterpret_cast<const uint32_t*>(s_q + g * QSTRIDE + col + 8);
+            if (WIDE) {
+                qa[kk][1] = *reinterpret_cast<const uint32_t*>(s_q + (g + 8) * QSTRIDE + col);
+                qa[kk][ROWS + 1] = *reinterpret_cast<const uint32_t*>(s_q + (g + 8) * QSTRIDE + col + 8);
+            }
+        }
+    } else {
         const uint16_t* qrow0 = p.q + (static_cast<size_t>(b) * p.Hq + h * G + g) * D;
         const bool v0 = g < G;
         const bool v1 = WIDE && (g + 8 < G);
@@ -257,6 +363,25 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
         }
         const int tok0 = tile_token0(j);
         const int n_valid = tok_end - tok0;                    // >= 1; < 16 only on the last tile
+
+        if (ROPE && j == append_j && append_ok) {
+            // The tile just loaded still has the stale slot of the new token: overwrite that row with
+            // the rotated k and the v computed (and written to the cache) during the prologue.
+            const int slot_in_tile = ctx - tok0;
+            auto tile_byte = [&](int col) {       // byte offset of (slot_in_tile, col) inside a K or V tile
+                return (col >> 6) * L::HALF_BYTES + slot_in_tile * 128 +
+                       ((((col & 63) >> 3) ^ (slot_in_tile & 7)) << 4) + ((col & 7) << 1);
+            };
+#pragma unroll
+            for (int u = 0; u < APPEND_PAIRS; ++u) {
+                const int i = lane + 32 * u;
+                *reinterpret_cast<uint16_t*>(smem_gen + (kbase - smem_base) + tile_byte(i)) = k_rot_lo[u];
+                *reinterpret_cast<uint16_t*>(smem_gen + (kbase - smem_base) + tile_byte(i + D / 2)) = k_rot_hi[u];
+            }
+            if (lane * 4 < D)
+                *reinterpret_cast<uint2*>(smem_gen + (vbase - smem_base) + tile_byte(lane * 4)) = v_new4;
+            __syncwarp();
+        }
 
         // ---- S = Q K^T for 16 tokens -------------------------------------------------------
         float s[2][4];
@@ -484,7 +609,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     }
 }
 
-template <int D, bool WIDE>
+template <int D, bool WIDE, bool ROPE>
 cudaError_t launch_one(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnParams& p, int B,
                        cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
@@ -500,7 +625,7 @@ cudaError_t launch_one(const CUtensorMap& k_map, const CUtensorMap& v_map, const
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, paged_decode_attn_kernel<D, WIDE>, k_map, v_map, p);
+    return cudaLaunchKernelEx(&cfg, paged_decode_attn_kernel<D, WIDE, ROPE>, k_map, v_map, p);
 }
 
 }  // namespace
@@ -509,7 +634,10 @@ cudaError_t attn_set_attributes(int smem_optin) {
     if (Smem<128>::TOTAL > smem_optin) return cudaErrorInvalidConfiguration;
     cudaError_t e;
 #define AC_SET(D_, W_)                                                                             \
-    e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_>,                                     \
+    e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, false>,                              \
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D_>::TOTAL);        \
+    if (e != cudaSuccess) return e;                                                                \
+    e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, true>,                               \
                              cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D_>::TOTAL);        \
     if (e != cudaSuccess) return e;
     AC_SET(128, false)
@@ -527,8 +655,28 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
                                      int num_splits, int split_tokens, float* partial_o,
                                      float* partial_lse, int32_t* arrivals, void* out, int B, int Hq,
                                      int Hkv, int d, int page_size, int32_t* status_flag,
-                                     cudaStream_t stream) {
+                                     const FusedRopeArgs* rope, cudaStream_t stream) {
     AttnParams p;
+    p.q_rot_out = nullptr;
+    p.k_new = p.v_new = nullptr;
+    p.k_cache = p.v_cache = nullptr;
+    p.stride_page = p.stride_token = p.stride_head = 0;
+    p.rope_cos = p.rope_sin = nullptr;
+    p.max_position = p.num_pages = 0;
+    if (rope != nullptr) {
+        p.q_rot_out = static_cast<uint16_t*>(rope->q_rot_out);
+        p.k_new = static_cast<const uint16_t*>(rope->k_new);
+        p.v_new = static_cast<const uint16_t*>(rope->v_new);
+        p.k_cache = static_cast<uint16_t*>(rope->k_cache);
+        p.v_cache = static_cast<uint16_t*>(rope->v_cache);
+        p.stride_page = rope->stride_page;
+        p.stride_token = rope->stride_token;
+        p.stride_head = rope->stride_head;
+        p.rope_cos = rope->rope_cos;
+        p.rope_sin = rope->rope_sin;
+        p.max_position = rope->max_position;
+        p.num_pages = rope->num_pages;
+    }
     p.arrivals = arrivals;
     p.fused_merge = arrivals != nullptr ? 1 : 0;
     // Worth its ~1 us per CTA only when the grid does not fit on the GPU at once, and kept to batch
@@ -554,12 +702,20 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
     p.Hkv = Hkv;
     p.page_size = page_size;
     const bool wide = Hq / Hkv > 8;
-    if (d == 128) {
-        return wide ? launch_one<128, true>(k_map, v_map, p, B, stream)
-                    : launch_one<128, false>(k_map, v_map, p, B, stream);
+    if (rope != nullptr) {
+        if (d == 128) {
+            return wide ? launch_one<128, true, true>(k_map, v_map, p, B, stream)
+                        : launch_one<128, false, true>(k_map, v_map, p, B, stream);
+        }
+        return wide ? launch_one<64, true, true>(k_map, v_map, p, B, stream)
+                    : launch_one<64, false, true>(k_map, v_map, p, B, stream);
     }
-    return wide ? launch_one<64, true>(k_map, v_map, p, B, stream)
-                : launch_one<64, false>(k_map, v_map, p, B, stream);
+    if (d == 128) {
+        return wide ? launch_one<128, true, false>(k_map, v_map, p, B, stream)
+                    : launch_one<128, false, false>(k_map, v_map, p, B, stream);
+    }
+    return wide ? launch_one<64, true, false>(k_map, v_map, p, B, stream)
+                : launch_one<64, false, false>(k_map, v_map, p, B, stream);
 }
 
 }  // namespace ac

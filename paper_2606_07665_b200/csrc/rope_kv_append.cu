@@ -16,18 +16,6 @@
 namespace ac {
 namespace {
 
-__device__ __forceinline__ uint16_t f64_to_bf16_rne(double x) {
-    float f = __double2float_rz(x);
-    uint32_t u = __float_as_uint(f);
-    if (static_cast<double>(f) != x) u |= 1u;          // sticky bit: round to odd (NaN stays NaN)
-    // fp32 -> bf16 nearest-even on the bit pattern; finite inputs only overflow to inf correctly.
-    if ((u & 0x7F800000u) == 0x7F800000u) {            // inf or NaN
-        return static_cast<uint16_t>((u >> 16) | ((u & 0xFFFFu) ? 0x40u : 0u));
-    }
-    u += 0x7FFFu + ((u >> 16) & 1u);
-    return static_cast<uint16_t>(u >> 16);
-}
-
 struct alignas(16) Vec8 {
     uint16_t v[8];
 };
@@ -42,8 +30,11 @@ __global__ void __launch_bounds__(128) rope_kv_append_kernel(
     const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, int max_position, int B,
     int Hq, int Hkv, int page_size, int num_pages, int32_t* status_flag) {
     // Let a dependent kernel (the attention launch that follows) begin its own set-up right away; it
-    // synchronises on this grid's completion before reading anything written here.
+    // synchronises on this grid's completion before reading anything written here.  This kernel
+    // itself may have been launched early, under the tail of the previous attention kernel, whose
+    // inputs (the rotated q buffer, the cache) it overwrites: wait for that kernel first.
     cudaTriggerProgrammaticLaunchCompletion();
+    cudaGridDependencySynchronize();
     constexpr int HALF = D / 2;
     constexpr int THREADS_PER_VEC = HALF / 8;            // 8 (D=128) or 4 (D=64)
     const int heads = Hq + Hkv;
@@ -96,14 +87,8 @@ __global__ void __launch_bounds__(128) rope_kv_append_kernel(
     Vec8 out_lo, out_hi;
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-        const double a = static_cast<double>(acdev::bf16_bits_to_float(lo.v[e]));
-        const double bb = static_cast<double>(acdev::bf16_bits_to_float(hi.v[e]));
-        const double cd = static_cast<double>(c[e]);
-        const double sd = static_cast<double>(s[e]);
-        // __dmul_rn/__dadd_rn keep the three operations separate (no contraction); the products
-        // are exact either way, so a fused form would round identically.
-        out_lo.v[e] = f64_to_bf16_rne(__dsub_rn(__dmul_rn(a, cd), __dmul_rn(bb, sd)));
-        out_hi.v[e] = f64_to_bf16_rne(__dadd_rn(__dmul_rn(bb, cd), __dmul_rn(a, sd)));
+        out_lo.v[e] = acdev::rope_first_half(lo.v[e], hi.v[e], c[e], s[e]);
+        out_hi.v[e] = acdev::rope_second_half(lo.v[e], hi.v[e], c[e], s[e]);
     }
     *reinterpret_cast<Vec8*>(dst + i0) = out_lo;
     *reinterpret_cast<Vec8*>(dst + HALF + i0) = out_hi;
@@ -134,13 +119,24 @@ cudaError_t launch_rope_kv_append(const void* q_in, void* q_out, const void* k_n
         static_cast<uint16_t*>(k_cache), static_cast<uint16_t*>(v_cache), stride_page,             \
         stride_token, stride_head, block_table, max_pages_per_seq, context_lens, rope_cos,         \
         rope_sin, max_position, B, Hq, Hkv, page_size, num_pages, status_flag
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
     if (d == 128) {
-        rope_kv_append_kernel<128><<<grid, block, 0, stream>>>(AC_ROPE_ARGS);
+        e = cudaLaunchKernelEx(&cfg, rope_kv_append_kernel<128>, AC_ROPE_ARGS);
     } else {
-        rope_kv_append_kernel<64><<<grid, block, 0, stream>>>(AC_ROPE_ARGS);
+        e = cudaLaunchKernelEx(&cfg, rope_kv_append_kernel<64>, AC_ROPE_ARGS);
     }
 #undef AC_ROPE_ARGS
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace ac

@@ -29,9 +29,11 @@ class DecodeStep:
     """
 
     def __init__(self, w, device="cuda:0", num_splits: int | None = None, layout: str = "token_major",
-                 max_context_len: int | None = None, fused_merge: bool = True):
+                 max_context_len: int | None = None, fused_merge: bool = True,
+                 fused_step: bool = False):
         self.w = w
-        self.fused_merge = bool(fused_merge)
+        self.fused_step = bool(fused_step)             # one launch: RoPE + append + attention + merge
+        self.fused_merge = bool(fused_merge) or self.fused_step
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         ac.ac_init(self.device.index if self.device.index is not None else -1)
@@ -102,13 +104,27 @@ class DecodeStep:
             ac.ac_splitkv_merge(self.workspace, self.num_splits, self.context_lens, self.out, self.B,
                                 self.Hq, self.d, stream)
 
+    def decode_step_fused(self, stream=None) -> None:
+        ac.ac_decode_step_fused(self.q_in, self.q_rot, self.k_new, self.v_new, self.k_cache, self.v_cache,
+                                self.stride_page, self.stride_token, self.stride_head, self.block_table,
+                                self.w.max_pages_per_seq, self.context_lens, self.rope_cos, self.rope_sin,
+                                self.w.max_position, 0.0, self.num_splits,
+                                self.workspace if self.num_splits > 1 else None, self.workspace_bytes,
+                                self.out, self.B, self.Hq, self.Hkv, self.d, self.ps, self.num_pages,
+                                self.max_context_len, self.status_flag, stream)
+
     def step(self, stream=None) -> None:
+        if self.fused_step:
+            self.decode_step_fused(stream)
+            return
         self.rope_kv_append(stream)
         self.attention(stream)
         self.merge(stream)
 
     @property
     def launches_per_step(self) -> int:
+        if self.fused_step:
+            return 1
         return 3 if (self.num_splits > 1 and not self.fused_merge) else 2
 
     def capture(self) -> torch.cuda.CUDAGraph:

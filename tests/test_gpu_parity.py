@@ -43,9 +43,12 @@ def check_out(got, ref, what=""):
 
 
 def run_and_compare(rt, w, num_splits=None, layout="token_major", check_cache=True, fused=True):
+    """fused: False = three launches (RoPE+append, attention, merge); True = merge inside the
+    attention kernel; "step" = the single-launch fused step."""
     import torch
     q_rot, k_after, v_after, out_ref = O.oracle_decode_step(w)
-    st = rt.DecodeStep(w, num_splits=num_splits, layout=layout, fused_merge=fused)
+    st = rt.DecodeStep(w, num_splits=num_splits, layout=layout, fused_merge=bool(fused),
+                       fused_step=(fused == "step"))
     st.step()
     torch.cuda.synchronize()
     assert int(st.status_flag.item()) == 0
@@ -77,8 +80,9 @@ def small(seed, **kw):
     dict(B=5, Hq=28, Hkv=4, page_size=32, num_pages=64, context_lens=[100, 64, 0, 255, 31], inactive_rows=(1, 3)),
     dict(B=2, Hq=32, Hkv=2, context_lens=[500, 77], rope_base=500000.0),
 ])
-def test_rope_append_bit_exact(rt, kw):
-    run_and_compare(rt, small(31, **kw))
+@pytest.mark.parametrize("fused", [True, "step"])
+def test_rope_append_bit_exact(rt, kw, fused):
+    run_and_compare(rt, small(31, **kw), fused=fused)
 
 
 def test_rope_append_bit_exact_with_far_position_angles(rt):
@@ -92,6 +96,7 @@ def test_rope_append_bit_exact_with_far_position_angles(rt):
     w.rope_cos = np.ascontiguousarray(cos[far])
     w.rope_sin = np.ascontiguousarray(sin[far])
     run_and_compare(rt, w)
+    run_and_compare(rt, w, fused="step")
 
 
 def test_rope_constructed_near_tie(rt):
@@ -103,8 +108,9 @@ def test_rope_constructed_near_tie(rt):
     w.k_new[:] = w.q[0]
     w.rope_cos[:] = 1.0
     w.rope_sin[:] = np.float32(-(2.0 ** -8) * (1 + 2.0 ** -20))
-    st, _ = run_and_compare(rt, w)
-    assert (rt.bits_of(st.q_rot)[0, :, :32] == 0x3F82).all()
+    for fused in (True, "step"):
+        st, _ = run_and_compare(rt, w, fused=fused)
+        assert (rt.bits_of(st.q_rot)[0, :, :32] == 0x3F82).all()
 
 
 def test_append_flags_out_of_range_and_writes_nothing(rt):
@@ -141,7 +147,7 @@ def test_append_flags_out_of_range_and_writes_nothing(rt):
     dict(context_lens=[63, 64, 65]),
     dict(B=4, context_lens=[1000, 3, 511, 700], num_pages=200, inactive_rows=(2,)),
 ])
-@pytest.mark.parametrize("splits,fused", [(1, True), (3, True), (3, False)])
+@pytest.mark.parametrize("splits,fused", [(1, True), (3, True), (3, False), (1, "step"), (3, "step")])
 def test_attention_small(rt, kw, splits, fused):
     run_and_compare(rt, small(41, **kw), num_splits=splits, fused=fused)
 
@@ -191,7 +197,7 @@ def test_merge_kernel_alone_against_oracle(rt):
     assert (rt.bits_of(out)[1] == 0).all()
 
 
-@pytest.mark.parametrize("splits,fused", [(1, True), (4, True), (4, False)])
+@pytest.mark.parametrize("splits,fused", [(1, True), (4, True), (4, False), (1, "step"), (4, "step")])
 def test_attention_head_major_layout(rt, splits, fused):
     run_and_compare(rt, small(43, Hq=16, Hkv=4, context_lens=[300, 45, 129]), num_splits=splits,
                     layout="head_major", fused=fused)
@@ -290,6 +296,56 @@ def test_graph_replay_equals_eager_and_tracks_updated_lengths(rt):
     check_out(st2.out_f64(), out_next, "replay with advanced lengths")
 
 
+def test_fused_step_flags_out_of_range_and_writes_nothing(rt):
+    import torch
+    w = small(35, B=3, context_lens=[40, 50, 60], num_pages=32)
+    st = rt.DecodeStep(w, num_splits=2, fused_step=True)
+    bt = w.block_table.copy()
+    bt[0, 40 // 16] = 10_000                  # page id outside the pool
+    st.block_table.copy_(torch.from_numpy(bt))
+    lens = w.context_lens.copy()
+    lens[1] = w.max_position + 5               # position outside the rope table (and the block table)
+    st.context_lens.copy_(torch.from_numpy(lens))
+    before_k, before_v = st.cache_bits()
+    st.step()
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) & 3 == 3
+    after_k, after_v = st.cache_bits()
+    # only row 2 appended
+    changed = np.unique(np.nonzero(after_k != before_k)[0]).tolist()
+    assert changed == [int(w.block_table[2, 60 // 16])]
+    q_rot, k_ref, v_ref, out_ref = O.oracle_decode_step(w)
+    check_out(st.out_f64()[2], out_ref[2], "row untouched by the bad rows")
+
+
+def test_fused_step_graph_replay_advances(rt):
+    import torch
+    w = small(36, B=3, Hq=28, Hkv=4, page_size=32, num_pages=96, context_lens=[600, 31, 257])
+    w.rope_cos, w.rope_sin = W.rope_table(w.max_position + 4, w.d, w.rope_base)
+    _, k1, v1, out1 = O.oracle_decode_step(w)
+    st = rt.DecodeStep(w, num_splits=2, fused_step=True, max_context_len=w.max_context_len + 4)
+    graph = st.capture()
+    fresh = rt.DecodeStep(w, num_splits=2)
+    st.k_cache.copy_(fresh.k_cache); st.v_cache.copy_(fresh.v_cache); st.out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    check_out(st.out_f64(), out1, "fused step replay")
+    kg, vg = st.cache_bits()
+    assert np.array_equal(kg, k1) and np.array_equal(vg, v1)
+    w2 = small(36, B=3, Hq=28, Hkv=4, page_size=32, num_pages=96, context_lens=[600, 31, 257])
+    w2.rope_cos, w2.rope_sin = w.rope_cos, w.rope_sin
+    w2.k_cache, w2.v_cache = k1, v1
+    w2.context_lens = (w2.context_lens + 1).astype(np.int32)
+    _, k2, v2, out2 = O.oracle_decode_step(w2)
+    st.context_lens.copy_(torch.from_numpy(w2.context_lens))
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) == 0
+    check_out(st.out_f64(), out2, "fused step replay, advanced lengths")
+    kg, vg = st.cache_bits()
+    assert np.array_equal(kg, k2) and np.array_equal(vg, v2)
+
+
 def test_peaked_scores(rt):
     w = W.make_workload("peaked", 48, B=2, Hq=16, Hkv=2, d=128, page_size=16, num_pages=300,
                         context_lens=[2000, 1500], rope_base=500000.0, peak_fraction=0.01)
@@ -301,26 +357,29 @@ def test_peaked_scores(rt):
 # the five benchmark workloads, in the launch configuration the benchmark uses (planned splits)
 # ---------------------------------------------------------------------------------------------
 
-def test_workload_tiny(rt):
-    run_and_compare(rt, W.tiny())
+@pytest.mark.parametrize("fused", [True, "step"])
+def test_workload_tiny(rt, fused):
+    run_and_compare(rt, W.tiny(), fused=fused)
 
 
-def test_workload_single_request(rt):
-    run_and_compare(rt, W.single_request())
+@pytest.mark.parametrize("fused", [True, "step"])
+def test_workload_single_request(rt, fused):
+    run_and_compare(rt, W.single_request(), fused=fused)
 
 
+@pytest.mark.parametrize("fused", [True, "step"])
 @pytest.mark.parametrize("batch", W.GRAPH_SWEEP_BATCHES)
-def test_workload_graph_sweep(rt, batch):
+def test_workload_graph_sweep(rt, batch, fused):
     import torch
     w = W.graph_sweep(batch)
-    st, out_ref = run_and_compare(rt, w)
+    st, out_ref = run_and_compare(rt, w, fused=fused)
     graph = st.capture()
     graph.replay()
     torch.cuda.synchronize()
     check_out(st.out_f64(), out_ref, "graph replay")
 
 
-@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("fused", [True, False, "step"])
 def test_workload_continuous_batching(rt, fused):
     run_and_compare(rt, W.continuous_batching(), fused=fused)
 
@@ -357,10 +416,11 @@ def test_fused_merge_repeated_launches_and_row_without_tokens(rt):
     assert int(counters.abs().sum().item()) == 0
 
 
-def test_workload_long_context_sampled_heads(rt):
+@pytest.mark.parametrize("fused_step", [False, True])
+def test_workload_long_context_sampled_heads(rt, fused_step):
     import torch
     w = W.long_context()
-    st = rt.DecodeStep(w)
+    st = rt.DecodeStep(w, fused_step=fused_step)
     st.step()
     torch.cuda.synchronize()
     assert int(st.status_flag.item()) == 0
