@@ -387,7 +387,8 @@ def run_ours(args):
             del st
             torch.cuda.empty_cache()
             for name in ("tiny", "single_request", "continuous_batching") + tuple(
-                    f"graph_sweep_b{b}" for b in W.GRAPH_SWEEP_BATCHES):
+                    f"graph_sweep_b{b}" for b in W.GRAPH_SWEEP_BATCHES) + ("gqa_group16",
+                                                                            "sliding_window_4k"):
                 ww = W.NAMED[name]()
                 us, info = time_in_graph(lambda: runner.DecodeStep(ww, device=device, fused_step=not args.three_launches),
                                          ww.kv_bytes, torch)

@@ -196,6 +196,39 @@ int ac_decode_step_fused(const void* q_in, void* q_rot_out, const void* k_new, c
                          void* out, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
                          int max_context_len, int32_t* status_flag, void* stream);
 
+/* Options of the _ex entry points.  Zero-initialise; unknown fields must stay zero. */
+typedef struct ac_attn_options {
+    int window;      /* > 0: sliding-window attention -- row b attends over its last `window` tokens
+                        only, i.e. tokens max(0, n_b - window) .. n_b - 1 (the paper wires a sliding
+                        window in for one of its model families, "Per-Model Adaptations"); 0: all */
+    int fused_merge; /* ac_paged_decode_attn_ex only: non-zero = behave as ac_paged_decode_attn_fused_merge */
+    int reserved[6];
+} ac_attn_options;
+
+/* ac_paged_decode_attn / ac_paged_decode_attn_fused_merge / ac_decode_step_fused with options
+ * (options == NULL means defaults).  With a window, tokens before the window's start are neither
+ * read (whole tiles) nor weighted (the first tile masks them), so their pages may already have been
+ * recycled; the splits partition the at most window + 63 tokens from the window's start rounded
+ * down to a multiple of 64, so pass min(max_context_len, window + 63) to ac_decode_plan. */
+int ac_paged_decode_attn_ex(const void* q_rot, const void* k_cache, const void* v_cache,
+                            int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                            const int32_t* block_table, int max_pages_per_seq,
+                            const int32_t* context_lens, int new_tokens, float softmax_scale,
+                            int num_splits, void* workspace, size_t workspace_bytes, void* out,
+                            int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                            int max_context_len, int32_t* status_flag, void* stream,
+                            const ac_attn_options* options);
+int ac_decode_step_fused_ex(const void* q_in, void* q_rot_out, const void* k_new, const void* v_new,
+                            void* k_cache, void* v_cache,
+                            int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                            const int32_t* block_table, int max_pages_per_seq,
+                            const int32_t* context_lens,
+                            const float* rope_cos, const float* rope_sin, int max_position,
+                            float softmax_scale, int num_splits, void* workspace, size_t workspace_bytes,
+                            void* out, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                            int max_context_len, int32_t* status_flag, void* stream,
+                            const ac_attn_options* options);
+
 /* A5: merge of the split partials ("cross-CTA merging" of family (iv), here as its own kernel):
  *   M = max_s lse_s,  w_s = exp(lse_s - M),  out[b,hq,:] = sum_s w_s partial_o[b,hq,s,:] / sum_s w_s
  * rounded to bf16.  Splits with lse = -inf are skipped (their partial_o is not read); a row whose

@@ -146,11 +146,13 @@ def gather_kv(cache, block_table_row, n_tokens, page_size, kv_head):
 
 
 def oracle_paged_decode_attn(q_rot, k_cache, v_cache, block_table, context_lens, page_size,
-                             new_tokens=1, softmax_scale=None, return_lse=False):
+                             new_tokens=1, softmax_scale=None, return_lse=False, window=0):
     """out fp64 [B,Hq,d] (and lse fp64 [B,Hq], natural log, of the scaled scores).
 
-    Row b attends over positions 0 .. context_lens[b] + new_tokens - 1.  Inactive rows
-    (context_lens[b] < 0) and rows with nothing to attend give a zero vector and lse = -inf.
+    Row b attends over positions 0 .. n_b - 1 with n_b = context_lens[b] + new_tokens, or, with a
+    sliding window (window > 0; the variant the paper's per-model adaptations mention), over its last
+    `window` positions max(0, n_b - window) .. n_b - 1 only.  Inactive rows (context_lens[b] < 0)
+    and rows with nothing to attend give a zero vector and lse = -inf.
     """
     q_rot = np.asarray(q_rot, dtype=np.uint16)
     B, Hq, d = q_rot.shape
@@ -165,9 +167,10 @@ def oracle_paged_decode_attn(q_rot, k_cache, v_cache, block_table, context_lens,
         n = int(context_lens[b]) + int(new_tokens)
         if n <= 0:
             continue
+        lo = max(0, n - int(window)) if window and window > 0 else 0
         for h in range(Hkv):
-            K = gather_kv(k_cache, block_table[b], n, page_size, h)
-            V = gather_kv(v_cache, block_table[b], n, page_size, h)
+            K = gather_kv(k_cache, block_table[b], n, page_size, h)[lo:]
+            V = gather_kv(v_cache, block_table[b], n, page_size, h)[lo:]
             for g in range(G):
                 hq = h * G + g
                 qv = bf16_to_f64(q_rot[b, hq])
@@ -251,7 +254,7 @@ def oracle_splitkv_merge(partial_o, partial_lse):
     return out, lse
 
 
-def oracle_decode_step(w, softmax_scale=None):
+def oracle_decode_step(w, softmax_scale=None, window=0):
     """Whole step on a workload object (fields as in the seeded generator): append, then attend.
 
     Returns (q_rot bits, k_cache_after bits, v_cache_after bits, out fp64).
@@ -260,5 +263,5 @@ def oracle_decode_step(w, softmax_scale=None):
         w.q, w.k_new, w.v_new, w.k_cache, w.v_cache, w.block_table, w.context_lens,
         w.rope_cos, w.rope_sin, w.page_size)
     out = oracle_paged_decode_attn(q_rot, k_after, v_after, w.block_table, w.context_lens,
-                                   w.page_size, new_tokens=1, softmax_scale=softmax_scale)
+                                   w.page_size, new_tokens=1, softmax_scale=softmax_scale, window=window)
     return q_rot, k_after, v_after, out

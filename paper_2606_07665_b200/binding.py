@@ -25,8 +25,13 @@ EXPORTS = ("ac_init", "ac_status_string", "ac_last_cuda_error", "ac_sm_count", "
            "ac_split_tokens", "ac_workspace_bytes", "ac_rope_kv_append", "ac_paged_decode_attn",
            "ac_splitkv_merge", "ac_decode_step_host", "ac_paged_decode_attn_static_scratch",
            "ac_fused_workspace_bytes", "ac_fused_workspace_reset", "ac_paged_decode_attn_fused_merge",
-           "ac_decode_step_fused")
+           "ac_decode_step_fused", "ac_paged_decode_attn_ex", "ac_decode_step_fused_ex")
 AC_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+class AcAttnOptions(ctypes.Structure):
+    """Mirror of ac_attn_options."""
+    _fields_ = [("window", c_int), ("fused_merge", c_int), ("reserved", c_int * 6)]
 
 
 class AcError(RuntimeError):
@@ -80,6 +85,10 @@ def lib():
                                            c_void_p, c_void_p, c_int, c_float, c_int, c_void_p, c_size_t,
                                            c_void_p] + [c_int] * 7 + [c_void_p, c_void_p])
         L.ac_decode_step_fused.restype = c_int
+        L.ac_paged_decode_attn_ex.argtypes = L.ac_paged_decode_attn.argtypes + [POINTER(AcAttnOptions)]
+        L.ac_paged_decode_attn_ex.restype = c_int
+        L.ac_decode_step_fused_ex.argtypes = L.ac_decode_step_fused.argtypes + [POINTER(AcAttnOptions)]
+        L.ac_decode_step_fused_ex.restype = c_int
         L.ac_splitkv_merge.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p]
         L.ac_splitkv_merge.restype = c_int
         L.ac_decode_step_host.argtypes = ([c_void_p] * 6 + [c_void_p] * 6 + [c_void_p] * 2 + [c_int64] * 3 +
@@ -193,7 +202,39 @@ def ac_decode_step_fused(q_in, q_rot_out, k_new, v_new, k_cache, v_cache, stride
         stride_token, stride_head, _ptr(block_table), max_pages_per_seq, _ptr(context_lens),
         _ptr(rope_cos), _ptr(rope_sin), max_position, softmax_scale, num_splits, _ptr(workspace),
         workspace_bytes, _ptr(out), B, Hq, Hkv, d, page_size, num_pages, max_context_len,
-        _ptr(status_flag), _stream(stream)), "ac_decode_step_fused")
+        _ptr(status_flag), _stream(stream)), "ac_decode_step_fused", "ac_paged_decode_attn_ex", "ac_decode_step_fused_ex")
+
+
+def _options(window: int = 0, fused_merge: bool = False):
+    opt = AcAttnOptions()
+    opt.window = int(window)
+    opt.fused_merge = 1 if fused_merge else 0
+    return ctypes.byref(opt)
+
+
+def ac_paged_decode_attn_ex(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
+                            max_pages_per_seq, context_lens, new_tokens, softmax_scale, num_splits,
+                            workspace, workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages,
+                            max_context_len, status_flag=None, stream=None, window=0, fused_merge=False):
+    _check(lib().ac_paged_decode_attn_ex(
+        _ptr(q_rot), _ptr(k_cache), _ptr(v_cache), stride_page, stride_token, stride_head,
+        _ptr(block_table), max_pages_per_seq, _ptr(context_lens), new_tokens, softmax_scale, num_splits,
+        _ptr(workspace), workspace_bytes, _ptr(out), B, Hq, Hkv, d, page_size, num_pages,
+        max_context_len, _ptr(status_flag), _stream(stream), _options(window, fused_merge)),
+        "ac_paged_decode_attn_ex")
+
+
+def ac_decode_step_fused_ex(q_in, q_rot_out, k_new, v_new, k_cache, v_cache, stride_page, stride_token,
+                            stride_head, block_table, max_pages_per_seq, context_lens, rope_cos, rope_sin,
+                            max_position, softmax_scale, num_splits, workspace, workspace_bytes, out, B,
+                            Hq, Hkv, d, page_size, num_pages, max_context_len, status_flag=None,
+                            stream=None, window=0):
+    _check(lib().ac_decode_step_fused_ex(
+        _ptr(q_in), _ptr(q_rot_out), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), stride_page,
+        stride_token, stride_head, _ptr(block_table), max_pages_per_seq, _ptr(context_lens),
+        _ptr(rope_cos), _ptr(rope_sin), max_position, softmax_scale, num_splits, _ptr(workspace),
+        workspace_bytes, _ptr(out), B, Hq, Hkv, d, page_size, num_pages, max_context_len,
+        _ptr(status_flag), _stream(stream), _options(window)), "ac_decode_step_fused_ex")
 
 
 def ac_splitkv_merge(workspace, num_splits, context_lens, out, B, Hq, d, stream=None):

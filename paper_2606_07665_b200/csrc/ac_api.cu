@@ -266,7 +266,7 @@ static int attn_common(const void* q_rot, const void* k_cache, const void* v_cac
                        float softmax_scale, int num_splits, void* workspace, size_t workspace_bytes,
                        void* out, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
                        int max_context_len, int32_t* status_flag, void* stream, bool fused_merge,
-                       const FusedRopeArgs* rope = nullptr) {
+                       const FusedRopeArgs* rope = nullptr, int window = 0) {
     if (!q_rot || !k_cache || !v_cache || !block_table || !context_lens) return AC_ERR_NULL;
     Shape s{B, Hq, Hkv, d, page_size, num_pages};
     int st = check_shape(s);
@@ -303,11 +303,15 @@ static int attn_common(const void* q_rot, const void* k_cache, const void* v_cac
     st = make_cache_map(&v_map, v_cache, s, stride_page, stride_token, stride_head);
     if (st != AC_OK) return st;
     const float scale = softmax_scale > 0.0f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d));
-    const int split_tokens = split_tokens_for(max_context_len, num_splits);
+    // With a sliding window a row attends over at most window + 63 tokens (its range starts at a
+    // multiple of 64 at or below the window's first token).
+    if (window < 0) return AC_ERR_SHAPE;
+    const int span = (window > 0 && window + 63 < max_context_len) ? window + 63 : max_context_len;
+    const int split_tokens = split_tokens_for(span, num_splits);
     cudaError_t e = launch_paged_decode_attn(k_map, v_map, q_rot, block_table,
                                              max_pages_per_seq, context_lens, new_tokens, scale,
                                              num_splits, split_tokens, partial_o, partial_lse, arrivals,
-                                             out, B, Hq, Hkv, d, page_size, status_flag, rope,
+                                             out, B, Hq, Hkv, d, page_size, status_flag, rope, window,
                                              static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
 }
@@ -362,6 +366,22 @@ int ac_decode_step_fused(const void* q_in, void* q_rot_out, const void* k_new, c
                          int max_position, float softmax_scale, int num_splits, void* workspace,
                          size_t workspace_bytes, void* out, int B, int Hq, int Hkv, int d, int page_size,
                          int num_pages, int max_context_len, int32_t* status_flag, void* stream) {
+    return ac_decode_step_fused_ex(q_in, q_rot_out, k_new, v_new, k_cache, v_cache, stride_page,
+                                   stride_token, stride_head, block_table, max_pages_per_seq,
+                                   context_lens, rope_cos, rope_sin, max_position, softmax_scale,
+                                   num_splits, workspace, workspace_bytes, out, B, Hq, Hkv, d, page_size,
+                                   num_pages, max_context_len, status_flag, stream, nullptr);
+}
+
+int ac_decode_step_fused_ex(const void* q_in, void* q_rot_out, const void* k_new, const void* v_new,
+                            void* k_cache, void* v_cache, int64_t stride_page, int64_t stride_token,
+                            int64_t stride_head, const int32_t* block_table, int max_pages_per_seq,
+                            const int32_t* context_lens, const float* rope_cos, const float* rope_sin,
+                            int max_position, float softmax_scale, int num_splits, void* workspace,
+                            size_t workspace_bytes, void* out, int B, int Hq, int Hkv, int d,
+                            int page_size, int num_pages, int max_context_len, int32_t* status_flag,
+                            void* stream, const ac_attn_options* options) {
+    const int window = options != nullptr ? options->window : 0;
     if (!q_in || !k_new || !v_new || !rope_cos || !rope_sin) return AC_ERR_NULL;
     if (max_position <= 0) return AC_ERR_SHAPE;
     if (q_rot_out == q_in) return AC_ERR_UNSUPPORTED;      // other CTAs still read the raw rows
@@ -384,7 +404,22 @@ int ac_decode_step_fused(const void* q_in, void* q_rot_out, const void* k_new, c
     return attn_common(q_in, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
                        max_pages_per_seq, context_lens, 1, softmax_scale, num_splits, workspace,
                        workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages, max_context_len,
-                       status_flag, stream, true, &rope);
+                       status_flag, stream, true, &rope, window);
+}
+
+int ac_paged_decode_attn_ex(const void* q_rot, const void* k_cache, const void* v_cache,
+                            int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                            const int32_t* block_table, int max_pages_per_seq,
+                            const int32_t* context_lens, int new_tokens, float softmax_scale,
+                            int num_splits, void* workspace, size_t workspace_bytes, void* out, int B,
+                            int Hq, int Hkv, int d, int page_size, int num_pages, int max_context_len,
+                            int32_t* status_flag, void* stream, const ac_attn_options* options) {
+    const bool fused = options != nullptr && options->fused_merge != 0;
+    const int window = options != nullptr ? options->window : 0;
+    return attn_common(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
+                       max_pages_per_seq, context_lens, new_tokens, softmax_scale, num_splits, workspace,
+                       workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages, max_context_len,
+                       status_flag, stream, fused, nullptr, window);
 }
 
 int ac_splitkv_merge(const void* workspace, int num_splits, const int32_t* context_lens, void* out,

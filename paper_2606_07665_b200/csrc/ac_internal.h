@@ -64,7 +64,7 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
                                      int num_splits, int split_tokens, float* partial_o,
                                      float* partial_lse, int32_t* arrivals, void* out, int B, int Hq,
                                      int Hkv, int d, int page_size, int32_t* status_flag,
-                                     const FusedRopeArgs* rope, cudaStream_t stream);
+                                     const FusedRopeArgs* rope, int window, cudaStream_t stream);
 cudaError_t launch_splitkv_merge(const float* partial_o, const float* partial_lse, int num_splits,
                                  const int32_t* context_lens, void* out, int B, int Hq, int d,
                                  cudaStream_t stream);

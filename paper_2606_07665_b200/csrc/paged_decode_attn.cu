@@ -81,6 +81,7 @@ struct AttnParams {
     int Hq, Hkv, page_size;
     int fused_merge;              // 1: the last CTA of a (request, KV head) merges the splits itself
     int longest_first;            // 1: grid row y serves the request with the y-th longest context
+    int window;                   // > 0: attend over the last `window` tokens of each row only
 };
 
 template <int D, bool WIDE, bool ROPE>
@@ -139,8 +140,8 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     // written is independent of that kernel, so with a programmatic dependent launch it overlaps the
     // preceding kernel's execution.  The preceding kernel is either the RoPE + append kernel of this
     // step (writes slot ctx) or the fused step of the previous token (wrote slot ctx - 1).
-    const int tok_begin = split * p.split_tokens;
-    const int tile_begin = tok_begin / TILE;
+    int tok_begin = split * p.split_tokens;          // both move up when a sliding window applies
+    int tile_begin = tok_begin / TILE;
     auto tile_token0 = [&](int j) { return (tile_begin + warp + j * WARPS) * TILE; };
     const int32_t* bt_row = p.block_table + static_cast<size_t>(b) * p.max_pages_per_seq;
     auto load_page_id = [&](int j) {
@@ -155,7 +156,19 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
 
     int n_tokens = ctx < 0 ? 0 : ctx + p.new_tokens;
     n_tokens = min(n_tokens, p.max_pages_per_seq * p.page_size);
-    const int tok_end = min(tok_begin + p.split_tokens, n_tokens);
+    // Sliding window: the row attends over tokens [tok_lo, n_tokens).  The splits partition the range
+    // that starts at tok_lo rounded down to a multiple of 64; tiles wholly below tok_lo are skipped
+    // and the first tile masks its leading tokens.
+    int tok_lo = 0, window_base = 0;
+    if (p.window > 0) {
+        tok_lo = max(0, n_tokens - p.window);
+        window_base = tok_lo / 64 * 64;
+        tok_begin = max(window_base + split * p.split_tokens, tok_lo / TILE * TILE);
+        tile_begin = tok_begin / TILE;
+#pragma unroll
+        for (int s = 0; s < STAGES; ++s) page_first[s] = load_page_id(s);     // the range moved
+    }
+    const int tok_end = min(window_base + (split + 1) * p.split_tokens, n_tokens);
 
     if (tok_begin >= tok_end) {
         // Nothing to attend over in this split.  The buffers written here may still be in use by
@@ -363,6 +376,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
         }
         const int tok0 = tile_token0(j);
         const int n_valid = tok_end - tok0;                    // >= 1; < 16 only on the last tile
+        const int lo_valid = tok_lo - tok0;                    // > 0 only on the first tile of a window
 
         if (ROPE && j == append_j && append_ok) {
             // The tile just loaded still has the stale slot of the new token: overwrite that row with
@@ -404,21 +418,26 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
             }
         }
 
-        if (n_valid < TILE) {
-            // Slots past the request's length hold arbitrary bits: mask their scores and clear their
-            // V rows (0 * NaN would poison the product).
+        if (n_valid < TILE || lo_valid > 0) {
+            // Slots past the request's length hold arbitrary bits, and tokens before a sliding
+            // window's start are not attended: mask their scores and clear their V rows (0 * NaN
+            // would poison the product).
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (nt * 8 + 2 * t + (e & 1) >= n_valid) s[nt][e] = -INFINITY;
+                for (int e = 0; e < 4; ++e) {
+                    const int col = nt * 8 + 2 * t + (e & 1);
+                    if (col >= n_valid || col < lo_valid) s[nt][e] = -INFINITY;
+                }
             const int chunks_per_row = L::HALVES * 8;
-            for (int idx = lane; idx < (TILE - n_valid) * chunks_per_row; idx += 32) {
-                const int row = n_valid + idx / chunks_per_row;
+            for (int idx = lane; idx < TILE * chunks_per_row; idx += 32) {
+                const int row = idx / chunks_per_row;
                 const int rem = idx % chunks_per_row;
-                uint4* dstz = reinterpret_cast<uint4*>(smem_gen + (vbase - smem_base) +
-                                                       (rem >> 3) * L::HALF_BYTES + row * 128 + (rem & 7) * 16);
-                *dstz = make_uint4(0u, 0u, 0u, 0u);
+                if (row >= n_valid || row < lo_valid) {
+                    uint4* dstz = reinterpret_cast<uint4*>(smem_gen + (vbase - smem_base) +
+                                                           (rem >> 3) * L::HALF_BYTES + row * 128 + (rem & 7) * 16);
+                    *dstz = make_uint4(0u, 0u, 0u, 0u);
+                }
             }
             __syncwarp();
         }
@@ -540,7 +559,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     // Publish this CTA's partials, take a ticket, and let the holder of the last ticket do the merge.
     // Nobody waits for anybody: CTAs that are not last simply exit.
     __shared__ int s_is_last;
-    const int n_active = (n_tokens + p.split_tokens - 1) / p.split_tokens;     // splits with tokens
+    const int n_active = (n_tokens - window_base + p.split_tokens - 1) / p.split_tokens;   // splits with tokens
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -655,8 +674,9 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
                                      int num_splits, int split_tokens, float* partial_o,
                                      float* partial_lse, int32_t* arrivals, void* out, int B, int Hq,
                                      int Hkv, int d, int page_size, int32_t* status_flag,
-                                     const FusedRopeArgs* rope, cudaStream_t stream) {
+                                     const FusedRopeArgs* rope, int window, cudaStream_t stream) {
     AttnParams p;
+    p.window = window > 0 ? window : 0;
     p.q_rot_out = nullptr;
     p.k_new = p.v_new = nullptr;
     p.k_cache = p.v_cache = nullptr;

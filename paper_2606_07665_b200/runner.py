@@ -30,8 +30,9 @@ class DecodeStep:
 
     def __init__(self, w, device="cuda:0", num_splits: int | None = None, layout: str = "token_major",
                  max_context_len: int | None = None, fused_merge: bool = True,
-                 fused_step: bool = False):
+                 fused_step: bool = False, window: int = 0):
         self.w = w
+        self.window = int(window) if window else int(getattr(w, "window", 0))   # > 0: sliding window
         self.fused_step = bool(fused_step)             # one launch: RoPE + append + attention + merge
         self.fused_merge = bool(fused_merge) or self.fused_step
         self.device = torch.device(device)
@@ -69,11 +70,14 @@ class DecodeStep:
         self.set_splits(num_splits)
 
     def set_splits(self, num_splits: int | None) -> None:
+        span = self.max_context_len
+        if self.window > 0:
+            span = min(span, self.window + 63)         # tokens a row can attend over, as the kernel counts
         if num_splits is None:
-            num_splits, _, _ = ac.ac_decode_plan(self.B, self.Hq, self.Hkv, self.d, self.ps,
-                                                 self.max_context_len, ac.ac_sm_count())
+            num_splits, _, _ = ac.ac_decode_plan(self.B, self.Hq, self.Hkv, self.d, self.ps, span,
+                                                 ac.ac_sm_count())
         self.num_splits = int(num_splits)
-        self.split_tokens = ac.ac_split_tokens(self.max_context_len, self.num_splits)
+        self.split_tokens = ac.ac_split_tokens(span, self.num_splits)
         # sized for either merge flavour: partials, then the fused path's arrival counters
         self.workspace_bytes = ac.ac_fused_workspace_bytes(self.B, self.Hq, self.Hkv, self.d,
                                                            self.num_splits)
@@ -91,6 +95,16 @@ class DecodeStep:
                              self.num_pages, self.status_flag, stream)
 
     def attention(self, stream=None, new_tokens: int = 1, q=None) -> None:
+        if self.window > 0:
+            ac.ac_paged_decode_attn_ex(self.q_rot if q is None else q, self.k_cache, self.v_cache,
+                                       self.stride_page, self.stride_token, self.stride_head,
+                                       self.block_table, self.w.max_pages_per_seq, self.context_lens,
+                                       new_tokens, 0.0, self.num_splits,
+                                       self.workspace if self.num_splits > 1 else None,
+                                       self.workspace_bytes, self.out, self.B, self.Hq, self.Hkv, self.d,
+                                       self.ps, self.num_pages, self.max_context_len, self.status_flag,
+                                       stream, window=self.window, fused_merge=self.fused_merge)
+            return
         fn = ac.ac_paged_decode_attn_fused_merge if self.fused_merge else ac.ac_paged_decode_attn
         fn(self.q_rot if q is None else q, self.k_cache, self.v_cache,
                                 self.stride_page, self.stride_token, self.stride_head, self.block_table,
@@ -105,13 +119,13 @@ class DecodeStep:
                                 self.Hq, self.d, stream)
 
     def decode_step_fused(self, stream=None) -> None:
-        ac.ac_decode_step_fused(self.q_in, self.q_rot, self.k_new, self.v_new, self.k_cache, self.v_cache,
-                                self.stride_page, self.stride_token, self.stride_head, self.block_table,
-                                self.w.max_pages_per_seq, self.context_lens, self.rope_cos, self.rope_sin,
-                                self.w.max_position, 0.0, self.num_splits,
-                                self.workspace if self.num_splits > 1 else None, self.workspace_bytes,
-                                self.out, self.B, self.Hq, self.Hkv, self.d, self.ps, self.num_pages,
-                                self.max_context_len, self.status_flag, stream)
+        ac.ac_decode_step_fused_ex(self.q_in, self.q_rot, self.k_new, self.v_new, self.k_cache,
+                                   self.v_cache, self.stride_page, self.stride_token, self.stride_head,
+                                   self.block_table, self.w.max_pages_per_seq, self.context_lens,
+                                   self.rope_cos, self.rope_sin, self.w.max_position, 0.0, self.num_splits,
+                                   self.workspace if self.num_splits > 1 else None, self.workspace_bytes,
+                                   self.out, self.B, self.Hq, self.Hkv, self.d, self.ps, self.num_pages,
+                                   self.max_context_len, self.status_flag, stream, window=self.window)
 
     def step(self, stream=None) -> None:
         if self.fused_step:

@@ -98,6 +98,7 @@ class DecodeWorkload:
     rope_sin: np.ndarray              # float32 [max_position, d/2]
     poison_page: int
     extra: dict = field(default_factory=dict)
+    window: int = 0                   # > 0: the step uses sliding-window attention of this length
 
     @property
     def max_pages_per_seq(self) -> int:
@@ -115,8 +116,10 @@ class DecodeWorkload:
 
     @property
     def attended_tokens(self) -> int:
-        act = self.context_lens[self.context_lens >= 0].astype(np.int64)
-        return int((act + 1).sum())
+        act = self.context_lens[self.context_lens >= 0].astype(np.int64) + 1
+        if self.window > 0:
+            act = np.minimum(act, self.window)
+        return int(act.sum())
 
     @property
     def kv_bytes(self) -> int:
@@ -238,10 +241,28 @@ def graph_sweep(batch: int) -> DecodeWorkload:
                          page_size=32, num_pages=pool, len_range=(512, 2048), rope_base=1000000.0)
 
 
+def gqa_group16() -> DecodeWorkload:
+    """High-ratio GQA (32 query : 2 KV heads, the shape the paper reports its generated kernel
+    collapsing on): batch 16, lengths uniform in [2048, 8192], head_dim 128, page_size 16."""
+    return make_workload("gqa_group16", 60, B=16, Hq=32, Hkv=2, d=128, page_size=16, num_pages=10000,
+                         len_range=(2048, 8192), rope_base=10000.0)
+
+
+def sliding_window_4k() -> DecodeWorkload:
+    """Sliding-window decode (window 4096, the variant the paper wires in for one model family):
+    batch 32, lengths uniform in [4096, 12288], 32 query / 8 KV heads, head_dim 128, page_size 16."""
+    w = make_workload("sliding_window_4k", 61, B=32, Hq=32, Hkv=8, d=128, page_size=16, num_pages=26000,
+                      len_range=(4096, 12288), rope_base=1000000.0)
+    w.window = 4096
+    return w
+
+
 NAMED = {
     "tiny": tiny,
     "single_request": single_request,
     "continuous_batching": continuous_batching,
     "long_context": long_context,
     **{f"graph_sweep_b{b}": (lambda b=b: graph_sweep(b)) for b in GRAPH_SWEEP_BATCHES},
+    "gqa_group16": gqa_group16,
+    "sliding_window_4k": sliding_window_4k,
 }

@@ -42,13 +42,14 @@ def check_out(got, ref, what=""):
     return worst
 
 
-def run_and_compare(rt, w, num_splits=None, layout="token_major", check_cache=True, fused=True):
+def run_and_compare(rt, w, num_splits=None, layout="token_major", check_cache=True, fused=True,
+                    window=0):
     """fused: False = three launches (RoPE+append, attention, merge); True = merge inside the
     attention kernel; "step" = the single-launch fused step."""
     import torch
-    q_rot, k_after, v_after, out_ref = O.oracle_decode_step(w)
+    q_rot, k_after, v_after, out_ref = O.oracle_decode_step(w, window=window)
     st = rt.DecodeStep(w, num_splits=num_splits, layout=layout, fused_merge=bool(fused),
-                       fused_step=(fused == "step"))
+                       fused_step=(fused == "step"), window=window)
     st.step()
     torch.cuda.synchronize()
     assert int(st.status_flag.item()) == 0
@@ -346,6 +347,23 @@ def test_fused_step_graph_replay_advances(rt):
     assert np.array_equal(kg, k2) and np.array_equal(vg, v2)
 
 
+@pytest.mark.parametrize("fused", [False, True, "step"])
+@pytest.mark.parametrize("window,splits", [(1, 1), (7, 1), (16, 2), (100, 1), (100, 3), (333, 2), (5000, 2)])
+def test_sliding_window(rt, window, splits, fused):
+    # windows that start inside a tile, on a tile edge, before the first token, and rows shorter than
+    # the window; everything before the window is poisoned to prove it is neither read nor weighted
+    w = small(51, B=4, Hq=16, Hkv=2, context_lens=[900, 5, 333, 99], num_pages=160, inactive_rows=(1,))
+    for b in range(w.B):
+        n = int(w.context_lens[b]) + 1
+        if n <= 0:
+            continue
+        for t in range(0, max(0, n - window)):
+            pg, sl = w.block_table[b, t // w.page_size], t % w.page_size
+            w.k_cache[pg, sl] = 0x7FC0
+            w.v_cache[pg, sl] = 0x7FC0
+    run_and_compare(rt, w, num_splits=splits, fused=fused, window=window)
+
+
 def test_peaked_scores(rt):
     w = W.make_workload("peaked", 48, B=2, Hq=16, Hkv=2, d=128, page_size=16, num_pages=300,
                         context_lens=[2000, 1500], rope_base=500000.0, peak_fraction=0.01)
@@ -414,6 +432,17 @@ def test_fused_merge_repeated_launches_and_row_without_tokens(rt):
     n = st.B * st.Hq * st.num_splits * (st.d + 1)
     counters = st.workspace.view(torch.int32)[n:n + st.B * st.Hkv]
     assert int(counters.abs().sum().item()) == 0
+
+
+@pytest.mark.parametrize("fused", [True, "step"])
+def test_workload_gqa_group16(rt, fused):
+    run_and_compare(rt, W.gqa_group16(), fused=fused)
+
+
+@pytest.mark.parametrize("fused", [True, "step"])
+def test_workload_sliding_window_4k(rt, fused):
+    w = W.sliding_window_4k()
+    run_and_compare(rt, w, fused=fused, window=w.window)
 
 
 @pytest.mark.parametrize("fused_step", [False, True])

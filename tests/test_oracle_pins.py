@@ -450,6 +450,40 @@ def test_peaked_workload_matches_brute_force():
     assert np.abs(out - brute_force_attention(w, q_rot, k_after, v_after)).max() < 1e-14
 
 
+def test_sliding_window_pins():
+    w = tiny_case(seed=18, lens=(29, 11), ps=4, pool=24)
+    q_rot, k_after, v_after, full = O.oracle_decode_step(w)
+    # a window at least as long as the context changes nothing
+    assert np.array_equal(O.oracle_decode_step(w, window=30)[3], full)
+    assert np.array_equal(O.oracle_decode_step(w, window=1000)[3], full)
+    # a window of one token returns the newest v exactly
+    one = O.oracle_decode_step(w, window=1)[3]
+    G = w.Hq // w.Hkv
+    for b in range(w.B):
+        for hq in range(w.Hq):
+            assert np.array_equal(one[b, hq], O.bf16_to_f64(w.v_new[b, hq // G]))
+    # brute force over the last 7 tokens, written with explicit indexing
+    win = O.oracle_decode_step(w, window=7)[3]
+    for b in range(w.B):
+        n = int(w.context_lens[b]) + 1
+        for hq in range(w.Hq):
+            h = hq // G
+            toks = list(range(max(0, n - 7), n))
+            qv = O.bf16_to_f64(q_rot[b, hq])
+            sc = [float(O.bf16_to_f64(k_after[w.block_table[b, t // 4], t % 4, h]) @ qv) / math.sqrt(w.d) for t in toks]
+            mx = max(sc)
+            ws = [math.exp(x - mx) for x in sc]
+            ref = sum(wt * O.bf16_to_f64(v_after[w.block_table[b, t // 4], t % 4, h]) for wt, t in zip(ws, toks)) / sum(ws)
+            assert np.abs(win[b, hq] - ref).max() < 1e-14
+    # tokens before the window may hold anything
+    k_bad, v_bad = k_after.copy(), v_after.copy()
+    for t in range(0, 30 - 7):
+        k_bad[w.block_table[0, t // 4], t % 4] = 0x7FC0
+        v_bad[w.block_table[0, t // 4], t % 4] = 0x7FC0
+    again = O.oracle_paged_decode_attn(q_rot, k_bad, v_bad, w.block_table, w.context_lens, w.page_size, window=7)
+    assert np.array_equal(again[0], win[0])
+
+
 def test_tiny_workload_oracle_result_is_frozen():
     import importlib.util
     import os
