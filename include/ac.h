@@ -126,6 +126,32 @@ int ac_rope_kv_append(const void* q_in, void* q_out, const void* k_new, const vo
                       int B, int Hq, int Hkv, int d, int page_size, int num_pages,
                       int32_t* status_flag, void* stream);
 
+/* Prelude variants of A1 (the paper's attention-prelude family (i) names "optionally ... per-head
+ * Q/K RMSNorm"; its per-model adaptations mention partial rotary embeddings).  Zero-initialise. */
+typedef struct ac_rope_options {
+    int rotary_dim;            /* 0 or d: rotate the whole vector; else even, < d: only elements
+                                  [0, rotary_dim) are rotated, the rest pass through; the rope tables
+                                  are then [max_position, rotary_dim/2] */
+    int interleaved;           /* 0: pair element i with i + rotary_dim/2; 1: pair 2i with 2i + 1 */
+    const void* q_norm_weight; /* device bf16 [d] or NULL: RMSNorm of every q head vector before the
+                                  rotation: y = bf16(bf16(x / sqrt(mean(x^2) + eps)) * w) */
+    const void* k_norm_weight; /* same for k (v is never normalised) */
+    float norm_eps;
+    int reserved[4];
+} ac_rope_options;
+
+/* ac_rope_kv_append with options (NULL = plain call).  Everything else as ac_rope_kv_append; the
+ * rotation keeps its exact-then-round arithmetic, the norm is evaluated in fp64 (sum of squares,
+ * square root and division correctly rounded) and rounded to bf16 where the formula above says. */
+int ac_rope_kv_append_ex(const void* q_in, void* q_out, const void* k_new, const void* v_new,
+                         void* k_cache, void* v_cache,
+                         int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                         const int32_t* block_table, int max_pages_per_seq,
+                         const int32_t* context_lens,
+                         const float* rope_cos, const float* rope_sin, int max_position,
+                         int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                         int32_t* status_flag, void* stream, const ac_rope_options* options);
+
 /* A4: paged decode attention, family (iv).  Row b attends over tokens 0 .. n_b - 1 with
  * n_b = context_lens[b] + new_tokens (new_tokens = 1 right after ac_rope_kv_append, 0 to attend
  * over the cached tokens only); token t lives in page block_table[b, t / page_size], slot

@@ -130,6 +130,83 @@ def oracle_rope_kv_append(q, k_new, v_new, k_cache, v_cache, block_table, contex
 
 
 # --------------------------------------------------------------------------------------------
+# Prelude variants of A1: per-head RMSNorm, partial rotary, interleaved pairing
+# --------------------------------------------------------------------------------------------
+
+
+def rms_norm_bf16(x_bits: np.ndarray, weight_bits: np.ndarray, eps: float) -> np.ndarray:
+    """Per-vector RMSNorm of bf16 vectors x[..., d] with a bf16 weight[d]; bf16 bits out.
+
+    y = bf16( bf16( x / sqrt(mean(x^2) + eps) ) * w ): normalise in high precision, round to the
+    model dtype, scale by the weight, round again (the attention-prelude family names the norm only
+    as "per-head Q/K RMSNorm"; this is the usual decoder implementation).  The mean of squares is the
+    exactly rounded sum (math.fsum) divided by d; eps is the fp32 value given.
+    """
+    import math
+    x = bf16_to_f64(x_bits)
+    w = bf16_to_f64(weight_bits)
+    d = x.shape[-1]
+    flat = x.reshape(-1, d)
+    out = np.empty(flat.shape, dtype=np.uint16)
+    eps64 = float(np.float32(eps))
+    for r in range(flat.shape[0]):
+        ss = math.fsum(float(v) * float(v) for v in flat[r])
+        inv = 1.0 / math.sqrt(ss / d + eps64)
+        y1 = f64_to_bf16_rne(flat[r] * inv)
+        out[r] = f64_to_bf16_rne(bf16_to_f64(y1) * w)
+    return out.reshape(x.shape)
+
+
+def rope_rotate_variant_bf16(x_bits, cos_row, sin_row, rotary_dim=None, interleaved=False):
+    """Rotation of the first rotary_dim elements of x[..., d] (bf16 bits), the rest passed through.
+
+    Half-split pairing: (x_i, x_{i+R/2}); interleaved: (x_{2i}, x_{2i+1}); i < R/2, angle i.
+    Same exact-then-round arithmetic as rope_rotate_bf16.
+    """
+    x_bits = np.asarray(x_bits, dtype=np.uint16)
+    d = x_bits.shape[-1]
+    R = d if not rotary_dim else int(rotary_dim)
+    out = x_bits.copy()
+    x = bf16_to_f64(x_bits)
+    c = np.asarray(cos_row, dtype=np.float64)[:R // 2]
+    s = np.asarray(sin_row, dtype=np.float64)[:R // 2]
+    if interleaved:
+        a = x[..., 0:R:2]
+        b = x[..., 1:R:2]
+        out[..., 0:R:2] = f64_to_bf16_rne(a * c - b * s)
+        out[..., 1:R:2] = f64_to_bf16_rne(b * c + a * s)
+    else:
+        a = x[..., :R // 2]
+        b = x[..., R // 2:R]
+        out[..., :R // 2] = f64_to_bf16_rne(a * c - b * s)
+        out[..., R // 2:R] = f64_to_bf16_rne(b * c + a * s)
+    return out
+
+
+def oracle_rope_kv_append_ex(q, k_new, v_new, k_cache, v_cache, block_table, context_lens,
+                             rope_cos, rope_sin, page_size, rotary_dim=None, interleaved=False,
+                             q_norm_weight=None, k_norm_weight=None, norm_eps=0.0):
+    """oracle_rope_kv_append with the prelude variants: optional RMSNorm of q / k head vectors first,
+    then the (partial, half-split or interleaved) rotation, then the append.  v is never touched."""
+    q_rot = np.array(q, dtype=np.uint16, copy=True)
+    k_out = np.array(k_cache, dtype=np.uint16, copy=True)
+    v_out = np.array(v_cache, dtype=np.uint16, copy=True)
+    for b in range(q_rot.shape[0]):
+        p = int(context_lens[b])
+        if p < 0:
+            continue
+        qb = q[b] if q_norm_weight is None else rms_norm_bf16(q[b], q_norm_weight, norm_eps)
+        kb = k_new[b] if k_norm_weight is None else rms_norm_bf16(k_new[b], k_norm_weight, norm_eps)
+        q_rot[b] = rope_rotate_variant_bf16(qb, rope_cos[p], rope_sin[p], rotary_dim, interleaved)
+        k_rot = rope_rotate_variant_bf16(kb, rope_cos[p], rope_sin[p], rotary_dim, interleaved)
+        page = int(block_table[b, p // page_size])
+        slot = p % page_size
+        k_out[page, slot] = k_rot
+        v_out[page, slot] = v_new[b]
+    return q_rot, k_out, v_out
+
+
+# --------------------------------------------------------------------------------------------
 # A4 + A5 as one definition: softmax(q K^T * scale) V per query head over the gathered pages
 # --------------------------------------------------------------------------------------------
 

@@ -25,13 +25,20 @@ EXPORTS = ("ac_init", "ac_status_string", "ac_last_cuda_error", "ac_sm_count", "
            "ac_split_tokens", "ac_workspace_bytes", "ac_rope_kv_append", "ac_paged_decode_attn",
            "ac_splitkv_merge", "ac_decode_step_host", "ac_paged_decode_attn_static_scratch",
            "ac_fused_workspace_bytes", "ac_fused_workspace_reset", "ac_paged_decode_attn_fused_merge",
-           "ac_decode_step_fused", "ac_paged_decode_attn_ex", "ac_decode_step_fused_ex")
+           "ac_decode_step_fused", "ac_paged_decode_attn_ex", "ac_decode_step_fused_ex",
+           "ac_rope_kv_append_ex")
 AC_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class AcAttnOptions(ctypes.Structure):
     """Mirror of ac_attn_options."""
     _fields_ = [("window", c_int), ("fused_merge", c_int), ("reserved", c_int * 6)]
+
+
+class AcRopeOptions(ctypes.Structure):
+    """Mirror of ac_rope_options."""
+    _fields_ = [("rotary_dim", c_int), ("interleaved", c_int), ("q_norm_weight", c_void_p),
+                ("k_norm_weight", c_void_p), ("norm_eps", c_float), ("reserved", c_int * 4)]
 
 
 class AcError(RuntimeError):
@@ -71,6 +78,8 @@ def lib():
         L.ac_rope_kv_append.argtypes = ([c_void_p] * 6 + [c_int64] * 3 + [c_void_p, c_int, c_void_p,
                                         c_void_p, c_void_p, c_int] + [c_int] * 6 + [c_void_p, c_void_p])
         L.ac_rope_kv_append.restype = c_int
+        L.ac_rope_kv_append_ex.argtypes = L.ac_rope_kv_append.argtypes + [POINTER(AcRopeOptions)]
+        L.ac_rope_kv_append_ex.restype = c_int
         L.ac_paged_decode_attn.argtypes = ([c_void_p] * 3 + [c_int64] * 3 + [c_void_p, c_int, c_void_p,
                                            c_int, c_float, c_int, c_void_p, c_size_t, c_void_p] +
                                            [c_int] * 7 + [c_void_p, c_void_p])
@@ -160,6 +169,25 @@ def ac_rope_kv_append(q_in, q_out, k_new, v_new, k_cache, v_cache, stride_page, 
            "ac_rope_kv_append")
 
 
+def ac_rope_kv_append_ex(q_in, q_out, k_new, v_new, k_cache, v_cache, stride_page, stride_token,
+                         stride_head, block_table, max_pages_per_seq, context_lens, rope_cos, rope_sin,
+                         max_position, B, Hq, Hkv, d, page_size, num_pages, status_flag=None, stream=None,
+                         rotary_dim=0, interleaved=False, q_norm_weight=None, k_norm_weight=None,
+                         norm_eps=0.0):
+    opt = AcRopeOptions()
+    opt.rotary_dim = int(rotary_dim)
+    opt.interleaved = 1 if interleaved else 0
+    opt.q_norm_weight = _ptr(q_norm_weight)
+    opt.k_norm_weight = _ptr(k_norm_weight)
+    opt.norm_eps = float(norm_eps)
+    _check(lib().ac_rope_kv_append_ex(_ptr(q_in), _ptr(q_out), _ptr(k_new), _ptr(v_new), _ptr(k_cache),
+                                      _ptr(v_cache), stride_page, stride_token, stride_head,
+                                      _ptr(block_table), max_pages_per_seq, _ptr(context_lens),
+                                      _ptr(rope_cos), _ptr(rope_sin), max_position, B, Hq, Hkv, d,
+                                      page_size, num_pages, _ptr(status_flag), _stream(stream),
+                                      ctypes.byref(opt)), "ac_rope_kv_append_ex")
+
+
 def ac_paged_decode_attn(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
                          max_pages_per_seq, context_lens, new_tokens, softmax_scale, num_splits,
                          workspace, workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages,
@@ -202,7 +230,8 @@ def ac_decode_step_fused(q_in, q_rot_out, k_new, v_new, k_cache, v_cache, stride
         stride_token, stride_head, _ptr(block_table), max_pages_per_seq, _ptr(context_lens),
         _ptr(rope_cos), _ptr(rope_sin), max_position, softmax_scale, num_splits, _ptr(workspace),
         workspace_bytes, _ptr(out), B, Hq, Hkv, d, page_size, num_pages, max_context_len,
-        _ptr(status_flag), _stream(stream)), "ac_decode_step_fused", "ac_paged_decode_attn_ex", "ac_decode_step_fused_ex")
+        _ptr(status_flag), _stream(stream)), "ac_decode_step_fused", "ac_paged_decode_attn_ex", "ac_decode_step_fused_ex",
+           "ac_rope_kv_append_ex")
 
 
 def _options(window: int = 0, fused_merge: bool = False):

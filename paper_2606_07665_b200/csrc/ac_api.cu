@@ -231,12 +231,12 @@ int ac_decode_plan(int B, int Hq, int Hkv, int d, int page_size, int max_context
     return AC_OK;
 }
 
-int ac_rope_kv_append(const void* q_in, void* q_out, const void* k_new, const void* v_new,
-                      void* k_cache, void* v_cache, int64_t stride_page, int64_t stride_token,
-                      int64_t stride_head, const int32_t* block_table, int max_pages_per_seq,
-                      const int32_t* context_lens, const float* rope_cos, const float* rope_sin,
-                      int max_position, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
-                      int32_t* status_flag, void* stream) {
+int ac_rope_kv_append_ex(const void* q_in, void* q_out, const void* k_new, const void* v_new,
+                         void* k_cache, void* v_cache, int64_t stride_page, int64_t stride_token,
+                         int64_t stride_head, const int32_t* block_table, int max_pages_per_seq,
+                         const int32_t* context_lens, const float* rope_cos, const float* rope_sin,
+                         int max_position, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                         int32_t* status_flag, void* stream, const ac_rope_options* options) {
     if (!q_in || !q_out || !k_new || !v_new || !k_cache || !v_cache || !block_table || !context_lens ||
         !rope_cos || !rope_sin)
         return AC_ERR_NULL;
@@ -249,15 +249,45 @@ int ac_rope_kv_append(const void* q_in, void* q_out, const void* k_new, const vo
     if (!aligned16(q_in) || !aligned16(q_out) || !aligned16(k_new) || !aligned16(v_new) ||
         !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(rope_cos) || !aligned16(rope_sin))
         return AC_ERR_ALIGN;
+    RopeVariant variant;
+    const RopeVariant* vp = nullptr;
+    if (options != nullptr) {
+        const int rd = options->rotary_dim == 0 ? d : options->rotary_dim;
+        if (rd < 2 || rd > d || (rd & 1)) return AC_ERR_SHAPE;
+        const bool plain = rd == d && !options->interleaved && !options->q_norm_weight &&
+                           !options->k_norm_weight;
+        if (!plain) {
+            variant.rotary_dim = rd;
+            variant.interleaved = options->interleaved ? 1 : 0;
+            variant.q_norm_weight = options->q_norm_weight;
+            variant.k_norm_weight = options->k_norm_weight;
+            variant.norm_eps = options->norm_eps;
+            if ((variant.q_norm_weight || variant.k_norm_weight) && !(options->norm_eps >= 0.0f))
+                return AC_ERR_SHAPE;
+            vp = &variant;
+        }
+    }
     int dev;
     st = current_ready_device(&dev);
     if (st != AC_OK) return st;
     cudaError_t e = launch_rope_kv_append(q_in, q_out, k_new, v_new, k_cache, v_cache, stride_page,
                                           stride_token, stride_head, block_table, max_pages_per_seq,
                                           context_lens, rope_cos, rope_sin, max_position, B, Hq, Hkv, d,
-                                          page_size, num_pages, status_flag,
+                                          page_size, num_pages, status_flag, vp,
                                           static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
+}
+
+int ac_rope_kv_append(const void* q_in, void* q_out, const void* k_new, const void* v_new,
+                      void* k_cache, void* v_cache, int64_t stride_page, int64_t stride_token,
+                      int64_t stride_head, const int32_t* block_table, int max_pages_per_seq,
+                      const int32_t* context_lens, const float* rope_cos, const float* rope_sin,
+                      int max_position, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                      int32_t* status_flag, void* stream) {
+    return ac_rope_kv_append_ex(q_in, q_out, k_new, v_new, k_cache, v_cache, stride_page, stride_token,
+                                stride_head, block_table, max_pages_per_seq, context_lens, rope_cos,
+                                rope_sin, max_position, B, Hq, Hkv, d, page_size, num_pages, status_flag,
+                                stream, nullptr);
 }
 
 static int attn_common(const void* q_rot, const void* k_cache, const void* v_cache, int64_t stride_page,

@@ -47,6 +47,15 @@ struct FusedRopeArgs {
     int max_position, num_pages;
 };
 
+// Prelude variants of the RoPE + append kernel (validated by the ABI layer).
+struct RopeVariant {
+    int rotary_dim;               // even, 2 .. d
+    int interleaved;              // 0: pair (i, i + rotary_dim/2); 1: pair (2i, 2i + 1)
+    const void* q_norm_weight;    // bf16 [d] or nullptr
+    const void* k_norm_weight;    // bf16 [d] or nullptr
+    float norm_eps;
+};
+
 // Per-kernel launchers; each validates nothing (the ABI layer did) and returns a cudaError_t.
 cudaError_t attn_set_attributes(int smem_optin);
 cudaError_t launch_rope_kv_append(const void* q_in, void* q_out, const void* k_new, const void* v_new,
@@ -56,7 +65,7 @@ cudaError_t launch_rope_kv_append(const void* q_in, void* q_out, const void* k_n
                                   const int32_t* context_lens, const float* rope_cos,
                                   const float* rope_sin, int max_position, int B, int Hq, int Hkv,
                                   int d, int page_size, int num_pages, int32_t* status_flag,
-                                  cudaStream_t stream);
+                                  const RopeVariant* variant, cudaStream_t stream);
 cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap& v_map,
                                      const void* q_rot,
                                      const int32_t* block_table, int max_pages_per_seq,

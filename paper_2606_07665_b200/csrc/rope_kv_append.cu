@@ -99,6 +99,125 @@ __global__ void __launch_bounds__(128) rope_kv_append_kernel(
     }
 }
 
+
+// Variants of the prelude (per-head RMSNorm of q/k before the rotation, partial rotary, interleaved
+// pairing): one warp per head vector.  The (optionally normalised) vector is parked in shared memory
+// so that every lane can read the partner of each of its elements, wherever the pairing puts it.
+//
+// RMSNorm arithmetic: sum of squares in fp64 (exact for bf16 inputs of moderate dynamic range),
+// r = 1 / sqrt(sum / d + eps) with correctly rounded fp64 sqrt and division, y = bf16(x * r), then
+// bf16(y * w): normalise, round to the model dtype, scale by the weight, round again.
+template <int D>
+__global__ void __launch_bounds__(128) rope_kv_append_ex_kernel(
+    const uint16_t* q_in, uint16_t* q_out, const uint16_t* __restrict__ k_new,
+    const uint16_t* __restrict__ v_new, uint16_t* __restrict__ k_cache, uint16_t* __restrict__ v_cache,
+    int64_t stride_page, int64_t stride_token, int64_t stride_head,
+    const int32_t* __restrict__ block_table, int max_pages_per_seq,
+    const int32_t* __restrict__ context_lens, const float* __restrict__ rope_cos,
+    const float* __restrict__ rope_sin, int max_position, int B, int Hq, int Hkv, int page_size,
+    int num_pages, int32_t* status_flag, int rotary_dim, int interleaved,
+    const uint16_t* __restrict__ q_norm_w, const uint16_t* __restrict__ k_norm_w, float norm_eps) {
+    cudaTriggerProgrammaticLaunchCompletion();
+    cudaGridDependencySynchronize();
+    constexpr int EPL = D / 32;                           // elements per lane: 4 (D=128) or 2 (D=64)
+    __shared__ uint16_t s_vec[4][D];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int heads = Hq + Hkv;
+    const long long vec = static_cast<long long>(blockIdx.x) * 4 + warp;
+    if (vec >= static_cast<long long>(B) * heads) return;
+    const int b = static_cast<int>(vec / heads);
+    const int hh = static_cast<int>(vec % heads);
+    const int p = context_lens[b];
+    if (p < 0) return;
+    const int page_idx = p / page_size;
+    if (p >= max_position || page_idx >= max_pages_per_seq) {
+        if (status_flag != nullptr && lane == 0) atomicOr(status_flag, AC_FLAG_POSITION_OOB);
+        return;
+    }
+    const bool is_q = hh < Hq;
+    const uint16_t* src;
+    uint16_t* dst;
+    const uint16_t* norm_w;
+    size_t cache_off = 0;
+    if (is_q) {
+        src = q_in + (static_cast<size_t>(b) * Hq + hh) * D;
+        dst = q_out + (static_cast<size_t>(b) * Hq + hh) * D;
+        norm_w = q_norm_w;
+    } else {
+        const int h = hh - Hq;
+        const int page = block_table[static_cast<size_t>(b) * max_pages_per_seq + page_idx];
+        if (page < 0 || page >= num_pages) {
+            if (status_flag != nullptr && lane == 0) atomicOr(status_flag, AC_FLAG_PAGE_OOB);
+            return;
+        }
+        cache_off = static_cast<size_t>(page) * stride_page +
+                    static_cast<size_t>(p - page_idx * page_size) * stride_token +
+                    static_cast<size_t>(h) * stride_head;
+        src = k_new + (static_cast<size_t>(b) * Hkv + h) * D;
+        dst = k_cache + cache_off;
+        norm_w = k_norm_w;
+    }
+
+    uint16_t x[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) x[e] = src[lane * EPL + e];
+    if (norm_w != nullptr) {
+        double ss = 0.0;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+            const double v = static_cast<double>(acdev::bf16_bits_to_float(x[e]));
+            ss = __dadd_rn(ss, __dmul_rn(v, v));
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) ss = __dadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, off));
+        const double r = __ddiv_rn(1.0, __dsqrt_rn(__dadd_rn(__ddiv_rn(ss, static_cast<double>(D)),
+                                                             static_cast<double>(norm_eps))));
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+            const double v = static_cast<double>(acdev::bf16_bits_to_float(x[e]));
+            const uint16_t y1 = acdev::f64_to_bf16_rne(__dmul_rn(v, r));
+            const double w = static_cast<double>(acdev::bf16_bits_to_float(norm_w[lane * EPL + e]));
+            x[e] = acdev::f64_to_bf16_rne(__dmul_rn(static_cast<double>(acdev::bf16_bits_to_float(y1)), w));
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) s_vec[warp][lane * EPL + e] = x[e];
+    __syncwarp();
+
+    const int half = rotary_dim / 2;
+    uint16_t out[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+        const int j = lane * EPL + e;
+        if (j >= rotary_dim) {
+            out[e] = x[e];
+            continue;
+        }
+        int i, partner;
+        bool first;
+        if (interleaved) {
+            i = j >> 1;
+            first = (j & 1) == 0;
+            partner = first ? j + 1 : j - 1;
+        } else {
+            first = j < half;
+            i = first ? j : j - half;
+            partner = first ? j + half : j - half;
+        }
+        const float c = rope_cos[static_cast<size_t>(p) * half + i];
+        const float sn = rope_sin[static_cast<size_t>(p) * half + i];
+        const uint16_t other = s_vec[warp][partner];
+        out[e] = first ? acdev::rope_first_half(x[e], other, c, sn) : acdev::rope_second_half(other, x[e], c, sn);
+    }
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) dst[lane * EPL + e] = out[e];
+    if (!is_q) {
+        const uint16_t* src_v = v_new + (static_cast<size_t>(b) * Hkv + (hh - Hq)) * D;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) v_cache[cache_off + lane * EPL + e] = src_v[lane * EPL + e];
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_rope_kv_append(const void* q_in, void* q_out, const void* k_new, const void* v_new,
@@ -108,7 +227,31 @@ cudaError_t launch_rope_kv_append(const void* q_in, void* q_out, const void* k_n
                                   const int32_t* context_lens, const float* rope_cos,
                                   const float* rope_sin, int max_position, int B, int Hq, int Hkv,
                                   int d, int page_size, int num_pages, int32_t* status_flag,
-                                  cudaStream_t stream) {
+                                  const RopeVariant* variant, cudaStream_t stream) {
+    if (variant != nullptr) {
+        cudaLaunchConfig_t cfg = {};
+        const long long vecs = static_cast<long long>(B) * (Hq + Hkv);
+        cfg.gridDim = dim3(static_cast<unsigned>((vecs + 3) / 4));
+        cfg.blockDim = dim3(128);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+#define AC_ROPE_EX_ARGS                                                                           \
+    static_cast<const uint16_t*>(q_in), static_cast<uint16_t*>(q_out),                             \
+        static_cast<const uint16_t*>(k_new), static_cast<const uint16_t*>(v_new),                  \
+        static_cast<uint16_t*>(k_cache), static_cast<uint16_t*>(v_cache), stride_page,             \
+        stride_token, stride_head, block_table, max_pages_per_seq, context_lens, rope_cos,         \
+        rope_sin, max_position, B, Hq, Hkv, page_size, num_pages, status_flag,                     \
+        variant->rotary_dim, variant->interleaved,                                                 \
+        static_cast<const uint16_t*>(variant->q_norm_weight),                                      \
+        static_cast<const uint16_t*>(variant->k_norm_weight), variant->norm_eps
+        if (d == 128) return cudaLaunchKernelEx(&cfg, rope_kv_append_ex_kernel<128>, AC_ROPE_EX_ARGS);
+        return cudaLaunchKernelEx(&cfg, rope_kv_append_ex_kernel<64>, AC_ROPE_EX_ARGS);
+#undef AC_ROPE_EX_ARGS
+    }
     const long long threads_per_vec = d / 16;
     const long long total = static_cast<long long>(B) * (Hq + Hkv) * threads_per_vec;
     const int block = 128;

@@ -87,6 +87,17 @@ class DecodeStep:
                                     self.d, self.num_splits)
 
     # -- the three calls -----------------------------------------------------------------------
+    def rope_kv_append_ex(self, stream=None, rotary_dim=0, interleaved=False, q_norm_weight=None,
+                          k_norm_weight=None, norm_eps=0.0) -> None:
+        """Prelude variants; norm weights are device int16 tensors holding bf16 bits."""
+        ac.ac_rope_kv_append_ex(self.q_in, self.q_rot, self.k_new, self.v_new, self.k_cache, self.v_cache,
+                                self.stride_page, self.stride_token, self.stride_head, self.block_table,
+                                self.w.max_pages_per_seq, self.context_lens, self.rope_cos, self.rope_sin,
+                                self.w.max_position, self.B, self.Hq, self.Hkv, self.d, self.ps,
+                                self.num_pages, self.status_flag, stream, rotary_dim=rotary_dim,
+                                interleaved=interleaved, q_norm_weight=q_norm_weight,
+                                k_norm_weight=k_norm_weight, norm_eps=norm_eps)
+
     def rope_kv_append(self, stream=None) -> None:
         ac.ac_rope_kv_append(self.q_in, self.q_rot, self.k_new, self.v_new, self.k_cache, self.v_cache,
                              self.stride_page, self.stride_token, self.stride_head, self.block_table,

@@ -114,6 +114,46 @@ def test_rope_constructed_near_tie(rt):
         assert (rt.bits_of(st.q_rot)[0, :, :32] == 0x3F82).all()
 
 
+@pytest.mark.parametrize("kw", [
+    dict(rotary_dim=64),                                       # partial rotary, half-split
+    dict(interleaved=True),
+    dict(rotary_dim=32, interleaved=True),
+    dict(norm=True),                                           # per-head Q/K RMSNorm, then full rotary
+    dict(norm=True, rotary_dim=64, interleaved=True),
+    dict(norm="q_only"),
+    dict(),                                                    # options present but plain
+])
+@pytest.mark.parametrize("d", [128, 64])
+def test_rope_prelude_variants_bit_exact_and_feed_attention(rt, kw, d):
+    import torch
+    kw = dict(kw)
+    norm = kw.pop("norm", False)
+    rotary_dim = min(kw.get("rotary_dim", 0), d)
+    interleaved = kw.get("interleaved", False)
+    w = small(37, B=4, Hq=12, Hkv=3, d=d, context_lens=[200, 0, 37, 333], num_pages=64, inactive_rows=(2,))
+    R = rotary_dim or d
+    w.rope_cos, w.rope_sin = W.rope_table(w.max_position, R, w.rope_base)      # [max_position, R/2]
+    rng = np.random.default_rng(3)
+    qw = W.f32_to_bf16_bits((1 + 0.2 * rng.standard_normal(d)).astype(np.float32)) if norm else None
+    kw_bits = W.f32_to_bf16_bits((1 + 0.2 * rng.standard_normal(d)).astype(np.float32)) if norm is True else None
+    q_rot, k_after, v_after = O.oracle_rope_kv_append_ex(
+        w.q, w.k_new, w.v_new, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.rope_cos, w.rope_sin,
+        w.page_size, rotary_dim=rotary_dim or None, interleaved=interleaved, q_norm_weight=qw,
+        k_norm_weight=kw_bits, norm_eps=1e-6)
+    out_ref = O.oracle_paged_decode_attn(q_rot, k_after, v_after, w.block_table, w.context_lens, w.page_size)
+    st = rt.DecodeStep(w, num_splits=2)
+    dev = lambda a: None if a is None else torch.from_numpy(a.view(np.int16)).cuda()
+    st.rope_kv_append_ex(rotary_dim=rotary_dim, interleaved=interleaved, q_norm_weight=dev(qw),
+                         k_norm_weight=dev(kw_bits), norm_eps=1e-6)
+    st.attention()
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) == 0
+    assert np.array_equal(rt.bits_of(st.q_rot), q_rot), "q after norm/rotation differs"
+    k_gpu, v_gpu = st.cache_bits()
+    assert np.array_equal(k_gpu, k_after) and np.array_equal(v_gpu, v_after)
+    check_out(st.out_f64(), out_ref, f"prelude variant {kw} norm={norm} d={d}")
+
+
 def test_append_flags_out_of_range_and_writes_nothing(rt):
     import torch
     w = small(34, B=2, context_lens=[40, 50], num_pages=32)

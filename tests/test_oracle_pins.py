@@ -484,6 +484,80 @@ def test_sliding_window_pins():
     assert np.array_equal(again[0], win[0])
 
 
+def test_rope_variants_reduce_to_the_plain_rotation():
+    rng = np.random.default_rng(31)
+    d = 16
+    x = W.f32_to_bf16_bits(rng.standard_normal((5, d)).astype(np.float32))
+    th = rng.uniform(-3, 3, d // 2)
+    c, s = np.cos(th).astype(np.float32), np.sin(th).astype(np.float32)
+    # full rotary dim, half-split: identical bits to the plain routine
+    assert np.array_equal(O.rope_rotate_variant_bf16(x, c, s), O.rope_rotate_bf16(x, c, s))
+    # interleaved == plain rotation of the de-interleaved vector, re-interleaved
+    deint = np.concatenate([x[:, 0::2], x[:, 1::2]], axis=-1)
+    plain = O.rope_rotate_bf16(deint, c, s)
+    want = np.empty_like(x)
+    want[:, 0::2] = plain[:, :d // 2]
+    want[:, 1::2] = plain[:, d // 2:]
+    assert np.array_equal(O.rope_rotate_variant_bf16(x, c, s, interleaved=True), want)
+    # partial rotary: tail untouched, head == plain rotation of the head slice with the first angles
+    R = 8
+    got = O.rope_rotate_variant_bf16(x, c, s, rotary_dim=R)
+    assert np.array_equal(got[:, R:], x[:, R:])
+    assert np.array_equal(got[:, :R], O.rope_rotate_bf16(x[:, :R], c[:R // 2], s[:R // 2]))
+    gi = O.rope_rotate_variant_bf16(x, c, s, rotary_dim=R, interleaved=True)
+    assert np.array_equal(gi[:, R:], x[:, R:])
+    # hand example, interleaved, d = 4: pairs (x0,x1) by 90 degrees, (x2,x3) by 0
+    hx = W.f32_to_bf16_bits(np.array([1.0, 2.0, 3.0, 4.0], np.float32))
+    hv = O.rope_rotate_variant_bf16(hx, np.array([0.0, 1.0], np.float32), np.array([1.0, 0.0], np.float32),
+                                    interleaved=True)
+    assert W.bf16_bits_to_f32(hv).tolist() == [-2.0, 1.0, 3.0, 4.0]
+
+
+def test_rms_norm_pins():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(32)
+    d = 64
+    x = W.f32_to_bf16_bits(rng.standard_normal((7, d)).astype(np.float32) * 3)
+    ones = np.full(d, 0x3F80, np.uint16)
+    w = W.f32_to_bf16_bits((1 + 0.1 * rng.standard_normal(d)).astype(np.float32))
+    # hand example: x = (3, 4), unit weight, eps = 0: rms = sqrt(12.5)
+    hx = W.f32_to_bf16_bits(np.array([3.0, 4.0], np.float32))
+    hy = O.rms_norm_bf16(hx, np.array([0x3F80, 0x3F80], np.uint16), 0.0)
+    assert hy.tolist() == O.f64_to_bf16_rne(np.array([3.0, 4.0]) / math.sqrt(12.5)).tolist()
+    # unit weight: the result is within one bf16 rounding of torch's fp64 rms_norm (library routine)
+    y = O.bf16_to_f64(O.rms_norm_bf16(x, ones, 1e-6))
+    ref = torch.nn.functional.rms_norm(torch.from_numpy(O.bf16_to_f64(x)), (d,), eps=float(np.float32(1e-6))).numpy()
+    assert np.abs(y - ref).max() <= 2.0 ** -8 * np.abs(ref).max()
+    assert np.array_equal(O.f64_to_bf16_rne(ref), O.rms_norm_bf16(x, ones, 1e-6))
+    # scaling the input by a power of two changes nothing when eps = 0
+    x4 = W.f32_to_bf16_bits(W.bf16_bits_to_f32(x) * np.float32(4.0))
+    assert np.array_equal(O.rms_norm_bf16(x4, w, 0.0), O.rms_norm_bf16(x, w, 0.0))
+    # the weight is applied after rounding the normalised value to bf16
+    y1 = O.rms_norm_bf16(x, ones, 1e-6)
+    want = O.f64_to_bf16_rne(O.bf16_to_f64(y1) * O.bf16_to_f64(w))
+    assert np.array_equal(O.rms_norm_bf16(x, w, 1e-6), want)
+    # mean of squares of the unit-weight output is ~1
+    assert np.allclose(np.mean(y ** 2, axis=-1), 1.0, atol=2e-3)
+
+
+def test_append_ex_defaults_equal_plain_append_and_norm_feeds_rotation():
+    w = tiny_case(seed=33, Hq=4, Hkv=2, d=8, lens=(9, 3))
+    plain = O.oracle_rope_kv_append(w.q, w.k_new, w.v_new, w.k_cache, w.v_cache, w.block_table,
+                                    w.context_lens, w.rope_cos, w.rope_sin, w.page_size)
+    ex = O.oracle_rope_kv_append_ex(w.q, w.k_new, w.v_new, w.k_cache, w.v_cache, w.block_table,
+                                    w.context_lens, w.rope_cos, w.rope_sin, w.page_size)
+    for a, b in zip(plain, ex):
+        assert np.array_equal(a, b)
+    wt = W.f32_to_bf16_bits(np.linspace(0.5, 1.5, 8).astype(np.float32))
+    q_rot, k_after, v_after = O.oracle_rope_kv_append_ex(
+        w.q, w.k_new, w.v_new, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.rope_cos,
+        w.rope_sin, w.page_size, q_norm_weight=wt, k_norm_weight=wt, norm_eps=1e-6)
+    p = int(w.context_lens[0])
+    want_q = O.rope_rotate_bf16(O.rms_norm_bf16(w.q[0], wt, 1e-6), w.rope_cos[p], w.rope_sin[p])
+    assert np.array_equal(q_rot[0], want_q)
+    assert np.array_equal(v_after, plain[2])          # v is never normalised
+
+
 def test_tiny_workload_oracle_result_is_frozen():
     import importlib.util
     import os
