@@ -197,6 +197,25 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------------------
+# replicas: the path has no exchange step, so N GPUs run N independent copies of the workload
+# ---------------------------------------------------------------------------------------------
+
+def max_over_ranks(values, world, device="cpu"):
+    """Element-wise maximum of per-rank timings (every rank gets the result)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def aggregate_throughput(kv_bytes_per_rank, ms_slowest_rank, world):
+    """Whole-job GB/s: every rank moves kv_bytes_per_rank per step; the step ends with the slowest."""
+    return world * kv_bytes_per_rank / (ms_slowest_rank * 1e-3) / 1e9
+
+
+# ---------------------------------------------------------------------------------------------
 # GPU arm
 # ---------------------------------------------------------------------------------------------
 
@@ -353,7 +372,8 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
 
     w = W.NAMED[args.workload]()
-    st = runner.DecodeStep(w, device=device, fused_step=not args.three_launches)
+    st = runner.DecodeStep(w, device=device, fused_step=not args.three_launches,
+                           fused_merge=not args.separate_merge)
 
     def barrier():
         if world > 1:
@@ -372,15 +392,12 @@ def run_ours(args):
     flag = int(st.status_flag.item())
     launches_per_step = st.launches_per_step
 
-    t = torch.tensor([ms_step, ms_attn, ms_e2e], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step, ms_attn, ms_e2e = t.tolist()
+    ms_step, ms_attn, ms_e2e = max_over_ranks([ms_step, ms_attn, ms_e2e], world, device)
 
     if rank == 0:
         kv = w.kv_bytes
-        value = world * kv / (ms_step * 1e-3) / 1e9
-        e2e_value = world * kv / (ms_e2e * 1e-3) / 1e9
+        value = aggregate_throughput(kv, ms_step, world)
+        e2e_value = aggregate_throughput(kv, ms_e2e, world)
         attn_gbs = kv / (ms_attn * 1e-3) / 1e9
         others = []
         if not args.only_headline:
@@ -454,6 +471,9 @@ def main():
     ap.add_argument("--three-launches", action="store_true",
                     help="time ac_rope_kv_append + ac_paged_decode_attn_fused_merge instead of the "
                          "single-launch ac_decode_step_fused")
+    ap.add_argument("--separate-merge", action="store_true",
+                    help="with --three-launches: use ac_paged_decode_attn + ac_splitkv_merge (three "
+                         "kernels) instead of the merge fused into the attention kernel")
     ap.add_argument("--only-headline", action="store_true",
                     help="skip the other workloads and the CPU baseline")
     args = ap.parse_args()
