@@ -207,6 +207,36 @@ def oracle_rope_kv_append_ex(q, k_new, v_new, k_cache, v_cache, block_table, con
 
 
 # --------------------------------------------------------------------------------------------
+# Attention-prelude fusion (kernel family (i)): QKV projection feeding A1/A2
+# --------------------------------------------------------------------------------------------
+
+
+def oracle_qkv_projection(x_bits, w_qkv_bits, Hq, Hkv, d):
+    """x [B,H] bf16, W_qkv [(Hq+2Hkv)*d, H] bf16 ([N,K] layout: one output feature per row, rows
+    ordered q heads, k heads, v heads).  y = x W^T in fp64, rounded once to bf16.
+
+    Returns (q [B,Hq,d], k_new [B,Hkv,d], v_new [B,Hkv,d]) as bf16 bits.  (The paper's family (i)
+    fuses "QKV projection + RoPE"; its template GEMV stores weights [N,K]; no bias is mentioned.)
+    """
+    x = bf16_to_f64(x_bits)
+    w = bf16_to_f64(w_qkv_bits)
+    y = f64_to_bf16_rne(x @ w.T)
+    B = x.shape[0]
+    q = y[:, :Hq * d].reshape(B, Hq, d)
+    k = y[:, Hq * d:(Hq + Hkv) * d].reshape(B, Hkv, d)
+    v = y[:, (Hq + Hkv) * d:].reshape(B, Hkv, d)
+    return q, k, v
+
+
+def oracle_qkv_rope_kv_append(x_bits, w_qkv_bits, k_cache, v_cache, block_table, context_lens,
+                              rope_cos, rope_sin, page_size, Hq, Hkv, d):
+    """Projection, then the plain A1 + A2 on its bf16 results.  Returns (q_rot, k_cache, v_cache)."""
+    q, k_new, v_new = oracle_qkv_projection(x_bits, w_qkv_bits, Hq, Hkv, d)
+    return oracle_rope_kv_append(q, k_new, v_new, k_cache, v_cache, block_table, context_lens,
+                                 rope_cos, rope_sin, page_size)
+
+
+# --------------------------------------------------------------------------------------------
 # A4 + A5 as one definition: softmax(q K^T * scale) V per query head over the gathered pages
 # --------------------------------------------------------------------------------------------
 

@@ -558,6 +558,38 @@ def test_append_ex_defaults_equal_plain_append_and_norm_feeds_rotation():
     assert np.array_equal(v_after, plain[2])          # v is never normalised
 
 
+def test_qkv_projection_pins():
+    rng = np.random.default_rng(41)
+    Hq, Hkv, d, H, B = 4, 2, 8, 24, 3
+    N = (Hq + 2 * Hkv) * d
+    x = W.f32_to_bf16_bits(rng.standard_normal((B, H)).astype(np.float32))
+    wq = W.f32_to_bf16_bits((rng.standard_normal((N, H)) / np.sqrt(H)).astype(np.float32))
+    q, k, v = O.oracle_qkv_projection(x, wq, Hq, Hkv, d)
+    assert q.shape == (B, Hq, d) and k.shape == (B, Hkv, d) and v.shape == (B, Hkv, d)
+    # brute force with exact rationals: feature n of row b is sum_j x[b,j] * W[n,j], rounded once
+    for b, n in ((0, 0), (1, Hq * d + 3), (2, N - 1), (1, 17)):
+        acc = sum(bf16_value(int(x[b, j])) * bf16_value(int(wq[n, j])) for j in range(H))
+        want = fraction_to_bf16(acc)
+        flat = np.concatenate([q[b].ravel(), k[b].ravel(), v[b].ravel()])
+        assert int(flat[n]) == want
+    # selection weights: row n of W is a unit vector -> feature n copies an input element exactly
+    sel = np.zeros((N, H), np.uint16)
+    for n in range(N):
+        sel[n, n % H] = 0x3F80
+    q2, k2, v2 = O.oracle_qkv_projection(x, sel, Hq, Hkv, d)
+    flat = np.concatenate([q2.reshape(B, -1), k2.reshape(B, -1), v2.reshape(B, -1)], axis=1)
+    assert np.array_equal(flat, x[:, np.arange(N) % H])
+    # the fused routine is the projection followed by the plain rotation + append
+    w = tiny_case(seed=42, Hq=Hq, Hkv=Hkv, d=d, lens=(9, 3, 0), B=3)
+    q_rot, k_after, v_after = O.oracle_qkv_rope_kv_append(x, wq, w.k_cache, w.v_cache, w.block_table,
+                                                          w.context_lens, w.rope_cos, w.rope_sin,
+                                                          w.page_size, Hq, Hkv, d)
+    ref = O.oracle_rope_kv_append(q, k, v, w.k_cache, w.v_cache, w.block_table, w.context_lens,
+                                  w.rope_cos, w.rope_sin, w.page_size)
+    for a, bb in zip((q_rot, k_after, v_after), ref):
+        assert np.array_equal(a, bb)
+
+
 def test_tiny_workload_oracle_result_is_frozen():
     import importlib.util
     import os
