@@ -152,6 +152,27 @@ int ac_rope_kv_append_ex(const void* q_in, void* q_out, const void* k_new, const
                          int B, int Hq, int Hkv, int d, int page_size, int num_pages,
                          int32_t* status_flag, void* stream, const ac_rope_options* options);
 
+/* Attention-prelude fusion, the paper's kernel family (i) ("QKV projection + RoPE"), with the KV
+ * append of the kv_append kernel folded in: one launch computes
+ *   y[b, n] = sum_k x[b, k] * w_qkv[n, k]     (bf16 operands, fp32 accumulation, rounded to bf16)
+ * for n over the (Hq + 2 Hkv) * d output features (rows of w_qkv ordered q heads, k heads, v heads,
+ * d rows per head; the [N, K] layout of the paper's decode GEMV), rotates the q and k features at
+ * position context_lens[b] exactly as ac_rope_kv_append does, writes q to q_out [B,Hq,d] and k, v
+ * into the cache slot block_table[b, p / page_size], p % page_size.  x is [B, H] bf16, H % 64 == 0.
+ * The projection is not bit-reproducible against an fp64 evaluation (fp32 accumulation order): its
+ * bf16 results can differ from the correctly rounded ones by one unit in the last place; the
+ * rotation and the stores are exact given those results.  Errors and status bits as
+ * ac_rope_kv_append.  The kernel streams w_qkv once from HBM for up to 32 batch rows (once per 32
+ * rows beyond that). */
+int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out,
+                          void* k_cache, void* v_cache,
+                          int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                          const int32_t* block_table, int max_pages_per_seq,
+                          const int32_t* context_lens,
+                          const float* rope_cos, const float* rope_sin, int max_position,
+                          int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                          int32_t* status_flag, void* stream);
+
 /* A4: paged decode attention, family (iv).  Row b attends over tokens 0 .. n_b - 1 with
  * n_b = context_lens[b] + new_tokens (new_tokens = 1 right after ac_rope_kv_append, 0 to attend
  * over the cached tokens only); token t lives in page block_table[b, t / page_size], slot

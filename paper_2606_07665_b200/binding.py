@@ -26,7 +26,7 @@ EXPORTS = ("ac_init", "ac_status_string", "ac_last_cuda_error", "ac_sm_count", "
            "ac_splitkv_merge", "ac_decode_step_host", "ac_paged_decode_attn_static_scratch",
            "ac_fused_workspace_bytes", "ac_fused_workspace_reset", "ac_paged_decode_attn_fused_merge",
            "ac_decode_step_fused", "ac_paged_decode_attn_ex", "ac_decode_step_fused_ex",
-           "ac_rope_kv_append_ex")
+           "ac_rope_kv_append_ex", "ac_qkv_rope_kv_append")
 AC_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -80,6 +80,10 @@ def lib():
         L.ac_rope_kv_append.restype = c_int
         L.ac_rope_kv_append_ex.argtypes = L.ac_rope_kv_append.argtypes + [POINTER(AcRopeOptions)]
         L.ac_rope_kv_append_ex.restype = c_int
+        L.ac_qkv_rope_kv_append.argtypes = ([c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p] +
+                                            [c_int64] * 3 + [c_void_p, c_int, c_void_p, c_void_p, c_void_p,
+                                            c_int] + [c_int] * 6 + [c_void_p, c_void_p])
+        L.ac_qkv_rope_kv_append.restype = c_int
         L.ac_paged_decode_attn.argtypes = ([c_void_p] * 3 + [c_int64] * 3 + [c_void_p, c_int, c_void_p,
                                            c_int, c_float, c_int, c_void_p, c_size_t, c_void_p] +
                                            [c_int] * 7 + [c_void_p, c_void_p])
@@ -188,6 +192,16 @@ def ac_rope_kv_append_ex(q_in, q_out, k_new, v_new, k_cache, v_cache, stride_pag
                                       ctypes.byref(opt)), "ac_rope_kv_append_ex")
 
 
+def ac_qkv_rope_kv_append(x, w_qkv, H, q_out, k_cache, v_cache, stride_page, stride_token, stride_head,
+                          block_table, max_pages_per_seq, context_lens, rope_cos, rope_sin, max_position,
+                          B, Hq, Hkv, d, page_size, num_pages, status_flag=None, stream=None):
+    _check(lib().ac_qkv_rope_kv_append(_ptr(x), _ptr(w_qkv), H, _ptr(q_out), _ptr(k_cache), _ptr(v_cache),
+                                       stride_page, stride_token, stride_head, _ptr(block_table),
+                                       max_pages_per_seq, _ptr(context_lens), _ptr(rope_cos),
+                                       _ptr(rope_sin), max_position, B, Hq, Hkv, d, page_size, num_pages,
+                                       _ptr(status_flag), _stream(stream)), "ac_qkv_rope_kv_append")
+
+
 def ac_paged_decode_attn(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
                          max_pages_per_seq, context_lens, new_tokens, softmax_scale, num_splits,
                          workspace, workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages,
@@ -231,7 +245,7 @@ def ac_decode_step_fused(q_in, q_rot_out, k_new, v_new, k_cache, v_cache, stride
         _ptr(rope_cos), _ptr(rope_sin), max_position, softmax_scale, num_splits, _ptr(workspace),
         workspace_bytes, _ptr(out), B, Hq, Hkv, d, page_size, num_pages, max_context_len,
         _ptr(status_flag), _stream(stream)), "ac_decode_step_fused", "ac_paged_decode_attn_ex", "ac_decode_step_fused_ex",
-           "ac_rope_kv_append_ex")
+           "ac_rope_kv_append_ex", "ac_qkv_rope_kv_append")
 
 
 def _options(window: int = 0, fused_merge: bool = False):

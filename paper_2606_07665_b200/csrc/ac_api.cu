@@ -133,6 +133,7 @@ int ac_init(int device) {
             g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
         }
         e = attn_set_attributes(st.smem_optin);
+        if (e == cudaSuccess) e = qkv_set_attributes(st.smem_optin);
         if (e != cudaSuccess) {
             status = fail_cuda(static_cast<int>(e));
             break;
@@ -288,6 +289,64 @@ int ac_rope_kv_append(const void* q_in, void* q_out, const void* k_new, const vo
                                 stride_head, block_table, max_pages_per_seq, context_lens, rope_cos,
                                 rope_sin, max_position, B, Hq, Hkv, d, page_size, num_pages, status_flag,
                                 stream, nullptr);
+}
+
+int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out, void* k_cache,
+                          void* v_cache, int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                          const int32_t* block_table, int max_pages_per_seq,
+                          const int32_t* context_lens, const float* rope_cos, const float* rope_sin,
+                          int max_position, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                          int32_t* status_flag, void* stream) {
+    if (!x || !w_qkv || !q_out || !k_cache || !v_cache || !block_table || !context_lens || !rope_cos ||
+        !rope_sin)
+        return AC_ERR_NULL;
+    Shape s{B, Hq, Hkv, d, page_size, num_pages};
+    int st = check_shape(s);
+    if (st != AC_OK) return st;
+    if (H <= 0 || max_pages_per_seq <= 0 || max_position <= 0) return AC_ERR_SHAPE;
+    if (H % 64 != 0) return AC_ERR_UNSUPPORTED;
+    st = check_strides(s, stride_page, stride_token, stride_head);
+    if (st != AC_OK) return st;
+    if (!aligned16(x) || !aligned16(w_qkv) || !aligned16(q_out) || !aligned16(k_cache) ||
+        !aligned16(v_cache))
+        return AC_ERR_ALIGN;
+    int dev;
+    st = current_ready_device(&dev);
+    if (st != AC_OK) return st;
+
+    // W [(Hq+2Hkv)*d, H] as (64 elements, row inside a half head, half, head, 64-element K block);
+    // x [B, H] as (64 elements, batch row, 64-element K block).
+    const cuuint64_t row_bytes = static_cast<cuuint64_t>(H) * 2;
+    CUtensorMap w_map, x_map;
+    {
+        cuuint64_t dims[5] = {64, static_cast<cuuint64_t>(d / 2), 2, static_cast<cuuint64_t>(Hq + 2 * Hkv),
+                              static_cast<cuuint64_t>(H / 64)};
+        cuuint64_t strides[4] = {row_bytes, row_bytes * (d / 2), row_bytes * d, 128};
+        cuuint32_t box[5] = {64, 16, 2, 1, 4};
+        cuuint32_t es[5] = {1, 1, 1, 1, 1};
+        CUresult r = g_encode_tiled(&w_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(w_qkv),
+                                    dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
+    }
+    {
+        cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(B), static_cast<cuuint64_t>(H / 64)};
+        cuuint64_t strides[2] = {row_bytes, 128};
+        cuuint32_t box[3] = {64, static_cast<cuuint32_t>(qkv_batch_tile(B)), 4};
+        cuuint32_t es[3] = {1, 1, 1};
+        CUresult r = g_encode_tiled(&x_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims,
+                                    strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
+    }
+    cudaError_t e = launch_qkv_rope_kv_append(w_map, x_map, q_out, k_cache, v_cache, stride_page,
+                                              stride_token, stride_head, block_table, max_pages_per_seq,
+                                              context_lens, rope_cos, rope_sin, max_position, B, H, Hq,
+                                              Hkv, d, page_size, num_pages, status_flag,
+                                              static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
 }
 
 static int attn_common(const void* q_rot, const void* k_cache, const void* v_cache, int64_t stride_page,

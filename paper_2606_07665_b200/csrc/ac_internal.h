@@ -74,6 +74,16 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
                                      float* partial_lse, int32_t* arrivals, void* out, int B, int Hq,
                                      int Hkv, int d, int page_size, int32_t* status_flag,
                                      const FusedRopeArgs* rope, int window, cudaStream_t stream);
+cudaError_t qkv_set_attributes(int smem_optin);
+int qkv_batch_tile(int B);
+cudaError_t launch_qkv_rope_kv_append(const CUtensorMap& w_map, const CUtensorMap& x_map, void* q_out,
+                                      void* k_cache, void* v_cache, int64_t stride_page,
+                                      int64_t stride_token, int64_t stride_head,
+                                      const int32_t* block_table, int max_pages_per_seq,
+                                      const int32_t* context_lens, const float* rope_cos,
+                                      const float* rope_sin, int max_position, int B, int H, int Hq,
+                                      int Hkv, int d, int page_size, int num_pages, int32_t* status_flag,
+                                      cudaStream_t stream);
 cudaError_t launch_splitkv_merge(const float* partial_o, const float* partial_lse, int num_splits,
                                  const int32_t* context_lens, void* out, int B, int Hq, int d,
                                  cudaStream_t stream);

@@ -1,0 +1,318 @@
+// Attention-prelude fusion: QKV projection (weight-streaming thin GEMM) + RoPE + KV append.
+//
+// y[b, n] = sum_k x[b, k] * W[n, k]  (x [B,H] bf16, W [(Hq+2Hkv)*d, H] bf16 in [N,K] layout, fp32
+// accumulation), rounded to bf16; q and k features are then rotated at position context_lens[b] with
+// the same exact-then-round arithmetic as the stand-alone RoPE kernel, q goes to q_out, k and v to
+// the request's cache slot.  Nothing but the final results touches global memory.
+//
+// The kernel is bound by streaming W once from HBM.  One CTA owns 16 rotary pairs of one head: W rows
+// i .. i+15 and i+d/2 .. i+d/2+15 (32 rows), all of K, one tile of up to 32 batch rows; the grid is
+// (d/32, Hq+2Hkv, ceil(B/32)) -- 192 CTAs for a 32/8-head, d=128 layer.  A producer warp issues, per
+// 256-wide K chunk, ONE 5-D tensor-map load for the 32 x 256 weight tile (the two row blocks and the
+// four 64-element K blocks are box dimensions, so the 16 KB land as eight swizzled [16 x 128 B]
+// blocks) and one 3-D load for the x tile, into a ring of stages guarded by full/empty mbarriers.
+// Eight consumer warps split each chunk's sixteen k-steps; A fragments (W) and B fragments (x) come
+// from shared memory by ldmatrix, products run on the bf16 m16n8k16 MMA (any batch size costs the
+// same weight traffic).  At the end the warps' partial sums are reduced through shared memory and
+// the epilogue rounds, rotates and scatters.
+#include <math.h>
+
+#include "ac_device.cuh"
+#include "ac_internal.h"
+
+namespace ac {
+namespace {
+
+using namespace acdev;
+
+constexpr int QKV_WARPS = 8;                          // consumer warps; warp QKV_WARPS produces
+constexpr int QKV_THREADS = (QKV_WARPS + 1) * 32;
+constexpr int KC = 256;                               // K elements per stage
+constexpr int KBLOCKS = KC / 64;                      // 128-byte column blocks per stage
+constexpr int W_BLOCK_BYTES = 16 * 128;               // one swizzled [16 rows x 64 elements] block
+constexpr int W_STAGE_BYTES = KBLOCKS * 2 * W_BLOCK_BYTES;     // 16 KB: [kblock][half][row][64]
+
+template <int BT>
+struct QkvSmem {
+    static constexpr int X_BLOCK_BYTES = BT * 128;                 // [BT batch rows x 64 elements]
+    static constexpr int X_STAGE_BYTES = KBLOCKS * X_BLOCK_BYTES;
+    static constexpr int STAGE_BYTES = W_STAGE_BYTES + X_STAGE_BYTES;
+    static constexpr int STAGES = BT <= 8 ? 5 : (BT <= 16 ? 4 : 3);
+    static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+    static constexpr int TOTAL = BAR_OFFSET + 2 * STAGES * 8 + 1024;
+    static_assert(QKV_WARPS * 32 * BT * 4 <= STAGES * STAGE_BYTES, "reduction buffer must fit");
+};
+
+struct QkvParams {
+    uint16_t* q_out;              // [B, Hq, d] rotated
+    uint16_t* k_cache;
+    uint16_t* v_cache;
+    int64_t stride_page, stride_token, stride_head;
+    const int32_t* block_table;
+    const int32_t* context_lens;
+    const float* rope_cos;
+    const float* rope_sin;
+    int32_t* status_flag;
+    int max_pages_per_seq, max_position, num_pages, page_size;
+    int B, H, Hq, Hkv, d;
+};
+
+template <int BT>
+__global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
+    const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map,
+    const QkvParams p) {
+    using L = QkvSmem<BT>;
+    constexpr int STAGES = L::STAGES;
+    constexpr int NT = BT / 8;                        // 8-wide batch tiles of the MMA
+
+    cudaTriggerProgrammaticLaunchCompletion();
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_addr(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_addr(smem_raw));
+    const uint32_t full_bar = smem_base + L::BAR_OFFSET;
+    const uint32_t empty_bar = full_bar + STAGES * 8;
+
+    const int blk = blockIdx.x;                       // block of 16 rotary pairs inside the head
+    const int hh = blockIdx.y;                        // head slot: q heads, then k heads, then v heads
+    const int b0 = blockIdx.z * BT;                   // first batch row of this tile
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int n_chunks = (p.H + KC - 1) / KC;
+
+    if (threadIdx.x == 0) {
+        tma_prefetch_descriptor(&w_map);
+        tma_prefetch_descriptor(&x_map);
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar + s * 8, 1);
+            mbar_init(empty_bar + s * 8, QKV_WARPS);
+        }
+        mbar_init_fence();
+    }
+    __syncthreads();
+    // x is produced by the kernel before this one; W and the tables are not.
+    cudaGridDependencySynchronize();
+
+    bool timed_out = false;
+    float acc[2][NT][4];
+#pragma unroll
+    for (int rb = 0; rb < 2; ++rb)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[rb][nt][e] = 0.0f;
+
+    if (warp == QKV_WARPS) {
+        // ---- producer: one thread streams the K chunks through the ring ----------------------------
+        if (lane == 0) {
+            const uint64_t stream_once = l2_policy_evict_first();
+            const uint64_t keep = l2_policy_evict_last();
+            for (int c = 0; c < n_chunks; ++c) {
+                const int stage = c % STAGES;
+                if (c >= STAGES && !mbar_wait_bounded(empty_bar + stage * 8, ((c / STAGES) - 1) & 1)) {
+                    timed_out = true;
+                    break;
+                }
+                const uint32_t dst = smem_base + stage * L::STAGE_BYTES;
+                mbar_arrive_expect_tx(full_bar + stage * 8, L::STAGE_BYTES);
+                tma_load_5d(dst, &w_map, full_bar + stage * 8, 0, 16 * blk, 0, hh, c * KBLOCKS, stream_once);
+                tma_load_3d(dst + W_STAGE_BYTES, &x_map, full_bar + stage * 8, 0, b0, c * KBLOCKS, keep);
+            }
+        }
+    } else {
+        // ---- consumers: warp w takes k-steps 2w and 2w+1 of every chunk ------------------------------
+        const int mi = lane >> 3, r8 = lane & 7;
+        const uint32_t a_row_off = ((mi & 1) * 8 + r8) * 128;    // A: matrices 0,2 rows 0-7; 1,3 rows 8-15
+        const int a_chunk = mi >> 1;                              //    matrices 0,1 k lo; 2,3 k hi
+        const uint32_t b_row_off = ((mi >> 1) * 8 + r8) * 128;   // B: matrices 0,1 batch 0-7; 2,3 batch 8-15
+        const int b_chunk = mi & 1;                               //    matrices 0,2 k lo; 1,3 k hi
+        for (int c = 0; c < n_chunks; ++c) {
+            const int stage = c % STAGES;
+            if (!mbar_wait_bounded(full_bar + stage * 8, (c / STAGES) & 1)) {
+                timed_out = true;
+                break;
+            }
+            const uint32_t wbase = smem_base + stage * L::STAGE_BYTES;
+            const uint32_t xbase = wbase + W_STAGE_BYTES;
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int ks = 2 * warp + u;                      // k-step (16 elements) inside the chunk
+                const int kb = ks >> 2;                           // 64-element block
+                const int ch = (ks & 3) * 2;                      // first 16-byte chunk of the k-step
+                uint32_t a[2][4];
+#pragma unroll
+                for (int rb = 0; rb < 2; ++rb) {
+                    const uint32_t addr = wbase + (kb * 2 + rb) * W_BLOCK_BYTES + a_row_off +
+                                          (((ch + a_chunk) ^ r8) << 4);
+                    ldmatrix_x4(a[rb][0], a[rb][1], a[rb][2], a[rb][3], addr);
+                }
+                if (NT == 1) {
+                    // eight batch rows: two 8x8 matrices (k lo, k hi); lanes 16-31 repeat valid addresses
+                    const uint32_t addr = xbase + kb * L::X_BLOCK_BYTES + r8 * 128 + (((ch + b_chunk) ^ r8) << 4);
+                    uint32_t bq0, bq1, bq2, bq3;
+                    ldmatrix_x4(bq0, bq1, bq2, bq3, addr);
+                    (void)bq2;
+                    (void)bq3;
+#pragma unroll
+                    for (int rb = 0; rb < 2; ++rb)
+                        mma_bf16_16816(acc[rb][0][0], acc[rb][0][1], acc[rb][0][2], acc[rb][0][3], a[rb][0],
+                                       a[rb][1], a[rb][2], a[rb][3], bq0, bq1);
+                } else {
+#pragma unroll
+                    for (int np = 0; np < NT / 2; ++np) {
+                        const uint32_t addr = xbase + kb * L::X_BLOCK_BYTES + np * 16 * 128 + b_row_off +
+                                              (((ch + b_chunk) ^ r8) << 4);
+                        uint32_t bq0, bq1, bq2, bq3;
+                        ldmatrix_x4(bq0, bq1, bq2, bq3, addr);
+#pragma unroll
+                        for (int rb = 0; rb < 2; ++rb) {
+                            mma_bf16_16816(acc[rb][2 * np][0], acc[rb][2 * np][1], acc[rb][2 * np][2],
+                                           acc[rb][2 * np][3], a[rb][0], a[rb][1], a[rb][2], a[rb][3], bq0, bq1);
+                            mma_bf16_16816(acc[rb][2 * np + 1][0], acc[rb][2 * np + 1][1], acc[rb][2 * np + 1][2],
+                                           acc[rb][2 * np + 1][3], a[rb][0], a[rb][1], a[rb][2], a[rb][3], bq2, bq3);
+                        }
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_bar + stage * 8);
+        }
+    }
+    if (timed_out && lane == 0 && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_WAIT_TIMEOUT);
+
+    // ---- reduce the warps' partial sums through shared memory ----------------------------------------
+    __syncthreads();                                   // every load has landed and been consumed
+    float* red = reinterpret_cast<float*>(smem_gen);   // [QKV_WARPS][32 rows][BT]
+    if (warp < QKV_WARPS) {
+        const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+        for (int rb = 0; rb < 2; ++rb)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                float* base = red + (warp * 32 + rb * 16) * BT + nt * 8 + 2 * t;
+                *reinterpret_cast<float2*>(base + g * BT) = make_float2(acc[rb][nt][0], acc[rb][nt][1]);
+                *reinterpret_cast<float2*>(base + (g + 8) * BT) = make_float2(acc[rb][nt][2], acc[rb][nt][3]);
+            }
+    }
+    __syncthreads();
+
+    // ---- epilogue: round, rotate, scatter --------------------------------------------------------
+    const int d = p.d, half = d / 2;
+    for (int item = threadIdx.x; item < 16 * BT; item += QKV_THREADS) {
+        const int j = item / BT;                       // pair inside the block
+        const int n = item - j * BT;
+        const int b = b0 + n;
+        if (b >= p.B) continue;
+        const int ctx = p.context_lens[b];
+        if (ctx < 0) continue;                         // inactive row
+        float y_lo = 0.0f, y_hi = 0.0f;
+#pragma unroll
+        for (int w = 0; w < QKV_WARPS; ++w) {
+            y_lo += red[(w * 32 + j) * BT + n];
+            y_hi += red[(w * 32 + 16 + j) * BT + n];
+        }
+        const uint32_t packed = pack_bf16x2(y_lo, y_hi);
+        uint16_t lo = static_cast<uint16_t>(packed & 0xFFFFu), hi = static_cast<uint16_t>(packed >> 16);
+        const int i = 16 * blk + j;                    // pair index inside the head
+        const int page_idx = ctx / p.page_size;
+        if (ctx >= p.max_position || page_idx >= p.max_pages_per_seq) {
+            if (p.status_flag != nullptr && j == 0 && blk == 0) atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
+            continue;
+        }
+        if (hh < p.Hq + p.Hkv) {                       // q and k features are rotated
+            const float c = p.rope_cos[static_cast<size_t>(ctx) * half + i];
+            const float sn = p.rope_sin[static_cast<size_t>(ctx) * half + i];
+            const uint16_t r0 = rope_first_half(lo, hi, c, sn);
+            const uint16_t r1 = rope_second_half(lo, hi, c, sn);
+            lo = r0;
+            hi = r1;
+        }
+        if (hh < p.Hq) {
+            uint16_t* dst = p.q_out + (static_cast<size_t>(b) * p.Hq + hh) * d;
+            dst[i] = lo;
+            dst[i + half] = hi;
+        } else {
+            const int page = p.block_table[static_cast<size_t>(b) * p.max_pages_per_seq + page_idx];
+            if (page < 0 || page >= p.num_pages) {
+                if (p.status_flag != nullptr && j == 0 && blk == 0) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
+                continue;
+            }
+            const bool is_k = hh < p.Hq + p.Hkv;
+            const int h = is_k ? hh - p.Hq : hh - p.Hq - p.Hkv;
+            uint16_t* dst = (is_k ? p.k_cache : p.v_cache) + static_cast<size_t>(page) * p.stride_page +
+                            static_cast<size_t>(ctx - page_idx * p.page_size) * p.stride_token +
+                            static_cast<size_t>(h) * p.stride_head;
+            dst[i] = lo;
+            dst[i + half] = hi;
+        }
+    }
+}
+
+template <int BT>
+cudaError_t launch_qkv(const CUtensorMap& w_map, const CUtensorMap& x_map, const QkvParams& p,
+                       cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.d / 32, p.Hq + 2 * p.Hkv, (p.B + BT - 1) / BT);
+    cfg.blockDim = dim3(QKV_THREADS);
+    cfg.dynamicSmemBytes = QkvSmem<BT>::TOTAL;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, qkv_rope_append_kernel<BT>, w_map, x_map, p);
+}
+
+}  // namespace
+
+cudaError_t qkv_set_attributes(int smem_optin) {
+    if (QkvSmem<32>::TOTAL > smem_optin) return cudaErrorInvalidConfiguration;
+    cudaError_t e;
+    e = cudaFuncSetAttribute(qkv_rope_append_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             QkvSmem<8>::TOTAL);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(qkv_rope_append_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             QkvSmem<16>::TOTAL);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(qkv_rope_append_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                QkvSmem<32>::TOTAL);
+}
+
+int qkv_batch_tile(int B) { return B <= 8 ? 8 : (B <= 16 ? 16 : 32); }
+
+cudaError_t launch_qkv_rope_kv_append(const CUtensorMap& w_map, const CUtensorMap& x_map, void* q_out,
+                                      void* k_cache, void* v_cache, int64_t stride_page,
+                                      int64_t stride_token, int64_t stride_head,
+                                      const int32_t* block_table, int max_pages_per_seq,
+                                      const int32_t* context_lens, const float* rope_cos,
+                                      const float* rope_sin, int max_position, int B, int H, int Hq,
+                                      int Hkv, int d, int page_size, int num_pages, int32_t* status_flag,
+                                      cudaStream_t stream) {
+    QkvParams p;
+    p.q_out = static_cast<uint16_t*>(q_out);
+    p.k_cache = static_cast<uint16_t*>(k_cache);
+    p.v_cache = static_cast<uint16_t*>(v_cache);
+    p.stride_page = stride_page;
+    p.stride_token = stride_token;
+    p.stride_head = stride_head;
+    p.block_table = block_table;
+    p.context_lens = context_lens;
+    p.rope_cos = rope_cos;
+    p.rope_sin = rope_sin;
+    p.status_flag = status_flag;
+    p.max_pages_per_seq = max_pages_per_seq;
+    p.max_position = max_position;
+    p.num_pages = num_pages;
+    p.page_size = page_size;
+    p.B = B;
+    p.H = H;
+    p.Hq = Hq;
+    p.Hkv = Hkv;
+    p.d = d;
+    const int bt = qkv_batch_tile(B);
+    if (bt == 8) return launch_qkv<8>(w_map, x_map, p, stream);
+    if (bt == 16) return launch_qkv<16>(w_map, x_map, p, stream);
+    return launch_qkv<32>(w_map, x_map, p, stream);
+}
+
+}  // namespace ac

@@ -205,6 +205,15 @@ def make_workload(name: str, seed: int, B: int, Hq: int, Hkv: int, d: int, page_
                           poison_page=poison_page, extra=extra)
 
 
+def make_projection_inputs(seed: int, B: int, H: int, Hq: int, Hkv: int, d: int):
+    """Hidden states x [B,H] ~ N(0,1) and QKV weights W [(Hq+2Hkv)*d, H] ~ N(0, 1/H), both bf16 bits
+    (so that the projected features are ~N(0,1) like the q/k/v tensors of the other workloads)."""
+    x = _normal_bf16(seed, 10, (B, H))
+    n = (Hq + 2 * Hkv) * d
+    w = bf16_bits_to_f32(_normal_bf16(seed, 11, (n, H))) * np.float32(1.0 / math.sqrt(H))
+    return x, f32_to_bf16_bits(w)
+
+
 GRAPH_SWEEP_BATCHES = (1, 8, 32, 128, 256)
 
 
