@@ -377,9 +377,49 @@ def time_prelude_fusion(torch, device, batches=(1, 8, 32), replicas=12, replays=
         torch.cuda.synchronize()
         us = t0.elapsed_time(t1) * 1e3 / (replays * replicas)
         wbytes = wq.size * 2
-        rows.append({"B": B, "weight_mb": round(wbytes / 1e6, 1), "us_per_call": round(us, 2),
-                     "weight_gbs": round(wbytes / us / 1e3, 1), "status_flag": int(st.status_flag.item())})
-        del graph, xs, ws, st
+        rows.append({"kernel": "ac_qkv_rope_kv_append", "B": B, "weight_mb": round(wbytes / 1e6, 1),
+                     "us_per_call": round(us, 2), "weight_gbs": round(wbytes / us / 1e3, 1),
+                     "status_flag": int(st.status_flag.item())})
+        del graph, xs, ws
+
+        # output projection + residual + RMSNorm on the same layer: W_o [4096, 4096] (33.6 MB)
+        K, N = Hq * d, H
+        rng = np.random.default_rng(72)
+        wo = W.f32_to_bf16_bits((rng.standard_normal((N, K), dtype=np.float32) / np.float32(np.sqrt(K))))
+        a = W.f32_to_bf16_bits(rng.standard_normal((B, K), dtype=np.float32) * np.float32(0.3))
+        res = W.f32_to_bf16_bits(rng.standard_normal((B, N), dtype=np.float32))
+        nw = W.f32_to_bf16_bits(np.ones(N, dtype=np.float32))
+        dev = lambda t: torch.from_numpy(t.view(np.int16)).to(device)
+        wos = [dev(wo) for _ in range(replicas)]
+        a_d, r_d, n_d = dev(a), dev(res), dev(nw)
+        h_d, y_d = torch.empty_like(r_d), torch.empty_like(r_d)
+
+        def ocall(i, stream):
+            ac.ac_oproj_residual_rmsnorm(a_d, wos[i], K, N, r_d, h_d, n_d, 1e-5, y_d, B, stream)
+
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(replicas):
+                ocall(i, side)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(replicas):
+                ocall(i, side)
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        t0.record()
+        for _ in range(replays):
+            graph.replay()
+        t1.record()
+        torch.cuda.synchronize()
+        us = t0.elapsed_time(t1) * 1e3 / (replays * replicas)
+        rows.append({"kernel": "ac_oproj_residual_rmsnorm", "B": B, "weight_mb": round(wo.size * 2 / 1e6, 1),
+                     "us_per_call": round(us, 2), "weight_gbs": round(wo.size * 2 / us / 1e3, 1)})
+        del graph, wos, st
         torch.cuda.empty_cache()
     return rows
 

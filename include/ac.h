@@ -173,6 +173,21 @@ int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out,
                           int B, int Hq, int Hkv, int d, int page_size, int num_pages,
                           int32_t* status_flag, void* stream);
 
+/* Output-projection fusion, the paper's kernel family (v) ("an output-projection (o_proj) kernel
+ * fusing GEMV + residual + post-RMSNorm"), consuming the attention output:
+ *   h[b, n]      = bf16( residual_in[b, n] + sum_k attn_out[b, k] * w_o[n, k] )   (fp32 sum, one rounding)
+ *   normed[b, :] = RMSNorm(h[b, :]) * norm_weight = bf16( bf16( h / sqrt(mean(h^2) + eps) ) * w )
+ * attn_out [B,K] bf16 (K = Hq*d, K % 64 == 0), w_o [N,K] bf16 ([N,K] layout, N % 32 == 0),
+ * residual_in/residual_out/normed_out [B,N] bf16 (residual_out may alias residual_in), norm_weight
+ * [N] bf16.  Two dependent launches on `stream`: the weight-streaming product with the residual add
+ * in its epilogue, then the row norm (it needs all N features of a row); the second starts under the
+ * first one's tail.  The norm is exact given h (fp64 sum of squares, correctly rounded sqrt and
+ * division); h can differ from the correctly rounded value by one bf16 step (fp32 accumulation). */
+int ac_oproj_residual_rmsnorm(const void* attn_out, const void* w_o, int K, int N,
+                              const void* residual_in, void* residual_out,
+                              const void* norm_weight, float norm_eps, void* normed_out,
+                              int B, void* stream);
+
 /* A4: paged decode attention, family (iv).  Row b attends over tokens 0 .. n_b - 1 with
  * n_b = context_lens[b] + new_tokens (new_tokens = 1 right after ac_rope_kv_append, 0 to attend
  * over the cached tokens only); token t lives in page block_table[b, t / page_size], slot

@@ -236,6 +236,19 @@ def oracle_qkv_rope_kv_append(x_bits, w_qkv_bits, k_cache, v_cache, block_table,
                                  rope_cos, rope_sin, page_size)
 
 
+def oracle_oproj_residual_rmsnorm(attn_out_bits, w_o_bits, residual_bits, norm_weight_bits, eps):
+    """Output projection + residual add + post-RMSNorm (kernel family (v)).
+
+    h = bf16(residual + attn_out W_o^T) with the sum in fp64 and one rounding; normed =
+    rms_norm_bf16(h, weight, eps).  attn_out [B,K], W_o [N,K], residual [B,N], weight [N]: bf16 bits.
+    Returns (h bits, normed bits).
+    """
+    a = bf16_to_f64(attn_out_bits)
+    w = bf16_to_f64(w_o_bits)
+    h = f64_to_bf16_rne(bf16_to_f64(residual_bits) + a @ w.T)
+    return h, rms_norm_bf16(h, norm_weight_bits, eps)
+
+
 # --------------------------------------------------------------------------------------------
 # A4 + A5 as one definition: softmax(q K^T * scale) V per query head over the gathered pages
 # --------------------------------------------------------------------------------------------

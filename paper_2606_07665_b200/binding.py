@@ -26,7 +26,7 @@ EXPORTS = ("ac_init", "ac_status_string", "ac_last_cuda_error", "ac_sm_count", "
            "ac_splitkv_merge", "ac_decode_step_host", "ac_paged_decode_attn_static_scratch",
            "ac_fused_workspace_bytes", "ac_fused_workspace_reset", "ac_paged_decode_attn_fused_merge",
            "ac_decode_step_fused", "ac_paged_decode_attn_ex", "ac_decode_step_fused_ex",
-           "ac_rope_kv_append_ex", "ac_qkv_rope_kv_append")
+           "ac_rope_kv_append_ex", "ac_qkv_rope_kv_append", "ac_oproj_residual_rmsnorm")
 AC_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -84,6 +84,9 @@ def lib():
                                             [c_int64] * 3 + [c_void_p, c_int, c_void_p, c_void_p, c_void_p,
                                             c_int] + [c_int] * 6 + [c_void_p, c_void_p])
         L.ac_qkv_rope_kv_append.restype = c_int
+        L.ac_oproj_residual_rmsnorm.argtypes = [c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p,
+                                                c_float, c_void_p, c_int, c_void_p]
+        L.ac_oproj_residual_rmsnorm.restype = c_int
         L.ac_paged_decode_attn.argtypes = ([c_void_p] * 3 + [c_int64] * 3 + [c_void_p, c_int, c_void_p,
                                            c_int, c_float, c_int, c_void_p, c_size_t, c_void_p] +
                                            [c_int] * 7 + [c_void_p, c_void_p])
@@ -202,6 +205,14 @@ def ac_qkv_rope_kv_append(x, w_qkv, H, q_out, k_cache, v_cache, stride_page, str
                                        _ptr(status_flag), _stream(stream)), "ac_qkv_rope_kv_append")
 
 
+def ac_oproj_residual_rmsnorm(attn_out, w_o, K, N, residual_in, residual_out, norm_weight, norm_eps,
+                              normed_out, B, stream=None):
+    _check(lib().ac_oproj_residual_rmsnorm(_ptr(attn_out), _ptr(w_o), K, N, _ptr(residual_in),
+                                           _ptr(residual_out), _ptr(norm_weight), norm_eps,
+                                           _ptr(normed_out), B, _stream(stream)),
+           "ac_oproj_residual_rmsnorm")
+
+
 def ac_paged_decode_attn(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
                          max_pages_per_seq, context_lens, new_tokens, softmax_scale, num_splits,
                          workspace, workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages,
@@ -245,7 +256,7 @@ def ac_decode_step_fused(q_in, q_rot_out, k_new, v_new, k_cache, v_cache, stride
         _ptr(rope_cos), _ptr(rope_sin), max_position, softmax_scale, num_splits, _ptr(workspace),
         workspace_bytes, _ptr(out), B, Hq, Hkv, d, page_size, num_pages, max_context_len,
         _ptr(status_flag), _stream(stream)), "ac_decode_step_fused", "ac_paged_decode_attn_ex", "ac_decode_step_fused_ex",
-           "ac_rope_kv_append_ex", "ac_qkv_rope_kv_append")
+           "ac_rope_kv_append_ex", "ac_qkv_rope_kv_append", "ac_oproj_residual_rmsnorm")
 
 
 def _options(window: int = 0, fused_merge: bool = False):

@@ -349,6 +349,51 @@ int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out, 
     return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
 }
 
+int ac_oproj_residual_rmsnorm(const void* attn_out, const void* w_o, int K, int N,
+                              const void* residual_in, void* residual_out, const void* norm_weight,
+                              float norm_eps, void* normed_out, int B, void* stream) {
+    if (!attn_out || !w_o || !residual_in || !residual_out || !norm_weight || !normed_out) return AC_ERR_NULL;
+    if (B <= 0 || K <= 0 || N <= 0 || !(norm_eps >= 0.0f)) return AC_ERR_SHAPE;
+    if (K % 64 != 0 || N % 32 != 0 || B > 65535 * 8) return AC_ERR_UNSUPPORTED;
+    if (!aligned16(attn_out) || !aligned16(w_o) || !aligned16(residual_in) || !aligned16(residual_out) ||
+        !aligned16(norm_weight) || !aligned16(normed_out))
+        return AC_ERR_ALIGN;
+    int dev;
+    int st = current_ready_device(&dev);
+    if (st != AC_OK) return st;
+    // W_o [N, K] as (64 elements, row inside a 16-row half, half, 32-row block, 64-element K block);
+    // attn_out [B, K] as (64 elements, batch row, 64-element K block).
+    const cuuint64_t row_bytes = static_cast<cuuint64_t>(K) * 2;
+    CUtensorMap w_map, x_map;
+    {
+        cuuint64_t dims[5] = {64, 16, 2, static_cast<cuuint64_t>(N / 32), static_cast<cuuint64_t>(K / 64)};
+        cuuint64_t strides[4] = {row_bytes, row_bytes * 16, row_bytes * 32, 128};
+        cuuint32_t box[5] = {64, 16, 2, 1, 4};
+        cuuint32_t es[5] = {1, 1, 1, 1, 1};
+        CUresult r = g_encode_tiled(&w_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(w_o), dims,
+                                    strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
+    }
+    {
+        cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(B), static_cast<cuuint64_t>(K / 64)};
+        cuuint64_t strides[2] = {row_bytes, 128};
+        cuuint32_t box[3] = {64, static_cast<cuuint32_t>(qkv_batch_tile(B)), 4};
+        cuuint32_t es[3] = {1, 1, 1};
+        CUresult r = g_encode_tiled(&x_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(attn_out),
+                                    dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
+    }
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_oproj_residual(w_map, x_map, residual_in, residual_out, B, K, N, cs);
+    if (e != cudaSuccess) return fail_cuda(static_cast<int>(e));
+    e = launch_rmsnorm_rows(residual_out, norm_weight, normed_out, B, N, norm_eps, cs);
+    return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
+}
+
 static int attn_common(const void* q_rot, const void* k_cache, const void* v_cache, int64_t stride_page,
                        int64_t stride_token, int64_t stride_head, const int32_t* block_table,
                        int max_pages_per_seq, const int32_t* context_lens, int new_tokens,

@@ -84,6 +84,11 @@ cudaError_t launch_qkv_rope_kv_append(const CUtensorMap& w_map, const CUtensorMa
                                       const float* rope_sin, int max_position, int B, int H, int Hq,
                                       int Hkv, int d, int page_size, int num_pages, int32_t* status_flag,
                                       cudaStream_t stream);
+cudaError_t launch_oproj_residual(const CUtensorMap& w_map, const CUtensorMap& x_map,
+                                  const void* residual_in, void* residual_out, int B, int K, int N,
+                                  cudaStream_t stream);
+cudaError_t launch_rmsnorm_rows(const void* h, const void* weight, void* out, int B, int N, float eps,
+                                cudaStream_t stream);
 cudaError_t launch_splitkv_merge(const float* partial_o, const float* partial_lse, int num_splits,
                                  const int32_t* context_lens, void* out, int B, int Hq, int d,
                                  cudaStream_t stream);

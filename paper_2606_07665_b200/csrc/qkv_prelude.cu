@@ -15,6 +15,10 @@
 // from shared memory by ldmatrix, products run on the bf16 m16n8k16 MMA (any batch size costs the
 // same weight traffic).  At the end the warps' partial sums are reduced through shared memory and
 // the epilogue rounds, rotates and scatters.
+//
+// The same weight-streaming body also serves the output projection (kernel family (v)): there a CTA
+// owns 32 consecutive output features and the epilogue adds the residual row and rounds once; the
+// RMSNorm that follows needs all H features of a row and runs as a second, dependent launch.
 #include <math.h>
 
 #include "ac_device.cuh"
@@ -24,6 +28,8 @@ namespace ac {
 namespace {
 
 using namespace acdev;
+
+enum { EPI_QKV_ROPE_APPEND = 0, EPI_RESIDUAL_ADD = 1 };
 
 constexpr int QKV_WARPS = 8;                          // consumer warps; warp QKV_WARPS produces
 constexpr int QKV_THREADS = (QKV_WARPS + 1) * 32;
@@ -54,10 +60,14 @@ struct QkvParams {
     const float* rope_sin;
     int32_t* status_flag;
     int max_pages_per_seq, max_position, num_pages, page_size;
-    int B, H, Hq, Hkv, d;
+    int B, H, Hq, Hkv, d;           // H = contraction length K of the product
+    // output projection only
+    const uint16_t* residual_in;  // [B, N] bf16
+    uint16_t* residual_out;       // [B, N] bf16 (may alias residual_in)
+    int N;                        // output features
 };
 
-template <int BT>
+template <int BT, int EPI>
 __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
     const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map,
     const QkvParams p) {
@@ -195,6 +205,23 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
     }
     __syncthreads();
 
+    if (EPI == EPI_RESIDUAL_ADD) {
+        // ---- epilogue of the output projection: h = bf16(residual + y), one rounding ----------------
+        for (int item = threadIdx.x; item < 32 * BT; item += QKV_THREADS) {
+            const int r = item / BT;                   // row inside the 32-feature block
+            const int n = item - r * BT;
+            const int b = b0 + n;
+            if (b >= p.B) continue;
+            float y = 0.0f;
+#pragma unroll
+            for (int w = 0; w < QKV_WARPS; ++w) y += red[(w * 32 + r) * BT + n];
+            const size_t idx = static_cast<size_t>(b) * p.N + 32 * hh + r;
+            const float res = bf16_bits_to_float(p.residual_in[idx]);
+            p.residual_out[idx] = static_cast<uint16_t>(pack_bf16x2(res + y, 0.0f) & 0xFFFFu);
+        }
+        return;
+    }
+
     // ---- epilogue: round, rotate, scatter --------------------------------------------------------
     const int d = p.d, half = d / 2;
     for (int item = threadIdx.x; item < 16 * BT; item += QKV_THREADS) {
@@ -247,11 +274,12 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
     }
 }
 
-template <int BT>
+template <int BT, int EPI>
 cudaError_t launch_qkv(const CUtensorMap& w_map, const CUtensorMap& x_map, const QkvParams& p,
                        cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.d / 32, p.Hq + 2 * p.Hkv, (p.B + BT - 1) / BT);
+    cfg.gridDim = EPI == EPI_RESIDUAL_ADD ? dim3(1, p.N / 32, (p.B + BT - 1) / BT)
+                                          : dim3(p.d / 32, p.Hq + 2 * p.Hkv, (p.B + BT - 1) / BT);
     cfg.blockDim = dim3(QKV_THREADS);
     cfg.dynamicSmemBytes = QkvSmem<BT>::TOTAL;
     cfg.stream = stream;
@@ -260,7 +288,7 @@ cudaError_t launch_qkv(const CUtensorMap& w_map, const CUtensorMap& x_map, const
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, qkv_rope_append_kernel<BT>, w_map, x_map, p);
+    return cudaLaunchKernelEx(&cfg, qkv_rope_append_kernel<BT, EPI>, w_map, x_map, p);
 }
 
 }  // namespace
@@ -268,14 +296,18 @@ cudaError_t launch_qkv(const CUtensorMap& w_map, const CUtensorMap& x_map, const
 cudaError_t qkv_set_attributes(int smem_optin) {
     if (QkvSmem<32>::TOTAL > smem_optin) return cudaErrorInvalidConfiguration;
     cudaError_t e;
-    e = cudaFuncSetAttribute(qkv_rope_append_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             QkvSmem<8>::TOTAL);
+#define AC_SET(BT_, EPI_)                                                                          \
+    e = cudaFuncSetAttribute(qkv_rope_append_kernel<BT_, EPI_>,                                    \
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, QkvSmem<BT_>::TOTAL);    \
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(qkv_rope_append_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             QkvSmem<16>::TOTAL);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(qkv_rope_append_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                QkvSmem<32>::TOTAL);
+    AC_SET(8, EPI_QKV_ROPE_APPEND)
+    AC_SET(16, EPI_QKV_ROPE_APPEND)
+    AC_SET(32, EPI_QKV_ROPE_APPEND)
+    AC_SET(8, EPI_RESIDUAL_ADD)
+    AC_SET(16, EPI_RESIDUAL_ADD)
+    AC_SET(32, EPI_RESIDUAL_ADD)
+#undef AC_SET
+    return cudaSuccess;
 }
 
 int qkv_batch_tile(int B) { return B <= 8 ? 8 : (B <= 16 ? 16 : 32); }
@@ -309,10 +341,80 @@ cudaError_t launch_qkv_rope_kv_append(const CUtensorMap& w_map, const CUtensorMa
     p.Hq = Hq;
     p.Hkv = Hkv;
     p.d = d;
+    p.residual_in = nullptr;
+    p.residual_out = nullptr;
+    p.N = 0;
     const int bt = qkv_batch_tile(B);
-    if (bt == 8) return launch_qkv<8>(w_map, x_map, p, stream);
-    if (bt == 16) return launch_qkv<16>(w_map, x_map, p, stream);
-    return launch_qkv<32>(w_map, x_map, p, stream);
+    if (bt == 8) return launch_qkv<8, EPI_QKV_ROPE_APPEND>(w_map, x_map, p, stream);
+    if (bt == 16) return launch_qkv<16, EPI_QKV_ROPE_APPEND>(w_map, x_map, p, stream);
+    return launch_qkv<32, EPI_QKV_ROPE_APPEND>(w_map, x_map, p, stream);
+}
+
+// ---- RMSNorm of whole rows (second launch of the output-projection fusion) -------------------------
+namespace {
+
+// One CTA per row: sum of squares in fp64 (exact for bf16 inputs of moderate range), then
+// y = bf16(bf16(h / sqrt(mean + eps)) * w), the arithmetic of the per-head norm of the prelude.
+__global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const uint16_t* __restrict__ h,
+                                                           const uint16_t* __restrict__ weight,
+                                                           uint16_t* __restrict__ out, int N, float eps) {
+    cudaTriggerProgrammaticLaunchCompletion();
+    cudaGridDependencySynchronize();
+    __shared__ double s_part[8];
+    const uint16_t* row = h + static_cast<size_t>(blockIdx.x) * N;
+    double ss = 0.0;
+    for (int i = threadIdx.x; i < N; i += 256) {
+        const double v = static_cast<double>(bf16_bits_to_float(row[i]));
+        ss = __dadd_rn(ss, __dmul_rn(v, v));
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) ss = __dadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, off));
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    double total = 0.0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) total = __dadd_rn(total, s_part[w]);
+    const double r = __ddiv_rn(1.0, __dsqrt_rn(__dadd_rn(__ddiv_rn(total, static_cast<double>(N)),
+                                                         static_cast<double>(eps))));
+    uint16_t* orow = out + static_cast<size_t>(blockIdx.x) * N;
+    for (int i = threadIdx.x; i < N; i += 256) {
+        const double v = static_cast<double>(bf16_bits_to_float(row[i]));
+        const uint16_t y1 = f64_to_bf16_rne(__dmul_rn(v, r));
+        const double w = static_cast<double>(bf16_bits_to_float(weight[i]));
+        orow[i] = f64_to_bf16_rne(__dmul_rn(static_cast<double>(bf16_bits_to_float(y1)), w));
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_oproj_residual(const CUtensorMap& w_map, const CUtensorMap& x_map,
+                                  const void* residual_in, void* residual_out, int B, int K, int N,
+                                  cudaStream_t stream) {
+    QkvParams p = {};
+    p.B = B;
+    p.H = K;
+    p.N = N;
+    p.residual_in = static_cast<const uint16_t*>(residual_in);
+    p.residual_out = static_cast<uint16_t*>(residual_out);
+    const int bt = qkv_batch_tile(B);
+    if (bt == 8) return launch_qkv<8, EPI_RESIDUAL_ADD>(w_map, x_map, p, stream);
+    if (bt == 16) return launch_qkv<16, EPI_RESIDUAL_ADD>(w_map, x_map, p, stream);
+    return launch_qkv<32, EPI_RESIDUAL_ADD>(w_map, x_map, p, stream);
+}
+
+cudaError_t launch_rmsnorm_rows(const void* h, const void* weight, void* out, int B, int N, float eps,
+                                cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(B);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, rmsnorm_rows_kernel, static_cast<const uint16_t*>(h),
+                              static_cast<const uint16_t*>(weight), static_cast<uint16_t*>(out), N, eps);
 }
 
 }  // namespace ac

@@ -82,3 +82,41 @@ def test_qkv_prelude_matches_oracle(B, H, Hq, Hkv, d, ps):
     err = np.abs(st.out_f64() - out_ref)
     assert err.max() <= 2e-2 and err.mean() <= 2e-3
     print(f"[prelude] B={B} H={H}: exact fraction of v = {ev:.4f}")
+
+
+@pytest.mark.parametrize("B,K,N", [(1, 256, 64), (5, 320, 96), (8, 1024, 512), (13, 512, 256), (31, 768, 128),
+                                   (40, 256, 64), (4, 4096, 4096)])
+def test_oproj_residual_rmsnorm_matches_oracle(B, K, N):
+    import torch
+    from paper_2606_07665_b200 import binding as ac
+    from paper_2606_07665_b200 import build, runner
+    build.build()
+    torch.cuda.set_device(0)
+    ac.ac_init(0)
+    rng = np.random.default_rng(B * 7 + K + N)
+    a = W.f32_to_bf16_bits((rng.standard_normal((B, K)) * 0.3).astype(np.float32))
+    wo = W.f32_to_bf16_bits((rng.standard_normal((N, K)) / np.sqrt(K)).astype(np.float32))
+    res = W.f32_to_bf16_bits(rng.standard_normal((B, N)).astype(np.float32))
+    nw = W.f32_to_bf16_bits((1 + 0.1 * rng.standard_normal(N)).astype(np.float32))
+    h_ref, normed_ref = O.oracle_oproj_residual_rmsnorm(a, wo, res, nw, 1e-5)
+    dev = lambda x: torch.from_numpy(x.view(np.int16)).cuda()
+    a_d, w_d, r_d, n_d = dev(a), dev(wo), dev(res), dev(nw)
+    h_d = torch.full((B, N), 0x7FC0, dtype=torch.int16, device="cuda")
+    y_d = torch.full((B, N), 0x7FC0, dtype=torch.int16, device="cuda")
+    ac.ac_oproj_residual_rmsnorm(a_d, w_d, K, N, r_d, h_d, n_d, 1e-5, y_d, B)
+    torch.cuda.synchronize()
+    h = runner.bits_of(h_d)
+    y = runner.bits_of(y_d)
+    hf, hr = W.bf16_bits_to_f32(h).astype(np.float64), W.bf16_bits_to_f32(h_ref).astype(np.float64)
+    assert np.isfinite(hf).all()
+    assert (np.abs(hf - hr) <= 2.0 ** -7 * np.abs(hr) + 1e-30).all()        # at most one bf16 step
+    assert np.mean(h == h_ref) >= 0.97
+    # the norm is exact given the h the kernel produced
+    assert np.array_equal(y, O.rms_norm_bf16(h, nw, 1e-5))
+    # and close to the oracle's end-to-end result
+    yf, yr = W.bf16_bits_to_f32(y).astype(np.float64), W.bf16_bits_to_f32(normed_ref).astype(np.float64)
+    assert np.abs(yf - yr).max() <= 2.0 ** -6 * np.abs(yr).max()
+    # in place on the residual stream
+    ac.ac_oproj_residual_rmsnorm(a_d, w_d, K, N, r_d, r_d, n_d, 1e-5, y_d, B)
+    torch.cuda.synchronize()
+    assert np.array_equal(runner.bits_of(r_d), h)

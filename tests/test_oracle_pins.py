@@ -590,6 +590,25 @@ def test_qkv_projection_pins():
         assert np.array_equal(a, bb)
 
 
+def test_oproj_residual_rmsnorm_pins():
+    rng = np.random.default_rng(43)
+    B, K, N = 3, 16, 8
+    a = W.f32_to_bf16_bits(rng.standard_normal((B, K)).astype(np.float32))
+    wo = W.f32_to_bf16_bits((rng.standard_normal((N, K)) / 4).astype(np.float32))
+    res = W.f32_to_bf16_bits(rng.standard_normal((B, N)).astype(np.float32))
+    nw = W.f32_to_bf16_bits((1 + 0.1 * rng.standard_normal(N)).astype(np.float32))
+    h, normed = O.oracle_oproj_residual_rmsnorm(a, wo, res, nw, 1e-5)
+    for b in range(B):
+        for n in range(N):
+            acc = bf16_value(int(res[b, n])) + sum(bf16_value(int(a[b, k])) * bf16_value(int(wo[n, k]))
+                                                   for k in range(K))
+            assert int(h[b, n]) == fraction_to_bf16(acc)            # residual + product, rounded once
+    assert np.array_equal(normed, O.rms_norm_bf16(h, nw, 1e-5))
+    # zero weights: h is the residual, bit for bit
+    h0, _ = O.oracle_oproj_residual_rmsnorm(a, np.zeros_like(wo), res, nw, 1e-5)
+    assert np.array_equal(h0, res)
+
+
 def test_tiny_workload_oracle_result_is_frozen():
     import importlib.util
     import os
