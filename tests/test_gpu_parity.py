@@ -404,6 +404,45 @@ def test_sliding_window(rt, window, splits, fused):
     run_and_compare(rt, w, num_splits=splits, fused=fused, window=window)
 
 
+@pytest.mark.parametrize("fused", [True, "step"])
+@pytest.mark.parametrize("kw", [
+    dict(B=2, Hq=16, Hkv=1, d=128, page_size=16, context_lens=[700, 33], num_pages=64),            # multi-query
+    dict(B=2, Hq=4, Hkv=4, d=64, page_size=256, context_lens=[1000, 255], num_pages=8),            # largest page
+    dict(B=3, Hq=8, Hkv=2, d=128, page_size=64, context_lens=[63, 64, 4000], num_pages=72),
+    dict(B=1, Hq=64, Hkv=4, d=64, page_size=16, context_lens=[129], num_pages=12),                 # group of 16, d = 64
+])
+def test_extreme_shapes(rt, kw, fused):
+    run_and_compare(rt, small(52, **kw), fused=fused)
+    run_and_compare(rt, small(52, **kw), fused=fused, num_splits=1, check_cache=False)
+
+
+@pytest.mark.parametrize("fused", [True, "step"])
+def test_many_short_requests(rt, fused):
+    # 1500 rows of 0..40 tokens: grid rows far beyond one wave, most tiles ragged, some rows inactive
+    rng = np.random.default_rng(12)
+    lens = rng.integers(0, 41, size=1500).tolist()
+    w = W.make_workload("many", 53, B=1500, Hq=8, Hkv=2, d=64, page_size=16, num_pages=4700,
+                        context_lens=lens, rope_base=10000.0, inactive_rows=(3, 700, 1499))
+    run_and_compare(rt, w, fused=fused)
+
+
+@pytest.mark.parametrize("fused", [True, "step"])
+def test_one_very_long_request(rt, fused):
+    # 400k tokens for one KV head: many splits, positions far into the rope table, > 2^24 cache elements
+    import torch
+    w = W.make_workload("verylong", 54, B=1, Hq=4, Hkv=1, d=128, page_size=32, num_pages=12600,
+                        context_lens=[400_000], rope_base=1000000.0)
+    st = rt.DecodeStep(w, fused_merge=True, fused_step=(fused == "step"))
+    st.step()
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) == 0 and st.num_splits > 8
+    q_rot, k_after, v_after, out_ref = O.oracle_decode_step(w)
+    assert np.array_equal(rt.bits_of(st.q_rot), q_rot)
+    k_gpu, v_gpu = st.cache_bits()
+    assert np.array_equal(k_gpu, k_after) and np.array_equal(v_gpu, v_after)
+    check_out(st.out_f64(), out_ref, "400k-token request")
+
+
 def test_peaked_scores(rt):
     w = W.make_workload("peaked", 48, B=2, Hq=16, Hkv=2, d=128, page_size=16, num_pages=300,
                         context_lens=[2000, 1500], rope_base=500000.0, peak_fraction=0.01)
