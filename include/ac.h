@@ -264,7 +264,13 @@ typedef struct ac_attn_options {
                         only, i.e. tokens max(0, n_b - window) .. n_b - 1 (the paper wires a sliding
                         window in for one of its model families, "Per-Model Adaptations"); 0: all */
     int fused_merge; /* ac_paged_decode_attn_ex only: non-zero = behave as ac_paged_decode_attn_fused_merge */
-    int reserved[6];
+    const int32_t* row_order; /* optional device array [B], a permutation of 0..B-1: grid row y serves
+                        request row_order[y].  CTAs are dispatched in grid order, so listing the requests
+                        by decreasing context length (what a scheduler that knows the lengths can do
+                        for free) shortens the tail of grids that are several waves deep.  Any
+                        permutation gives the same results.  NULL: the kernel ranks the requests
+                        itself when B <= 128 and serves them in index order otherwise. */
+    int reserved[4];
 } ac_attn_options;
 
 /* ac_paged_decode_attn / ac_paged_decode_attn_fused_merge / ac_decode_step_fused with options

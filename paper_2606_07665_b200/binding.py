@@ -32,7 +32,7 @@ AC_STATIC_SCRATCH_BYTES = 8 << 20
 
 class AcAttnOptions(ctypes.Structure):
     """Mirror of ac_attn_options."""
-    _fields_ = [("window", c_int), ("fused_merge", c_int), ("reserved", c_int * 6)]
+    _fields_ = [("window", c_int), ("fused_merge", c_int), ("row_order", c_void_p), ("reserved", c_int * 4)]
 
 
 class AcRopeOptions(ctypes.Structure):
@@ -259,22 +259,24 @@ def ac_decode_step_fused(q_in, q_rot_out, k_new, v_new, k_cache, v_cache, stride
            "ac_rope_kv_append_ex", "ac_qkv_rope_kv_append", "ac_oproj_residual_rmsnorm")
 
 
-def _options(window: int = 0, fused_merge: bool = False):
+def _options(window: int = 0, fused_merge: bool = False, row_order=None):
     opt = AcAttnOptions()
     opt.window = int(window)
     opt.fused_merge = 1 if fused_merge else 0
+    opt.row_order = _ptr(row_order)
     return ctypes.byref(opt)
 
 
 def ac_paged_decode_attn_ex(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
                             max_pages_per_seq, context_lens, new_tokens, softmax_scale, num_splits,
                             workspace, workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages,
-                            max_context_len, status_flag=None, stream=None, window=0, fused_merge=False):
+                            max_context_len, status_flag=None, stream=None, window=0, fused_merge=False,
+                            row_order=None):
     _check(lib().ac_paged_decode_attn_ex(
         _ptr(q_rot), _ptr(k_cache), _ptr(v_cache), stride_page, stride_token, stride_head,
         _ptr(block_table), max_pages_per_seq, _ptr(context_lens), new_tokens, softmax_scale, num_splits,
         _ptr(workspace), workspace_bytes, _ptr(out), B, Hq, Hkv, d, page_size, num_pages,
-        max_context_len, _ptr(status_flag), _stream(stream), _options(window, fused_merge)),
+        max_context_len, _ptr(status_flag), _stream(stream), _options(window, fused_merge, row_order)),
         "ac_paged_decode_attn_ex")
 
 
@@ -282,13 +284,13 @@ def ac_decode_step_fused_ex(q_in, q_rot_out, k_new, v_new, k_cache, v_cache, str
                             stride_head, block_table, max_pages_per_seq, context_lens, rope_cos, rope_sin,
                             max_position, softmax_scale, num_splits, workspace, workspace_bytes, out, B,
                             Hq, Hkv, d, page_size, num_pages, max_context_len, status_flag=None,
-                            stream=None, window=0):
+                            stream=None, window=0, row_order=None):
     _check(lib().ac_decode_step_fused_ex(
         _ptr(q_in), _ptr(q_rot_out), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), stride_page,
         stride_token, stride_head, _ptr(block_table), max_pages_per_seq, _ptr(context_lens),
         _ptr(rope_cos), _ptr(rope_sin), max_position, softmax_scale, num_splits, _ptr(workspace),
         workspace_bytes, _ptr(out), B, Hq, Hkv, d, page_size, num_pages, max_context_len,
-        _ptr(status_flag), _stream(stream), _options(window)), "ac_decode_step_fused_ex")
+        _ptr(status_flag), _stream(stream), _options(window, False, row_order)), "ac_decode_step_fused_ex")
 
 
 def ac_splitkv_merge(workspace, num_splits, context_lens, out, B, Hq, d, stream=None):

@@ -400,7 +400,8 @@ static int attn_common(const void* q_rot, const void* k_cache, const void* v_cac
                        float softmax_scale, int num_splits, void* workspace, size_t workspace_bytes,
                        void* out, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
                        int max_context_len, int32_t* status_flag, void* stream, bool fused_merge,
-                       const FusedRopeArgs* rope = nullptr, int window = 0) {
+                       const FusedRopeArgs* rope = nullptr, int window = 0,
+                       const int32_t* row_order = nullptr) {
     if (!q_rot || !k_cache || !v_cache || !block_table || !context_lens) return AC_ERR_NULL;
     Shape s{B, Hq, Hkv, d, page_size, num_pages};
     int st = check_shape(s);
@@ -446,7 +447,7 @@ static int attn_common(const void* q_rot, const void* k_cache, const void* v_cac
                                              max_pages_per_seq, context_lens, new_tokens, scale,
                                              num_splits, split_tokens, partial_o, partial_lse, arrivals,
                                              out, B, Hq, Hkv, d, page_size, status_flag, rope, window,
-                                             static_cast<cudaStream_t>(stream));
+                                             row_order, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
 }
 
@@ -516,6 +517,7 @@ int ac_decode_step_fused_ex(const void* q_in, void* q_rot_out, const void* k_new
                             int page_size, int num_pages, int max_context_len, int32_t* status_flag,
                             void* stream, const ac_attn_options* options) {
     const int window = options != nullptr ? options->window : 0;
+    const int32_t* row_order = options != nullptr ? options->row_order : nullptr;
     if (!q_in || !k_new || !v_new || !rope_cos || !rope_sin) return AC_ERR_NULL;
     if (max_position <= 0) return AC_ERR_SHAPE;
     if (q_rot_out == q_in) return AC_ERR_UNSUPPORTED;      // other CTAs still read the raw rows
@@ -538,7 +540,7 @@ int ac_decode_step_fused_ex(const void* q_in, void* q_rot_out, const void* k_new
     return attn_common(q_in, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
                        max_pages_per_seq, context_lens, 1, softmax_scale, num_splits, workspace,
                        workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages, max_context_len,
-                       status_flag, stream, true, &rope, window);
+                       status_flag, stream, true, &rope, window, row_order);
 }
 
 int ac_paged_decode_attn_ex(const void* q_rot, const void* k_cache, const void* v_cache,
@@ -550,10 +552,11 @@ int ac_paged_decode_attn_ex(const void* q_rot, const void* k_cache, const void* 
                             int32_t* status_flag, void* stream, const ac_attn_options* options) {
     const bool fused = options != nullptr && options->fused_merge != 0;
     const int window = options != nullptr ? options->window : 0;
+    const int32_t* row_order = options != nullptr ? options->row_order : nullptr;
     return attn_common(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
                        max_pages_per_seq, context_lens, new_tokens, softmax_scale, num_splits, workspace,
                        workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages, max_context_len,
-                       status_flag, stream, fused, nullptr, window);
+                       status_flag, stream, fused, nullptr, window, row_order);
 }
 
 int ac_splitkv_merge(const void* workspace, int num_splits, const int32_t* context_lens, void* out,

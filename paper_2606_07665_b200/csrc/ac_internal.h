@@ -73,7 +73,8 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
                                      int num_splits, int split_tokens, float* partial_o,
                                      float* partial_lse, int32_t* arrivals, void* out, int B, int Hq,
                                      int Hkv, int d, int page_size, int32_t* status_flag,
-                                     const FusedRopeArgs* rope, int window, cudaStream_t stream);
+                                     const FusedRopeArgs* rope, int window, const int32_t* row_order,
+                                     cudaStream_t stream);
 cudaError_t qkv_set_attributes(int smem_optin);
 int qkv_batch_tile(int B);
 cudaError_t launch_qkv_rope_kv_append(const CUtensorMap& w_map, const CUtensorMap& x_map, void* q_out,

@@ -80,6 +80,7 @@ struct AttnParams {
     int split_tokens;
     int Hq, Hkv, page_size;
     int fused_merge;              // 1: the last CTA of a (request, KV head) merges the splits itself
+    const int32_t* row_order;     // optional [B] permutation: grid row y serves request row_order[y]
     int longest_first;            // 1: grid row y serves the request with the y-th longest context
     int window;                   // > 0: attend over the last `window` tokens of each row only
 };
@@ -102,7 +103,11 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     int b = blockIdx.y;
-    if (p.longest_first) {
+    if (p.row_order != nullptr) {
+        // The caller (a scheduler that knows the lengths) supplied the order in which grid rows serve
+        // requests, normally longest first.
+        b = p.row_order[blockIdx.y];
+    } else if (p.longest_first) {
         // The hardware hands out CTAs in grid order; when the grid is several waves deep, serving
         // the longest requests first keeps the short ones for the tail of the grid (greedy
         // longest-processing-time order).  Every CTA derives the same ranking from context_lens:
@@ -674,8 +679,10 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
                                      int num_splits, int split_tokens, float* partial_o,
                                      float* partial_lse, int32_t* arrivals, void* out, int B, int Hq,
                                      int Hkv, int d, int page_size, int32_t* status_flag,
-                                     const FusedRopeArgs* rope, int window, cudaStream_t stream) {
+                                     const FusedRopeArgs* rope, int window, const int32_t* row_order,
+                                     cudaStream_t stream) {
     AttnParams p;
+    p.row_order = row_order;
     p.window = window > 0 ? window : 0;
     p.q_rot_out = nullptr;
     p.k_new = p.v_new = nullptr;

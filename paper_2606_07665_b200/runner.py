@@ -30,7 +30,7 @@ class DecodeStep:
 
     def __init__(self, w, device="cuda:0", num_splits: int | None = None, layout: str = "token_major",
                  max_context_len: int | None = None, fused_merge: bool = True,
-                 fused_step: bool = False, window: int = 0):
+                 fused_step: bool = False, window: int = 0, row_order="auto"):
         self.w = w
         self.window = int(window) if window else int(getattr(w, "window", 0))   # > 0: sliding window
         self.fused_step = bool(fused_step)             # one launch: RoPE + append + attention + merge
@@ -64,6 +64,12 @@ class DecodeStep:
         self.context_lens = torch.from_numpy(w.context_lens).to(self.device)
         self.rope_cos = torch.from_numpy(w.rope_cos).to(self.device)
         self.rope_sin = torch.from_numpy(w.rope_sin).to(self.device)
+        # Scheduling hint: requests by decreasing length (what a scheduler that knows the lengths
+        # hands over with the block table).  "auto": only where the kernel does not rank by itself.
+        if isinstance(row_order, str) and row_order == "auto":
+            row_order = (np.argsort(-w.context_lens.astype(np.int64), kind="stable").astype(np.int32)
+                         if w.B > 128 else None)
+        self.row_order = None if row_order is None else torch.from_numpy(np.asarray(row_order, np.int32)).to(self.device)
         self.out = torch.zeros((self.B, self.Hq, self.d), dtype=torch.int16, device=self.device)
         self.status_flag = torch.zeros(1, dtype=torch.int32, device=self.device)
         self.max_context_len = int(max_context_len) if max_context_len else w.max_context_len
@@ -106,7 +112,7 @@ class DecodeStep:
                              self.num_pages, self.status_flag, stream)
 
     def attention(self, stream=None, new_tokens: int = 1, q=None) -> None:
-        if self.window > 0:
+        if self.window > 0 or self.row_order is not None:
             ac.ac_paged_decode_attn_ex(self.q_rot if q is None else q, self.k_cache, self.v_cache,
                                        self.stride_page, self.stride_token, self.stride_head,
                                        self.block_table, self.w.max_pages_per_seq, self.context_lens,
@@ -114,7 +120,8 @@ class DecodeStep:
                                        self.workspace if self.num_splits > 1 else None,
                                        self.workspace_bytes, self.out, self.B, self.Hq, self.Hkv, self.d,
                                        self.ps, self.num_pages, self.max_context_len, self.status_flag,
-                                       stream, window=self.window, fused_merge=self.fused_merge)
+                                       stream, window=self.window, fused_merge=self.fused_merge,
+                                       row_order=self.row_order)
             return
         fn = ac.ac_paged_decode_attn_fused_merge if self.fused_merge else ac.ac_paged_decode_attn
         fn(self.q_rot if q is None else q, self.k_cache, self.v_cache,
@@ -136,7 +143,8 @@ class DecodeStep:
                                    self.rope_cos, self.rope_sin, self.w.max_position, 0.0, self.num_splits,
                                    self.workspace if self.num_splits > 1 else None, self.workspace_bytes,
                                    self.out, self.B, self.Hq, self.Hkv, self.d, self.ps, self.num_pages,
-                                   self.max_context_len, self.status_flag, stream, window=self.window)
+                                   self.max_context_len, self.status_flag, stream, window=self.window,
+                                   row_order=self.row_order)
 
     def step(self, stream=None) -> None:
         if self.fused_step:

@@ -494,6 +494,31 @@ def test_longest_first_row_order_with_ties_and_inactive_rows(rt, splits):
     assert (rt.bits_of(st.out)[[0, 17, 99]] == 0).all()
 
 
+@pytest.mark.parametrize("fused", [False, True, "step"])
+def test_caller_supplied_row_order(rt, fused):
+    # any permutation of the rows gives the same result; the runner's default for large batches is
+    # "longest first", here also a random one and the identity, on a grid several waves deep
+    import torch
+    rng = np.random.default_rng(13)
+    lens = rng.integers(0, 600, size=200).tolist()
+    w = W.make_workload("order", 55, B=200, Hq=8, Hkv=4, d=64, page_size=16, num_pages=8000,
+                        context_lens=lens, rope_base=10000.0, inactive_rows=(5, 150))
+    q_rot, k_after, v_after, out_ref = O.oracle_decode_step(w)
+    outs = []
+    for order in ("auto", rng.permutation(200).astype(np.int32), None):
+        st = rt.DecodeStep(w, num_splits=2, fused_merge=bool(fused), fused_step=(fused == "step"),
+                           row_order=order)
+        assert (st.row_order is not None) == (order is not None)
+        st.step()
+        torch.cuda.synchronize()
+        assert int(st.status_flag.item()) == 0
+        check_out(st.out_f64(), out_ref, "row order")
+        k_gpu, v_gpu = st.cache_bits()
+        assert np.array_equal(k_gpu, k_after) and np.array_equal(v_gpu, v_after)
+        outs.append(rt.bits_of(st.out).copy())
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+
+
 def test_fused_merge_repeated_launches_and_row_without_tokens(rt):
     # The arrival counters reset themselves: many launches on one workspace stay correct, also when a
     # row has no tokens at all (its output is +0) and when most splits of a short row are empty.
