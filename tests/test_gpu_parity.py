@@ -443,6 +443,22 @@ def test_one_very_long_request(rt, fused):
     check_out(st.out_f64(), out_ref, "400k-token request")
 
 
+@pytest.mark.parametrize("fused", [False, True, "step"])
+def test_batch_of_only_inactive_rows(rt, fused):
+    # a bucket that is all padding: nothing is written to the cache, every output row is +0
+    import torch
+    w = small(56, B=3, context_lens=[40, 50, 60], num_pages=32, inactive_rows=(0, 1, 2))
+    st = rt.DecodeStep(w, num_splits=2, fused_merge=bool(fused), fused_step=(fused == "step"))
+    before_k, before_v = st.cache_bits()
+    st.out.fill_(0x7FC0)
+    st.step()
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) == 0
+    after_k, after_v = st.cache_bits()
+    assert np.array_equal(before_k, after_k) and np.array_equal(before_v, after_v)
+    assert (rt.bits_of(st.out) == 0).all()
+
+
 def test_peaked_scores(rt):
     w = W.make_workload("peaked", 48, B=2, Hq=16, Hkv=2, d=128, page_size=16, num_pages=300,
                         context_lens=[2000, 1500], rope_base=500000.0, peak_fraction=0.01)
