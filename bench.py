@@ -424,6 +424,54 @@ def time_prelude_fusion(torch, device, batches=(1, 8, 32), replicas=12, replays=
     return rows
 
 
+def time_attention_block(torch, device, batches=(1, 8, 32), replicas=8, replays=20):
+    """The whole attention block of an 8B-class layer for one decode step -- QKV projection + RoPE +
+    append, paged attention (contexts uniform in [512, 2048]), output projection + residual + RMSNorm
+    -- as the chain of launches a serving graph would hold, cycled over `replicas` separate copies of
+    weights and caches inside one captured graph (84 MB of weights + the K/V per copy, cold in L2)."""
+    from paper_2606_07665_b200 import runner
+    H, Hq, Hkv, d, ps = 4096, 32, 8, 128, 16
+    rows = []
+    for B in batches:
+        lens = np.random.default_rng(100 + B).integers(512, 2049, size=B).tolist()
+        w = W.make_workload("block", 73, B=B, Hq=Hq, Hkv=Hkv, d=d, page_size=ps, num_pages=B * 132 + 8,
+                            context_lens=lens, rope_base=500000.0)
+        hidden, wq = W.make_projection_inputs(74, B, H, Hq, Hkv, d)
+        rng = np.random.default_rng(75)
+        wo = W.f32_to_bf16_bits(rng.standard_normal((H, Hq * d), dtype=np.float32) / np.float32(np.sqrt(Hq * d)))
+        nw = W.f32_to_bf16_bits(np.ones(H, dtype=np.float32))
+        blocks = [runner.AttentionBlockStep(w, hidden, wq, wo, nw, 1e-5, device=device) for _ in range(replicas)]
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for blk in blocks:
+                blk.step(side)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for blk in blocks:
+                blk.step(side)
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        t0 = torch.cuda.Event(enable_timing=True)
+        t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(replays):
+            graph.replay()
+        t1.record()
+        torch.cuda.synchronize()
+        us = t0.elapsed_time(t1) * 1e3 / (replays * replicas)
+        moved = wq.size * 2 + wo.size * 2 + w.kv_bytes
+        rows.append({"B": B, "us_per_block": round(us, 2), "bytes_mb": round(moved / 1e6, 1),
+                     "gbs": round(moved / us / 1e3, 1), "num_splits": blocks[0].step_.num_splits,
+                     "launches": 4, "status_flag": int(blocks[0].step_.status_flag.item())})
+        del graph, blocks
+        torch.cuda.empty_cache()
+    return rows
+
+
 def time_single_graph_call(st, torch, reps=30):
     """us per call when every call is its own graph launch (host launch overhead included), L2
     flushed between calls: write a buffer 4x L2, then read it so its dirty lines are written back."""
@@ -519,12 +567,16 @@ def run_ours(args):
             prelude = time_prelude_fusion(torch, device)
             for r in prelude:
                 r["frac_of_hbm_peak"] = round(r["weight_gbs"] / peak, 4)
+            block = time_attention_block(torch, device)
+            for r in block:
+                r["frac_of_hbm_peak"] = round(r["gbs"] / peak, 4)
             cpu_bytes, cpu_s, cpu_desc = oracle_sample_seconds(w, 12.0)
             cpu = {"value": cpu_bytes / cpu_s / 1e9, "unit": UNIT, "cores": cpu_threads_used(),
                    "kind": "oracle", "sample": cpu_desc}
         else:
             cpu = None
             prelude = []
+            block = []
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -548,7 +600,7 @@ def run_ours(args):
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
             "gpu_launches": args.steps * launches_per_step,
             "clocks": clocks, "status_flag": flag, "workloads": others,
-            "prelude_fusion": prelude,
+            "prelude_fusion": prelude, "attention_block": block,
         }
         print(json.dumps(line))
     if world > 1:

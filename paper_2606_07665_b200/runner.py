@@ -191,3 +191,36 @@ class DecodeStep:
         po = ws[:n * self.d].reshape(self.B, self.Hq, self.num_splits, self.d)
         pl = ws[n * self.d:n * self.d + n].reshape(self.B, self.Hq, self.num_splits)
         return po, pl
+
+
+class AttentionBlockStep:
+    """The attention block of one decoder layer for one decode step, as three launches in a row:
+    QKV projection + RoPE + KV append, paged decode attention with the merge fused in, output
+    projection + residual + RMSNorm.  ``hidden`` [B,H], ``w_qkv`` [(Hq+2Hkv)*d, H], ``w_o`` [H, Hq*d],
+    ``norm_weight`` [H] are uint16 arrays of bf16 bits; ``hidden`` is both the projection's input and
+    the residual stream."""
+
+    def __init__(self, w, hidden, w_qkv, w_o, norm_weight, norm_eps=1e-5, device="cuda:0",
+                 num_splits: int | None = None):
+        self.step_ = DecodeStep(w, device=device, num_splits=num_splits, fused_merge=True)
+        st = self.step_
+        self.H = int(hidden.shape[1])
+        self.norm_eps = float(norm_eps)
+        self.hidden = _dev_u16(hidden, st.device)
+        self.w_qkv = _dev_u16(w_qkv, st.device)
+        self.w_o = _dev_u16(w_o, st.device)
+        self.norm_weight = _dev_u16(norm_weight, st.device)
+        self.residual_out = torch.empty_like(self.hidden)
+        self.normed_out = torch.empty_like(self.hidden)
+
+    def step(self, stream=None) -> None:
+        st = self.step_
+        ac.ac_qkv_rope_kv_append(self.hidden, self.w_qkv, self.H, st.q_rot, st.k_cache, st.v_cache,
+                                 st.stride_page, st.stride_token, st.stride_head, st.block_table,
+                                 st.w.max_pages_per_seq, st.context_lens, st.rope_cos, st.rope_sin,
+                                 st.w.max_position, st.B, st.Hq, st.Hkv, st.d, st.ps, st.num_pages,
+                                 st.status_flag, stream)
+        st.attention(stream)
+        ac.ac_oproj_residual_rmsnorm(st.out, self.w_o, st.Hq * st.d, self.H, self.hidden,
+                                     self.residual_out, self.norm_weight, self.norm_eps, self.normed_out,
+                                     st.B, stream)

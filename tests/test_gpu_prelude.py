@@ -120,3 +120,59 @@ def test_oproj_residual_rmsnorm_matches_oracle(B, K, N):
     ac.ac_oproj_residual_rmsnorm(a_d, w_d, K, N, r_d, r_d, n_d, 1e-5, y_d, B)
     torch.cuda.synchronize()
     assert np.array_equal(runner.bits_of(r_d), h)
+
+
+def test_attention_block_chain_matches_oracle_chain():
+    """Projection -> attention -> output projection, the three launches back to back on one stream,
+    against the same chain in the oracle.  One-ulp differences of the bf16 projections propagate, so
+    the end results are compared with a tolerance relative to their scale."""
+    import torch
+    from paper_2606_07665_b200 import binding as ac
+    from paper_2606_07665_b200 import build, runner
+    build.build()
+    torch.cuda.set_device(0)
+    ac.ac_init(0)
+    B, H, Hq, Hkv, d, ps = 6, 1024, 8, 2, 128, 16
+    rng = np.random.default_rng(77)
+    lens = rng.integers(0, 900, size=B).tolist()
+    w = W.make_workload("block", 78, B=B, Hq=Hq, Hkv=Hkv, d=d, page_size=ps, num_pages=B * 60 + 4,
+                        context_lens=lens, rope_base=10000.0)
+    hidden, wq = W.make_projection_inputs(79, B, H, Hq, Hkv, d)
+    wo = W.f32_to_bf16_bits((rng.standard_normal((H, Hq * d)) / np.sqrt(Hq * d)).astype(np.float32))
+    nw = W.f32_to_bf16_bits((1 + 0.1 * rng.standard_normal(H)).astype(np.float32))
+    # oracle chain
+    q_rot, k_after, v_after = O.oracle_qkv_rope_kv_append(hidden, wq, w.k_cache, w.v_cache, w.block_table,
+                                                          w.context_lens, w.rope_cos, w.rope_sin, ps, Hq, Hkv, d)
+    attn = O.oracle_paged_decode_attn(q_rot, k_after, v_after, w.block_table, w.context_lens, ps)
+    attn_bits = O.f64_to_bf16_rne(attn).reshape(B, Hq * d)
+    h_ref, y_ref = O.oracle_oproj_residual_rmsnorm(attn_bits, wo, hidden, nw, 1e-5)
+    blk = runner.AttentionBlockStep(w, hidden, wq, wo, nw, 1e-5, num_splits=2)
+    blk.step()
+    torch.cuda.synchronize()
+    assert int(blk.step_.status_flag.item()) == 0
+    for got_t, ref in ((blk.residual_out, h_ref), (blk.normed_out, y_ref)):
+        got = W.bf16_bits_to_f32(runner.bits_of(got_t)).astype(np.float64)
+        want = W.bf16_bits_to_f32(ref).astype(np.float64)
+        rms = np.sqrt(np.mean(want ** 2))
+        assert np.isfinite(got).all()
+        assert np.abs(got - want).max() <= 3e-2 * rms
+        assert np.abs(got - want).mean() <= 2e-3 * rms
+    # captured as one graph and replayed: same bits as the eager chain
+    first = runner.bits_of(blk.normed_out).copy()
+    blk2 = runner.AttentionBlockStep(w, hidden, wq, wo, nw, 1e-5, num_splits=2)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        blk2.step(side)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    fresh = runner.DecodeStep(w)
+    blk2.step_.k_cache.copy_(fresh.k_cache); blk2.step_.v_cache.copy_(fresh.v_cache)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        blk2.step(side)
+    blk2.step_.k_cache.copy_(fresh.k_cache); blk2.step_.v_cache.copy_(fresh.v_cache)
+    blk2.normed_out.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert np.array_equal(runner.bits_of(blk2.normed_out), first)
