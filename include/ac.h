@@ -25,6 +25,13 @@
  *     device memory on the host: each call only validates its arguments and enqueues work on
  *     `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream).  The three kernel
  *     calls may therefore be recorded in a CUDA Graph; ac_init must have been called before capture.
+ *   - The kernels are launched with programmatic stream serialization and signal launch completion
+ *     early, so that in a chain of calls each kernel's set-up overlaps the tail of the one before.
+ *     Before synchronising on the preceding kernel the attention kernels read only context_lens,
+ *     block_table and cache tiles below the one holding slot context_lens[b] - 1.  This is invisible
+ *     unless the kernel enqueued directly before one of these calls BOTH writes context_lens or
+ *     block_table AND itself signals programmatic launch completion before finishing; such a
+ *     producer must not signal early (copies and ordinary kernels are always safe).
  *   - Tensors q/k/v/cache/out are bf16 (16-bit patterns); rope tables and partials are fp32;
  *     block_table and context_lens are int32.  The innermost dimension (head_dim) is contiguous.
  *   - Return value: AC_OK (0) or an ac_status > 0.  On any non-zero return nothing was launched.
@@ -309,7 +316,10 @@ int ac_splitkv_merge(const void* workspace, int num_splits, const int32_t* conte
  * end-to-end timing): copies q/k_new/v_new/block_table/context_lens from the *_host buffers (pinned
  * memory recommended) into the caller's device buffers of the same name, resets the arrival
  * counters, enqueues ac_decode_step_fused for the given num_splits (workspace_bytes >=
- * ac_fused_workspace_bytes), and copies the bf16 result from out into out_host.  Everything is asynchronous on `stream`; the caller
+ * ac_fused_workspace_bytes), and copies the bf16 result from out into out_host.  When the host
+ * buffers are pinned memory the GPU can address and their sizes are multiples of 16 bytes, the five
+ * inputs are gathered (and the counters cleared) by ONE small kernel reading host memory directly
+ * instead of five copy-engine transfers; otherwise each buffer gets its own cudaMemcpyAsync.  Everything is asynchronous on `stream`; the caller
  * synchronises the stream before reading out_host.  The KV cache pools and rope tables stay on the
  * device (they are the layer's resident state, not a per-step input).  No paper counterpart. */
 int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* v_new_host,

@@ -599,20 +599,49 @@ int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* 
     st = current_ready_device(&dev);
     if (st != AC_OK) return st;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    st = ac_fused_workspace_reset(workspace, workspace_bytes, B, Hq, Hkv, d, num_splits, stream);
-    if (st != AC_OK) return st;
     const size_t q_bytes = static_cast<size_t>(B) * Hq * d * 2;
     const size_t kv_bytes = static_cast<size_t>(B) * Hkv * d * 2;
-    cudaError_t e;
-    if ((e = cudaMemcpyAsync(q, q_host, q_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(k_new, k_new_host, kv_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(v_new, v_new_host, kv_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(block_table, block_table_host,
-                             static_cast<size_t>(B) * max_pages_per_seq * sizeof(int32_t),
-                             cudaMemcpyHostToDevice, cs)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(context_lens, context_lens_host, static_cast<size_t>(B) * sizeof(int32_t),
-                             cudaMemcpyHostToDevice, cs)) != cudaSuccess)
-        return fail_cuda(static_cast<int>(e));
+    const size_t bt_bytes = static_cast<size_t>(B) * max_pages_per_seq * sizeof(int32_t);
+    const size_t len_bytes = static_cast<size_t>(B) * sizeof(int32_t);
+    cudaError_t e = cudaErrorInvalidValue;
+    {
+        // Preferred: one kernel gathers the five host buffers (pinned, GPU-addressable) and clears the
+        // arrival counters.  Sizes that are not multiples of 16 bytes, or host memory the GPU cannot
+        // address, fall back to one copy-engine transfer per buffer.
+        const size_t len_padded = (len_bytes + 15) / 16 * 16, bt_padded = (bt_bytes + 15) / 16 * 16;
+        const bool tails_ok = len_padded == len_bytes && bt_padded == bt_bytes;
+        if (tails_ok) {
+            const void* src[5] = {q_host, k_new_host, v_new_host, block_table_host, context_lens_host};
+            void* dst[5] = {q, k_new, v_new, block_table, context_lens};
+            const size_t bytes[5] = {q_bytes, kv_bytes, kv_bytes, bt_bytes, len_bytes};
+            void* zero_dst = nullptr;
+            size_t zero_bytes = 0;
+            if (num_splits > 1) {
+                // counters follow the partials; clear from the 16-byte boundary at or below their start
+                // (the bytes before it belong to partial_lse, which every launch rewrites before use)
+                const size_t off = ac_workspace_bytes(B, Hq, d, num_splits);
+                const size_t lo = off / 16 * 16;
+                const size_t hi = (off + static_cast<size_t>(B) * Hkv * sizeof(int32_t) + 15) / 16 * 16;
+                if (hi <= workspace_bytes) {
+                    zero_dst = static_cast<char*>(workspace) + lo;
+                    zero_bytes = hi - lo;
+                }
+            }
+            if (num_splits == 1 || zero_dst != nullptr)
+                e = launch_stage_inputs(src, dst, bytes, zero_dst, zero_bytes, cs);
+        }
+    }
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        st = ac_fused_workspace_reset(workspace, workspace_bytes, B, Hq, Hkv, d, num_splits, stream);
+        if (st != AC_OK) return st;
+        if ((e = cudaMemcpyAsync(q, q_host, q_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(k_new, k_new_host, kv_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(v_new, v_new_host, kv_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(block_table, block_table_host, bt_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(context_lens, context_lens_host, len_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess)
+            return fail_cuda(static_cast<int>(e));
+    }
     st = ac_decode_step_fused(q, nullptr, k_new, v_new, k_cache, v_cache, stride_page, stride_token,
                               stride_head, block_table, max_pages_per_seq, context_lens, rope_cos,
                               rope_sin, max_position, softmax_scale, num_splits, workspace,

@@ -90,6 +90,8 @@ cudaError_t launch_oproj_residual(const CUtensorMap& w_map, const CUtensorMap& x
                                   cudaStream_t stream);
 cudaError_t launch_rmsnorm_rows(const void* h, const void* weight, void* out, int B, int N, float eps,
                                 cudaStream_t stream);
+cudaError_t launch_stage_inputs(const void* const src[5], void* const dst[5], const size_t bytes[5],
+                                void* zero_dst, size_t zero_bytes, cudaStream_t stream);
 cudaError_t launch_splitkv_merge(const float* partial_o, const float* partial_lse, int num_splits,
                                  const int32_t* context_lens, void* out, int B, int Hq, int d,
                                  cudaStream_t stream);

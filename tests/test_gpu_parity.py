@@ -459,6 +459,42 @@ def test_batch_of_only_inactive_rows(rt, fused):
     assert (rt.bits_of(st.out) == 0).all()
 
 
+@pytest.mark.parametrize("kw,splits", [
+    (dict(B=4, Hq=8, Hkv=2, context_lens=[200, 37, 333, 0], num_pages=96), 3),     # gathered by one kernel
+    (dict(B=4, Hq=8, Hkv=2, context_lens=[200, 37, 333, 0], num_pages=96), 1),
+    (dict(B=3, Hq=8, Hkv=2, context_lens=[200, 37, 333], num_pages=96), 2),        # sizes not 16-byte multiples
+    (dict(B=1, Hq=8, Hkv=2, context_lens=[77], num_pages=16), 2),
+])
+def test_decode_step_from_host_buffers(rt, kw, splits):
+    import torch
+    from paper_2606_07665_b200 import binding as ac
+    w = small(57, **kw)
+    q_rot, k_after, v_after, out_ref = O.oracle_decode_step(w)
+    st = rt.DecodeStep(w, num_splits=splits)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+    h_q, h_k, h_v, h_bt, h_len = pin(w.q), pin(w.k_new), pin(w.v_new), pin(w.block_table), pin(w.context_lens)
+    h_out = torch.full((w.B, w.Hq, w.d), 0x7FC0, dtype=torch.int16).pin_memory()
+    # device staging buffers start with garbage: everything must come from the host buffers
+    for t in (st.q_in, st.k_new, st.v_new):
+        t.fill_(0x7FC0)
+    st.block_table.fill_(-7)
+    st.context_lens.fill_(-1)
+    st.workspace.view(torch.int32).fill_(123456)              # the call clears its own counters
+    for rep in range(2):
+        ac.ac_decode_step_host(h_q, h_k, h_v, h_bt, h_len, h_out, st.q_in, st.k_new, st.v_new, st.block_table,
+                               st.context_lens, st.out, st.k_cache, st.v_cache, st.stride_page, st.stride_token,
+                               st.stride_head, w.max_pages_per_seq, st.rope_cos, st.rope_sin, w.max_position,
+                               0.0, st.num_splits, st.workspace if st.num_splits > 1 else None,
+                               st.workspace_bytes, st.B, st.Hq, st.Hkv, st.d, st.ps, st.num_pages,
+                               st.max_context_len, st.status_flag)
+        torch.cuda.synchronize()
+        assert int(st.status_flag.item()) == 0
+        got = W.bf16_bits_to_f32(h_out.numpy().view(np.uint16)).astype(np.float64)
+        check_out(got, out_ref, f"host step rep {rep}")
+        k_gpu, v_gpu = st.cache_bits()
+        assert np.array_equal(k_gpu, k_after) and np.array_equal(v_gpu, v_after)
+
+
 def test_peaked_scores(rt):
     w = W.make_workload("peaked", 48, B=2, Hq=16, Hkv=2, d=128, page_size=16, num_pages=300,
                         context_lens=[2000, 1500], rope_base=500000.0, peak_fraction=0.01)
