@@ -576,56 +576,48 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     __syncthreads();
     if (!s_is_last) return;
     __threadfence();
-    // The rings are idle now (every warp passed the barriers above): stage the log-sum-exps of the
-    // G rows there so that each thread reads them from shared memory, then stream the partials with
-    // four independent 16-byte loads in flight per thread.
-    constexpr int LSE_CAPACITY = L::RING_BYTES / 4;
-    float* s_lse = reinterpret_cast<float*>(smem_gen);
-    const size_t hq0 = static_cast<size_t>(b) * p.Hq + h * G;
-    const bool staged = G * n_active <= LSE_CAPACITY;
-    if (staged) {
-        for (int i = threadIdx.x; i < G * n_active; i += THREADS) {
-            const int row = i / n_active;
-            s_lse[i] = __ldcg(p.partial_lse + (hq0 + row) * S + (i - row * n_active));
-        }
-        __syncthreads();
-    }
+    // Each thread owns four consecutive output elements of one query row and walks the splits in
+    // groups of sixteen: all loads of a group (sixteen 16-byte partial loads and their log-sum-exps)
+    // are issued before any is used, so a group costs one L2 round trip, and groups are combined with
+    // the same running-maximum rescaling as the main loop.
     constexpr int D4 = D / 4;
+    constexpr int GROUP = 16;
+    const size_t hq0 = static_cast<size_t>(b) * p.Hq + h * G;
     for (int e = threadIdx.x; e < G * D4; e += THREADS) {
         const int row = e / D4;
         const int c4 = e - row * D4;
         const float* lse_g = p.partial_lse + (hq0 + row) * S;
-        auto lse_at = [&](int sidx) { return staged ? s_lse[row * n_active + sidx] : __ldcg(lse_g + sidx); };
-        float M = -INFINITY;
-        for (int sidx = 0; sidx < n_active; ++sidx) M = fmaxf(M, lse_at(sidx));
         const float4* po = reinterpret_cast<const float4*>(p.partial_o + (hq0 + row) * S * D) + c4;
+        float M = -INFINITY, den = 0.0f;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        float den = 0.0f;
-        int sidx = 0;
-        for (; sidx + 4 <= n_active; sidx += 4) {
-            float4 v[4];
-            float wgt[4];
+        for (int s0 = 0; s0 < n_active; s0 += GROUP) {
+            float4 v[GROUP];
+            float l[GROUP];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = __ldcg(po + static_cast<size_t>(sidx + u) * D4);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) wgt[u] = __expf(lse_at(sidx + u) - M);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                acc.x = fmaf(wgt[u], v[u].x, acc.x);
-                acc.y = fmaf(wgt[u], v[u].y, acc.y);
-                acc.z = fmaf(wgt[u], v[u].z, acc.z);
-                acc.w = fmaf(wgt[u], v[u].w, acc.w);
-                den += wgt[u];
+            for (int u = 0; u < GROUP; ++u) {
+                const bool on = s0 + u < n_active;
+                l[u] = on ? __ldcg(lse_g + s0 + u) : -INFINITY;
+                v[u] = on ? __ldcg(po + static_cast<size_t>(s0 + u) * D4) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
-        }
-        for (; sidx < n_active; ++sidx) {
-            const float4 v = __ldcg(po + static_cast<size_t>(sidx) * D4);
-            const float wgt = __expf(lse_at(sidx) - M);
-            acc.x = fmaf(wgt, v.x, acc.x);
-            acc.y = fmaf(wgt, v.y, acc.y);
-            acc.z = fmaf(wgt, v.z, acc.z);
-            acc.w = fmaf(wgt, v.w, acc.w);
-            den += wgt;
+            float gm = M;
+#pragma unroll
+            for (int u = 0; u < GROUP; ++u) gm = fmaxf(gm, l[u]);
+            const float rescale = __expf(M - gm);              // 0 on the first group (M = -inf)
+            acc.x *= rescale;
+            acc.y *= rescale;
+            acc.z *= rescale;
+            acc.w *= rescale;
+            den *= rescale;
+            M = gm;
+#pragma unroll
+            for (int u = 0; u < GROUP; ++u) {
+                const float wgt = __expf(l[u] - M);            // 0 for the padding entries
+                acc.x = fmaf(wgt, v[u].x, acc.x);
+                acc.y = fmaf(wgt, v[u].y, acc.y);
+                acc.z = fmaf(wgt, v[u].z, acc.z);
+                acc.w = fmaf(wgt, v[u].w, acc.w);
+                den += wgt;
+            }
         }
         const float inv = 1.0f / den;
         *reinterpret_cast<uint2*>(p.out + (hq0 + row) * D + c4 * 4) =
