@@ -223,6 +223,25 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
         tma_load_5d(dst + L::K_BYTES, &v_map, bar, 0, slot, 0, h, page, policy);
     };
 
+    // Fused step: the rotary angles of this CTA's query rows depend only on ctx; fetch them now so
+    // that they are in registers when q itself can be read (after the dependency is met).
+    constexpr int QP = ROPE ? (16 * (D / 2) + THREADS - 1) / THREADS : 1;   // rotary pairs per thread
+    const bool rope_ok = ROPE && ctx < p.max_position;
+    float q_cos[QP], q_sin[QP];
+    if (ROPE) {
+        const float* cos_row = p.rope_cos + static_cast<size_t>(ctx) * (D / 2);
+        const float* sin_row = p.rope_sin + static_cast<size_t>(ctx) * (D / 2);
+#pragma unroll
+        for (int k = 0; k < QP; ++k) {
+            const int idx = threadIdx.x + k * THREADS;
+            const int row = idx / (D / 2);
+            const int i = idx - row * (D / 2);
+            const bool on = rope_ok && row < G;
+            q_cos[k] = on ? cos_row[i] : 1.0f;
+            q_sin[k] = on ? sin_row[i] : 0.0f;
+        }
+    }
+
     // ---- prologue: fill the ring -------------------------------------------------------------
     int issued = 0;
     bool dependency_met = false;
@@ -239,6 +258,19 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     }
     int page_next = issued < n_my ? load_page_id(issued) : 0;
     if (!dependency_met) cudaGridDependencySynchronize();      // q was written by the preceding kernel
+    uint16_t q_raw_lo[QP], q_raw_hi[QP];
+    if (ROPE) {
+        const uint16_t* qsrc = p.q + (static_cast<size_t>(b) * p.Hq + h * G) * D;
+#pragma unroll
+        for (int k = 0; k < QP; ++k) {
+            const int idx = threadIdx.x + k * THREADS;
+            const int row = idx / (D / 2);
+            const int i = idx - row * (D / 2);
+            const bool on = row < G;
+            q_raw_lo[k] = on ? qsrc[row * D + i] : static_cast<uint16_t>(0);
+            q_raw_hi[k] = on ? qsrc[row * D + i + D / 2] : static_cast<uint16_t>(0);
+        }
+    }
 
     // ---- fused step: rotate and append the new k/v early, under the latency of the first tiles ------
     constexpr int APPEND_PAIRS = D / 64;          // rotary pairs per lane (D/2 pairs over 32 lanes)
@@ -246,7 +278,6 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     uint2 v_new4 = make_uint2(0u, 0u);
     int append_j = -1;                            // index of this warp's tile that holds the new slot
     bool append_ok = false;
-    const bool rope_ok = ROPE && ctx < p.max_position;
     if (ROPE) {
         if (!rope_ok && threadIdx.x == 0 && p.status_flag != nullptr)
             atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
@@ -292,24 +323,22 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     if (ROPE) {
         // The CTA rotates its G query rows once (pair i with i + D/2, exact then rounded, as the
         // stand-alone kernel does) into shared memory; every warp then reads its fragments from there.
-        const uint16_t* qsrc = p.q + (static_cast<size_t>(b) * p.Hq + h * G) * D;
-        const float* cos_row = p.rope_cos + static_cast<size_t>(ctx) * (D / 2);
-        const float* sin_row = p.rope_sin + static_cast<size_t>(ctx) * (D / 2);
         uint16_t* qdst = (p.q_rot_out != nullptr && split == 0)
                              ? p.q_rot_out + (static_cast<size_t>(b) * p.Hq + h * G) * D : nullptr;
-        for (int idx = threadIdx.x; idx < 16 * (D / 2); idx += THREADS) {
+#pragma unroll
+        for (int k = 0; k < QP; ++k) {
+            const int idx = threadIdx.x + k * THREADS;
+            if (idx >= 16 * (D / 2)) break;
             const int row = idx / (D / 2);
             const int i = idx - row * (D / 2);
             uint16_t r0 = 0, r1 = 0;
             if (row < G) {
-                const uint16_t a = qsrc[row * D + i], bb = qsrc[row * D + i + D / 2];
                 if (rope_ok) {
-                    const float c = cos_row[i], sn = sin_row[i];
-                    r0 = rope_first_half(a, bb, c, sn);
-                    r1 = rope_second_half(a, bb, c, sn);
+                    r0 = rope_first_half(q_raw_lo[k], q_raw_hi[k], q_cos[k], q_sin[k]);
+                    r1 = rope_second_half(q_raw_lo[k], q_raw_hi[k], q_cos[k], q_sin[k]);
                 } else {
-                    r0 = a;
-                    r1 = bb;
+                    r0 = q_raw_lo[k];
+                    r1 = q_raw_hi[k];
                 }
                 if (qdst != nullptr && rope_ok) {
                     qdst[row * D + i] = r0;
