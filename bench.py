@@ -513,6 +513,11 @@ def run_ours(args):
     ac.ac_init(local)
     peak, peak_kind = measured_peak()
 
+    if args.prelude_only:
+        if rank == 0:
+            print(json.dumps({"prelude_fusion": time_prelude_fusion(torch, device, batches=(8,), replicas=4,
+                                                                   replays=3)}))
+        return
     w = W.NAMED[args.workload]()
     st = runner.DecodeStep(w, device=device, fused_step=not args.three_launches,
                            fused_merge=not args.separate_merge)
@@ -625,6 +630,9 @@ def main():
     ap.add_argument("--separate-merge", action="store_true",
                     help="with --three-launches: use ac_paged_decode_attn + ac_splitkv_merge (three "
                          "kernels) instead of the merge fused into the attention kernel")
+    ap.add_argument("--prelude-only", action="store_true",
+                    help="time only the projection fusions (ac_qkv_rope_kv_append, ac_oproj_residual_rmsnorm) "
+                         "at batch 8 and print their rows; used for profiling those kernels")
     ap.add_argument("--only-headline", action="store_true",
                     help="skip the other workloads and the CPU baseline")
     args = ap.parse_args()
