@@ -220,26 +220,35 @@ def aggregate_throughput(kv_bytes_per_rank, ms_slowest_rank, world):
 # ---------------------------------------------------------------------------------------------
 
 def time_headline(st, steps, warmup, torch):
-    """K steps back to back; CUDA events around the whole region and around each attention launch."""
+    """K steps back to back between one pair of CUDA events on the launching stream.
+
+    With the single-launch fused step the step IS the dominant kernel, so its average launch
+    duration is the bracketed time / K (no event is recorded between launches: an event node between
+    two kernels would undo the programmatic overlap of their tail and ramp).  With separate launches
+    an event pair around every attention launch gives that kernel's own duration.
+    """
     stream = torch.cuda.current_stream()
     for _ in range(warmup):
         st.step(stream)
     torch.cuda.synchronize()
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
     t0 = torch.cuda.Event(enable_timing=True)
     t1 = torch.cuda.Event(enable_timing=True)
+    if st.fused_step:
+        t0.record(stream)
+        for _ in range(steps):
+            st.decode_step_fused(stream)
+        t1.record(stream)
+        torch.cuda.synchronize()
+        per_step = t0.elapsed_time(t1) / steps
+        return per_step, per_step
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
     t0.record(stream)
     for i in range(steps):
-        if st.fused_step:                # one launch: RoPE + append + attention + merge
-            ev[i][0].record(stream)
-            st.decode_step_fused(stream)
-            ev[i][1].record(stream)
-        else:
-            st.rope_kv_append(stream)
-            ev[i][0].record(stream)
-            st.attention(stream)
-            ev[i][1].record(stream)
-            st.merge(stream)
+        st.rope_kv_append(stream)
+        ev[i][0].record(stream)
+        st.attention(stream)
+        ev[i][1].record(stream)
+        st.merge(stream)
     t1.record(stream)
     torch.cuda.synchronize()
     total_ms = t0.elapsed_time(t1)
