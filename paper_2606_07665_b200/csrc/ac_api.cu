@@ -362,7 +362,7 @@ int ac_oproj_residual_rmsnorm(const void* attn_out, const void* w_o, int K, int 
                               float norm_eps, void* normed_out, int B, void* stream) {
     if (!attn_out || !w_o || !residual_in || !residual_out || !norm_weight || !normed_out) return AC_ERR_NULL;
     if (B <= 0 || K <= 0 || N <= 0 || !(norm_eps >= 0.0f)) return AC_ERR_SHAPE;
-    if (K % 64 != 0 || N % 32 != 0 || B > 65535 * 8) return AC_ERR_UNSUPPORTED;
+    if (K % 64 != 0 || N % 32 != 0 || B > 65535) return AC_ERR_UNSUPPORTED;
     if (!aligned16(attn_out) || !aligned16(w_o) || !aligned16(residual_in) || !aligned16(residual_out) ||
         !aligned16(norm_weight) || !aligned16(normed_out))
         return AC_ERR_ALIGN;

@@ -353,19 +353,29 @@ cudaError_t launch_qkv_rope_kv_append(const CUtensorMap& w_map, const CUtensorMa
 // ---- RMSNorm of whole rows (second launch of the output-projection fusion) -------------------------
 namespace {
 
-// One CTA per row: sum of squares in fp64 (exact for bf16 inputs of moderate range), then
-// y = bf16(bf16(h / sqrt(mean + eps)) * w), the arithmetic of the per-head norm of the prelude.
+// NORM_SLICES CTAs per row: each recomputes the row's sum of squares in fp64 (exact for bf16 inputs
+// of moderate range, so every CTA gets the same value; the row is a few KB and sits in L2) and
+// normalises its own slice: y = bf16(bf16(h / sqrt(mean + eps)) * w), the arithmetic of the per-head
+// norm of the prelude.
+constexpr int NORM_SLICES = 8;
+
 __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const uint16_t* __restrict__ h,
                                                            const uint16_t* __restrict__ weight,
                                                            uint16_t* __restrict__ out, int N, float eps) {
     cudaTriggerProgrammaticLaunchCompletion();
     cudaGridDependencySynchronize();
     __shared__ double s_part[8];
-    const uint16_t* row = h + static_cast<size_t>(blockIdx.x) * N;
+    const uint16_t* row = h + static_cast<size_t>(blockIdx.y) * N;
     double ss = 0.0;
-    for (int i = threadIdx.x; i < N; i += 256) {
-        const double v = static_cast<double>(bf16_bits_to_float(row[i]));
-        ss = __dadd_rn(ss, __dmul_rn(v, v));
+    for (int i = threadIdx.x * 8; i < N; i += 256 * 8) {          // N % 32 == 0: 16-byte pieces
+        const uint4 v8 = *reinterpret_cast<const uint4*>(row + i);
+        const uint32_t w4[4] = {v8.x, v8.y, v8.z, v8.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const double lo = static_cast<double>(__uint_as_float(w4[e] << 16));
+            const double hi = static_cast<double>(__uint_as_float(w4[e] & 0xFFFF0000u));
+            ss = __dadd_rn(ss, __dadd_rn(__dmul_rn(lo, lo), __dmul_rn(hi, hi)));
+        }
     }
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1) ss = __dadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, off));
@@ -376,8 +386,11 @@ __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const uint16_t* __res
     for (int w = 0; w < 8; ++w) total = __dadd_rn(total, s_part[w]);
     const double r = __ddiv_rn(1.0, __dsqrt_rn(__dadd_rn(__ddiv_rn(total, static_cast<double>(N)),
                                                          static_cast<double>(eps))));
-    uint16_t* orow = out + static_cast<size_t>(blockIdx.x) * N;
-    for (int i = threadIdx.x; i < N; i += 256) {
+    uint16_t* orow = out + static_cast<size_t>(blockIdx.y) * N;
+    const int per = (N + NORM_SLICES - 1) / NORM_SLICES;
+    const int lo_i = blockIdx.x * per;
+    const int hi_i = min(N, lo_i + per);
+    for (int i = lo_i + threadIdx.x; i < hi_i; i += 256) {
         const double v = static_cast<double>(bf16_bits_to_float(row[i]));
         const uint16_t y1 = f64_to_bf16_rne(__dmul_rn(v, r));
         const double w = static_cast<double>(bf16_bits_to_float(weight[i]));
@@ -405,7 +418,7 @@ cudaError_t launch_oproj_residual(const CUtensorMap& w_map, const CUtensorMap& x
 cudaError_t launch_rmsnorm_rows(const void* h, const void* weight, void* out, int B, int N, float eps,
                                 cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(B);
+    cfg.gridDim = dim3(NORM_SLICES, B);
     cfg.blockDim = dim3(256);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
