@@ -339,7 +339,7 @@ def time_in_graph(make_step, kv_bytes, torch, replays=20):
     return us, info
 
 
-def time_prelude_fusion(torch, device, batches=(1, 8, 32), replicas=12, replays=20):
+def time_prelude_fusion(torch, device, batches=(1, 8, 32, 128, 256), replicas=12, replays=20):
     """Attention-prelude fusion (QKV projection + RoPE + KV append, one launch) on an 8B-class layer:
     hidden 4096, 32 query / 8 KV heads, head_dim 128 -> 6144 x 4096 bf16 weights (50.3 MB), streamed
     from HBM once per call.  `replicas` separate copies of the weights are cycled inside one captured

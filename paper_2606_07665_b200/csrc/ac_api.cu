@@ -24,6 +24,9 @@ struct Shape {
     int B, Hq, Hkv, d, page_size, num_pages;
 };
 
+// Largest batch the warp-MMA projection kernels take; beyond it the tcgen05 kernels are used.
+constexpr int kWarpMmaMaxBatch = 32;
+
 int check_shape(const Shape& s) {
     if (s.B <= 0 || s.Hq <= 0 || s.Hkv <= 0 || s.d <= 0 || s.page_size <= 0 || s.num_pages <= 0)
         return AC_ERR_SHAPE;
@@ -134,6 +137,7 @@ int ac_init(int device) {
         }
         e = attn_set_attributes(st.smem_optin);
         if (e == cudaSuccess) e = qkv_set_attributes(st.smem_optin);
+        if (e == cudaSuccess) e = proj_tc_set_attributes(st.smem_optin);
         if (e != cudaSuccess) {
             status = fail_cuda(static_cast<int>(e));
             break;
@@ -326,6 +330,33 @@ int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out, 
     // x [B, H] as (64 elements, batch row, 64-element K block).
     const cuuint64_t row_bytes = static_cast<cuuint64_t>(H) * 2;
     CUtensorMap w_map, x_map;
+    if (B > kWarpMmaMaxBatch) {
+        // Batched decode: 128-row batch tiles on the tcgen05 path (boxes of 32 pairs x one K block).
+        cuuint64_t wdims[5] = {64, static_cast<cuuint64_t>(d / 2), 2, static_cast<cuuint64_t>(Hq + 2 * Hkv),
+                               static_cast<cuuint64_t>(H / 64)};
+        cuuint64_t wstrides[4] = {row_bytes, row_bytes * (d / 2), row_bytes * d, 128};
+        cuuint32_t wbox[5] = {64, 32, 2, 1, 2};
+        cuuint32_t es5[5] = {1, 1, 1, 1, 1};
+        CUresult r = g_encode_tiled(&w_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(w_qkv),
+                                    wdims, wstrides, wbox, es5, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
+        cuuint64_t xdims[3] = {64, static_cast<cuuint64_t>(B), static_cast<cuuint64_t>(H / 64)};
+        cuuint64_t xstrides[2] = {row_bytes, 128};
+        cuuint32_t xbox[3] = {64, 128, 2};
+        cuuint32_t es3[3] = {1, 1, 1};
+        r = g_encode_tiled(&x_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), xdims, xstrides,
+                           xbox, es3, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
+        cudaError_t e = launch_qkv_rope_kv_append_tc(w_map, x_map, q_out, k_cache, v_cache, stride_page,
+                                                     stride_token, stride_head, block_table,
+                                                     max_pages_per_seq, context_lens, rope_cos, rope_sin,
+                                                     max_position, B, H, Hq, Hkv, d, page_size, num_pages,
+                                                     status_flag, static_cast<cudaStream_t>(stream));
+        return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
+    }
     {
         cuuint64_t dims[5] = {64, static_cast<cuuint64_t>(d / 2), 2, static_cast<cuuint64_t>(Hq + 2 * Hkv),
                               static_cast<cuuint64_t>(H / 64)};
@@ -373,6 +404,30 @@ int ac_oproj_residual_rmsnorm(const void* attn_out, const void* w_o, int K, int 
     // attn_out [B, K] as (64 elements, batch row, 64-element K block).
     const cuuint64_t row_bytes = static_cast<cuuint64_t>(K) * 2;
     CUtensorMap w_map, x_map;
+    cudaStream_t cs_tc = static_cast<cudaStream_t>(stream);
+    if (B > kWarpMmaMaxBatch && N % 64 == 0) {
+        cuuint64_t wdims[5] = {64, 32, 2, static_cast<cuuint64_t>(N / 64), static_cast<cuuint64_t>(K / 64)};
+        cuuint64_t wstrides[4] = {row_bytes, row_bytes * 32, row_bytes * 64, 128};
+        cuuint32_t wbox[5] = {64, 32, 2, 1, 2};
+        cuuint32_t es5[5] = {1, 1, 1, 1, 1};
+        CUresult r = g_encode_tiled(&w_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(w_o), wdims,
+                                    wstrides, wbox, es5, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
+        cuuint64_t xdims[3] = {64, static_cast<cuuint64_t>(B), static_cast<cuuint64_t>(K / 64)};
+        cuuint64_t xstrides[2] = {row_bytes, 128};
+        cuuint32_t xbox[3] = {64, 128, 2};
+        cuuint32_t es3[3] = {1, 1, 1};
+        r = g_encode_tiled(&x_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(attn_out), xdims,
+                           xstrides, xbox, es3, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
+        cudaError_t e = launch_oproj_residual_tc(w_map, x_map, residual_in, residual_out, B, K, N, cs_tc);
+        if (e != cudaSuccess) return fail_cuda(static_cast<int>(e));
+        e = launch_rmsnorm_rows(residual_out, norm_weight, normed_out, B, N, norm_eps, cs_tc);
+        return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
+    }
     {
         cuuint64_t dims[5] = {64, 16, 2, static_cast<cuuint64_t>(N / 32), static_cast<cuuint64_t>(K / 64)};
         cuuint64_t strides[4] = {row_bytes, row_bytes * 16, row_bytes * 32, 128};

@@ -90,6 +90,18 @@ cudaError_t launch_oproj_residual(const CUtensorMap& w_map, const CUtensorMap& x
                                   cudaStream_t stream);
 cudaError_t launch_rmsnorm_rows(const void* h, const void* weight, void* out, int B, int N, float eps,
                                 cudaStream_t stream);
+cudaError_t proj_tc_set_attributes(int smem_optin);
+cudaError_t launch_qkv_rope_kv_append_tc(const CUtensorMap& w_map, const CUtensorMap& x_map, void* q_out,
+                                         void* k_cache, void* v_cache, int64_t stride_page,
+                                         int64_t stride_token, int64_t stride_head,
+                                         const int32_t* block_table, int max_pages_per_seq,
+                                         const int32_t* context_lens, const float* rope_cos,
+                                         const float* rope_sin, int max_position, int B, int K, int Hq,
+                                         int Hkv, int d, int page_size, int num_pages,
+                                         int32_t* status_flag, cudaStream_t stream);
+cudaError_t launch_oproj_residual_tc(const CUtensorMap& w_map, const CUtensorMap& x_map,
+                                     const void* residual_in, void* residual_out, int B, int K, int N,
+                                     cudaStream_t stream);
 cudaError_t launch_stage_inputs(const void* const src[5], void* const dst[5], const size_t bytes[5],
                                 void* zero_dst, size_t zero_bytes, cudaStream_t stream);
 cudaError_t launch_splitkv_merge(const float* partial_o, const float* partial_lse, int num_splits,

@@ -35,6 +35,11 @@ def _close_bf16(got_bits, ref_bits, what):
     (31, 768, 8, 2, 128, 16),         # batch tile of 32
     (40, 256, 4, 2, 64, 16),          # two batch tiles
     (4, 4096, 32, 8, 128, 16),        # 8B-class layer: 6144 x 4096 weights
+    (33, 256, 4, 2, 128, 16),         # smallest batch on the tcgen05 path; rows 33..127 of the tile are padding
+    (100, 512, 8, 2, 64, 16),
+    (128, 1024, 8, 2, 128, 32),       # exactly one 128-row tile
+    (200, 320, 4, 4, 128, 16),        # two tiles, K not a multiple of the stage count
+    (64, 4096, 32, 8, 128, 16),       # 8B-class layer, batched
 ])
 def test_qkv_prelude_matches_oracle(B, H, Hq, Hkv, d, ps):
     import torch
@@ -85,7 +90,8 @@ def test_qkv_prelude_matches_oracle(B, H, Hq, Hkv, d, ps):
 
 
 @pytest.mark.parametrize("B,K,N", [(1, 256, 64), (5, 320, 96), (8, 1024, 512), (13, 512, 256), (31, 768, 128),
-                                   (40, 256, 64), (4, 4096, 4096)])
+                                   (40, 256, 64), (4, 4096, 4096), (33, 128, 64), (100, 512, 192), (128, 1024, 256),
+                                   (200, 320, 128), (40, 256, 96), (64, 4096, 4096)])
 def test_oproj_residual_rmsnorm_matches_oracle(B, K, N):
     import torch
     from paper_2606_07665_b200 import binding as ac
@@ -109,7 +115,9 @@ def test_oproj_residual_rmsnorm_matches_oracle(B, K, N):
     y = runner.bits_of(y_d)
     hf, hr = W.bf16_bits_to_f32(h).astype(np.float64), W.bf16_bits_to_f32(h_ref).astype(np.float64)
     assert np.isfinite(hf).all()
-    assert (np.abs(hf - hr) <= 2.0 ** -7 * np.abs(hr) + 1e-30).all()        # at most one bf16 step
+    # at most one bf16 step; where residual and projection cancel, the fp32 accumulation error of
+    # the projection (relative to ITS magnitude, ~1) shows in the small sum
+    assert (np.abs(hf - hr) <= 2.0 ** -7 * np.abs(hr) + 3e-5).all()
     assert np.mean(h == h_ref) >= 0.97
     # the norm is exact given the h the kernel produced
     assert np.array_equal(y, O.rms_norm_bf16(h, nw, 1e-5))
