@@ -524,7 +524,8 @@ def run_ours(args):
 
     if args.prelude_only:
         if rank == 0:
-            print(json.dumps({"prelude_fusion": time_prelude_fusion(torch, device, batches=(8,), replicas=4,
+            print(json.dumps({"prelude_fusion": time_prelude_fusion(torch, device, batches=(args.prelude_batch,),
+                                                                   replicas=4,
                                                                    replays=3)}))
         return
     w = W.NAMED[args.workload]()
@@ -639,6 +640,8 @@ def main():
     ap.add_argument("--separate-merge", action="store_true",
                     help="with --three-launches: use ac_paged_decode_attn + ac_splitkv_merge (three "
                          "kernels) instead of the merge fused into the attention kernel")
+    ap.add_argument("--prelude-batch", type=int, default=8,
+                    help="batch rows for --prelude-only (above 32 the tcgen05 projection kernel runs)")
     ap.add_argument("--prelude-only", action="store_true",
                     help="time only the projection fusions (ac_qkv_rope_kv_append, ac_oproj_residual_rmsnorm) "
                          "at batch 8 and print their rows; used for profiling those kernels")

@@ -2,6 +2,8 @@
 #include <math.h>
 #include <stdlib.h>
 
+#include <mutex>
+
 #include "ac_internal.h"
 
 namespace ac {
@@ -9,6 +11,7 @@ namespace ac {
 namespace {
 
 DeviceState g_devices[kMaxDevices];
+std::mutex g_init_mutex;                 // ac_init may be called from one host thread per device
 thread_local int t_last_cuda_error = 0;
 int g_last_sm_count = 0;
 
@@ -104,6 +107,7 @@ int ac_init(int device) {
         if (e != cudaSuccess) return fail_cuda(static_cast<int>(e));
     }
     if (device >= kMaxDevices) return AC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_init_mutex);
     int prev = -1;
     e = cudaGetDevice(&prev);
     if (e != cudaSuccess) return fail_cuda(static_cast<int>(e));

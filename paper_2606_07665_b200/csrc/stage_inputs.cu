@@ -36,8 +36,8 @@ __global__ void __launch_bounds__(256) stage_inputs_kernel(const StageList list)
 
 // All sizes in bytes and multiples of 16 except the last piece of each buffer, which the caller
 // rounds up (device buffers from cudaMalloc-class allocators are padded well beyond 16 bytes; host
-// sizes are checked by the caller).  Returns cudaErrorInvalidValue when a source is not
-// device-addressable host memory or a size is not a multiple of 16.
+// sizes are checked by the caller).  Returns cudaErrorInvalidValue, having launched nothing, when a
+// source is not device-addressable host memory or a size or address is not a multiple of 16.
 cudaError_t launch_stage_inputs(const void* const src[5], void* const dst[5], const size_t bytes[5],
                                 void* zero_dst, size_t zero_bytes, cudaStream_t stream) {
     StageList list;
@@ -51,12 +51,14 @@ cudaError_t launch_stage_inputs(const void* const src[5], void* const dst[5], co
             return cudaErrorInvalidValue;
         }
         if (attr.type != cudaMemoryTypeHost || attr.devicePointer == nullptr) return cudaErrorInvalidValue;
+        if ((reinterpret_cast<uintptr_t>(attr.devicePointer) | reinterpret_cast<uintptr_t>(dst[b])) & 15u)
+            return cudaErrorInvalidValue;                 // the kernel moves 16-byte pieces
         list.src[b] = static_cast<const uint4*>(attr.devicePointer);
         list.dst[b] = static_cast<uint4*>(dst[b]);
         list.chunks[b] = bytes[b] / 16;
         total += list.chunks[b];
     }
-    if (zero_bytes % 16 != 0) return cudaErrorInvalidValue;
+    if (zero_bytes % 16 != 0 || (reinterpret_cast<uintptr_t>(zero_dst) & 15u)) return cudaErrorInvalidValue;
     list.zero_dst = static_cast<uint4*>(zero_dst);
     list.zero_chunks = zero_dst != nullptr ? zero_bytes / 16 : 0;
     total += list.zero_chunks;
