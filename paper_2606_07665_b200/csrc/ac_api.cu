@@ -348,7 +348,7 @@ int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out, 
         if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
         cuuint64_t xdims[3] = {64, static_cast<cuuint64_t>(B), static_cast<cuuint64_t>(H / 64)};
         cuuint64_t xstrides[2] = {row_bytes, 128};
-        cuuint32_t xbox[3] = {64, 128, 2};
+        cuuint32_t xbox[3] = {64, static_cast<cuuint32_t>(proj_tc_batch_rows(B)), 2};
         cuuint32_t es3[3] = {1, 1, 1};
         r = g_encode_tiled(&x_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), xdims, xstrides,
                            xbox, es3, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -421,7 +421,7 @@ int ac_oproj_residual_rmsnorm(const void* attn_out, const void* w_o, int K, int 
         if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
         cuuint64_t xdims[3] = {64, static_cast<cuuint64_t>(B), static_cast<cuuint64_t>(K / 64)};
         cuuint64_t xstrides[2] = {row_bytes, 128};
-        cuuint32_t xbox[3] = {64, 128, 2};
+        cuuint32_t xbox[3] = {64, static_cast<cuuint32_t>(proj_tc_batch_rows(B)), 2};
         cuuint32_t es3[3] = {1, 1, 1};
         r = g_encode_tiled(&x_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(attn_out), xdims,
                            xstrides, xbox, es3, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,

@@ -91,6 +91,7 @@ cudaError_t launch_oproj_residual(const CUtensorMap& w_map, const CUtensorMap& x
 cudaError_t launch_rmsnorm_rows(const void* h, const void* weight, void* out, int B, int N, float eps,
                                 cudaStream_t stream);
 cudaError_t proj_tc_set_attributes(int smem_optin);
+int proj_tc_batch_rows(int B);          // rows of the x box the tcgen05 kernels expect for batch B
 cudaError_t launch_qkv_rope_kv_append_tc(const CUtensorMap& w_map, const CUtensorMap& x_map, void* q_out,
                                          void* k_cache, void* v_cache, int64_t stride_page,
                                          int64_t stride_token, int64_t stride_head,

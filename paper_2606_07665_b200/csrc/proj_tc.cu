@@ -31,18 +31,16 @@ using namespace acdev;
 enum { TC_EPI_QKV_ROPE_APPEND = 0, TC_EPI_RESIDUAL_ADD = 1 };
 
 constexpr int TC_THREADS = 192;
-constexpr int TC_M = 128;                       // batch rows per CTA
+constexpr int TC_M = 128;                       // rows of the MMA tile: batch rows per CTA, at most
 constexpr int TC_N = 64;                        // output features per CTA
 constexpr int TC_KBLK = 2;                      // 64-element (128-byte) K blocks per stage
 constexpr int TC_KC = 64 * TC_KBLK;             // K elements per stage
-constexpr int TC_STAGES = 4;
-constexpr int TC_A_BLOCK = TC_M * 128;          // one swizzled [128 rows x 128 B] block of x: 16 KB
+constexpr int TC_MAX_STAGES = 12;
+constexpr int TC_RING_BYTES = 216 * 1024;       // holds as many stages as fit: 4 at 128 batch rows, 8 at 40
 constexpr int TC_B_BLOCK = TC_N * 128;          // one swizzled [64 rows x 128 B] block of W: 8 KB
-constexpr int TC_A_BYTES = TC_KBLK * TC_A_BLOCK;
 constexpr int TC_B_BYTES = TC_KBLK * TC_B_BLOCK;
-constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
-constexpr int TC_BAR_OFFSET = TC_STAGES * TC_STAGE_BYTES;
-constexpr int TC_SMEM_TOTAL = TC_BAR_OFFSET + (2 * TC_STAGES + 1) * 8 + 16 + 1024;
+constexpr int TC_BAR_OFFSET = TC_RING_BYTES;
+constexpr int TC_SMEM_TOTAL = TC_BAR_OFFSET + (2 * TC_MAX_STAGES + 1) * 8 + 16 + 1024;
 constexpr uint32_t TC_TMEM_COLS = 64;
 
 struct TcParams {
@@ -57,6 +55,7 @@ struct TcParams {
     int32_t* status_flag;
     int max_pages_per_seq, max_position, num_pages, page_size;
     int B, K, Hq, Hkv, d;
+    int x_rows;                   // batch rows a CTA loads and owns: a multiple of 8, at most TC_M
     const uint16_t* residual_in;
     uint16_t* residual_out;
     int N;
@@ -132,6 +131,14 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
         : "memory");
 }
 
+// 32 lanes x 8 consecutive 32-bit columns.
+__device__ __forceinline__ void tmem_ld_32x8(uint32_t taddr, uint32_t (&r)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+}
+
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 template <int EPI>
@@ -143,15 +150,23 @@ __global__ void __launch_bounds__(TC_THREADS, 1) proj_tc_kernel(const __grid_con
     const uint32_t smem_base = (smem_addr(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_addr(smem_raw));
     const uint32_t full_bar = smem_base + TC_BAR_OFFSET;
-    const uint32_t empty_bar = full_bar + TC_STAGES * 8;
-    const uint32_t done_bar = empty_bar + TC_STAGES * 8;
+    const uint32_t empty_bar = full_bar + TC_MAX_STAGES * 8;
+    const uint32_t done_bar = empty_bar + TC_MAX_STAGES * 8;
     const uint32_t tmem_slot = done_bar + 8;                       // 4 bytes: TMEM base address
     volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + TC_BAR_OFFSET +
-                                                                            (2 * TC_STAGES + 1) * 8);
+                                                                            (2 * TC_MAX_STAGES + 1) * 8);
 
     const int blk = blockIdx.x;          // block of 32 pairs inside the head (QKV) / unused (o_proj)
     const int hh = blockIdx.y;           // head slot (QKV) / block of 64 output features (o_proj)
-    const int b0 = blockIdx.z * TC_M;
+    // The x box holds x_rows rows per 64-element block; the MMA always reads 128.  Rows past x_rows are
+    // whatever the ring holds: every accumulator row depends on its own x row only, and the epilogue
+    // skips them.  A stage is the x tile followed by the W tile.  The weights come from DRAM with
+    // microseconds of latency, so the ring is as deep as shared memory allows.
+    const int b0 = blockIdx.z * p.x_rows;
+    const uint32_t a_block = static_cast<uint32_t>(p.x_rows) * 128u;
+    const uint32_t a_bytes = TC_KBLK * a_block;
+    const uint32_t stage_bytes = a_bytes + TC_B_BYTES;       // a multiple of 1024
+    const int stages = min(TC_MAX_STAGES, TC_RING_BYTES / static_cast<int>(stage_bytes));
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int n_chunks = (p.K + TC_KC - 1) / TC_KC;
@@ -159,7 +174,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) proj_tc_kernel(const __grid_con
     if (threadIdx.x == 0) {
         tma_prefetch_descriptor(&w_map);
         tma_prefetch_descriptor(&x_map);
-        for (int s = 0; s < TC_STAGES; ++s) {
+        for (int s = 0; s < TC_MAX_STAGES; ++s) {
             mbar_init(full_bar + s * 8, 1);
             mbar_init(empty_bar + s * 8, 1);
         }
@@ -178,44 +193,54 @@ __global__ void __launch_bounds__(TC_THREADS, 1) proj_tc_kernel(const __grid_con
         if (lane == 0) {
             const uint64_t stream_once = l2_policy_evict_first();
             const uint64_t keep = l2_policy_evict_last();
+            int stage = 0;
+            uint32_t round = 0;                              // how often the ring has wrapped
             for (int c = 0; c < n_chunks; ++c) {
-                const int stage = c % TC_STAGES;
-                if (c >= TC_STAGES && !mbar_wait_bounded(empty_bar + stage * 8, ((c / TC_STAGES) - 1) & 1)) {
+                if (round > 0 && !mbar_wait_bounded(empty_bar + stage * 8, (round - 1) & 1)) {
                     timed_out = true;
                     break;
                 }
-                const uint32_t dst = smem_base + stage * TC_STAGE_BYTES;
-                mbar_arrive_expect_tx(full_bar + stage * 8, TC_STAGE_BYTES);
+                const uint32_t dst = smem_base + stage * stage_bytes;
+                mbar_arrive_expect_tx(full_bar + stage * 8, stage_bytes);
                 tma_load_3d(dst, &x_map, full_bar + stage * 8, 0, b0, c * TC_KBLK, keep);
                 if (EPI == TC_EPI_QKV_ROPE_APPEND)
-                    tma_load_5d(dst + TC_A_BYTES, &w_map, full_bar + stage * 8, 0, 32 * blk, 0, hh, c * TC_KBLK,
+                    tma_load_5d(dst + a_bytes, &w_map, full_bar + stage * 8, 0, 32 * blk, 0, hh, c * TC_KBLK,
                                 stream_once);
                 else
-                    tma_load_5d(dst + TC_A_BYTES, &w_map, full_bar + stage * 8, 0, 0, 0, hh, c * TC_KBLK,
+                    tma_load_5d(dst + a_bytes, &w_map, full_bar + stage * 8, 0, 0, 0, hh, c * TC_KBLK,
                                 stream_once);
+                if (++stage == stages) {
+                    stage = 0;
+                    ++round;
+                }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16_m128_n64();
+            int stage = 0;
+            uint32_t round = 0;
             for (int c = 0; c < n_chunks; ++c) {
-                const int stage = c % TC_STAGES;
-                if (!mbar_wait_bounded(full_bar + stage * 8, (c / TC_STAGES) & 1)) {
+                if (!mbar_wait_bounded(full_bar + stage * 8, round & 1)) {
                     timed_out = true;
                     break;
                 }
                 tc_fence_after_sync();
-                const uint32_t a_addr = smem_base + stage * TC_STAGE_BYTES;
+                const uint32_t a_addr = smem_base + stage * stage_bytes;
 #pragma unroll
                 for (int kb = 0; kb < TC_KBLK; ++kb) {
-                    const uint64_t adesc = umma_desc_k_major_sw128(a_addr + kb * TC_A_BLOCK);
-                    const uint64_t bdesc = umma_desc_k_major_sw128(a_addr + TC_A_BYTES + kb * TC_B_BLOCK);
+                    const uint64_t adesc = umma_desc_k_major_sw128(a_addr + kb * a_block);
+                    const uint64_t bdesc = umma_desc_k_major_sw128(a_addr + a_bytes + kb * TC_B_BLOCK);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)           // 16 elements = 32 bytes = 2 descriptor units
                         umma_bf16(tmem_d, adesc + 2 * ks, bdesc + 2 * ks, idesc,
                                   (c > 0 || kb > 0 || ks > 0) ? 1u : 0u);
                 }
                 umma_commit(empty_bar + stage * 8);          // the stage is free once these MMAs have read it
+                if (++stage == stages) {
+                    stage = 0;
+                    ++round;
+                }
             }
             umma_commit(done_bar);                           // accumulator complete (or as far as we got)
         }
@@ -224,25 +249,88 @@ __global__ void __launch_bounds__(TC_THREADS, 1) proj_tc_kernel(const __grid_con
 
     if (warp >= 2) {
         // ---- epilogue: thread = batch row, 64 accumulator columns -------------------------------------
-        const bool ready = mbar_wait_bounded(done_bar, 0);
-        if (!ready && lane == 0 && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_WAIT_TIMEOUT);
-        tc_fence_after_sync();
+        // Everything that does not need the accumulator is done first, under the main loop: the row's
+        // position, its destination and (QKV) its rotary angles.
         const int quarter = warp & 3;                        // TMEM lanes this warp may read
         const int row = quarter * 32 + lane;
         const int b = b0 + row;
-        uint32_t lo_bits[32], hi_bits[32];
-        tmem_ld_32x32(tmem_d + (static_cast<uint32_t>(quarter * 32) << 16), lo_bits);        // columns 0-31
-        tmem_ld_32x32(tmem_d + (static_cast<uint32_t>(quarter * 32) << 16) + 32, hi_bits);   // columns 32-63
-        tmem_ld_wait();
-        if (ready && b < p.B) {
-            if (EPI == TC_EPI_RESIDUAL_ADD) {
+        bool ok = row < p.x_rows && b < p.B;
+        uint16_t* dst = nullptr;
+        const uint16_t* res = nullptr;
+        bool rotate = false;
+        const float* cos_row = nullptr;                      // angles of this row's 32 pairs (QKV, q and k heads)
+        const float* sin_row = nullptr;
+        float c_nxt[8], s_nxt[8];                            // angles of the next group of 8 pairs
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            c_nxt[e] = 1.0f;
+            s_nxt[e] = 0.0f;
+        }
+        const int i0 = 32 * blk;                             // first pair of this CTA (QKV)
+        if (EPI == TC_EPI_RESIDUAL_ADD) {
+            if (ok) {
                 const size_t idx = static_cast<size_t>(b) * p.N + 64 * hh;
+                dst = p.residual_out + idx;
+                res = p.residual_in + idx;
+            }
+        } else if (ok) {
+            const int ctx = p.context_lens[b];
+            const int d = p.d, half_d = d / 2;
+            int page_idx = 0;
+            ok = ctx >= 0;
+            if (ok) {
+                page_idx = ctx / p.page_size;
+                if (ctx >= p.max_position || page_idx >= p.max_pages_per_seq) {
+                    if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
+                    ok = false;
+                }
+            }
+            rotate = hh < p.Hq + p.Hkv;
+            if (ok) {
+                if (hh < p.Hq) {
+                    dst = p.q_out + (static_cast<size_t>(b) * p.Hq + hh) * d;
+                } else {
+                    const int page = p.block_table[static_cast<size_t>(b) * p.max_pages_per_seq + page_idx];
+                    if (page < 0 || page >= p.num_pages) {
+                        if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
+                        ok = false;
+                    } else {
+                        const bool is_k = hh < p.Hq + p.Hkv;
+                        const int h = is_k ? hh - p.Hq : hh - p.Hq - p.Hkv;
+                        dst = (is_k ? p.k_cache : p.v_cache) + static_cast<size_t>(page) * p.stride_page +
+                              static_cast<size_t>(ctx - page_idx * p.page_size) * p.stride_token +
+                              static_cast<size_t>(h) * p.stride_head;
+                    }
+                }
+            }
+            if (ok && rotate) {
+                cos_row = p.rope_cos + static_cast<size_t>(ctx) * half_d + i0;
+                sin_row = p.rope_sin + static_cast<size_t>(ctx) * half_d + i0;
+                const float4 ca = *reinterpret_cast<const float4*>(cos_row), cb = *reinterpret_cast<const float4*>(cos_row + 4);
+                const float4 sa = *reinterpret_cast<const float4*>(sin_row), sb = *reinterpret_cast<const float4*>(sin_row + 4);
+                c_nxt[0] = ca.x; c_nxt[1] = ca.y; c_nxt[2] = ca.z; c_nxt[3] = ca.w;
+                c_nxt[4] = cb.x; c_nxt[5] = cb.y; c_nxt[6] = cb.z; c_nxt[7] = cb.w;
+                s_nxt[0] = sa.x; s_nxt[1] = sa.y; s_nxt[2] = sa.z; s_nxt[3] = sa.w;
+                s_nxt[4] = sb.x; s_nxt[5] = sb.y; s_nxt[6] = sb.z; s_nxt[7] = sb.w;
+            }
+        }
+
+        const bool ready = mbar_wait_bounded(done_bar, 0);
+        if (!ready && lane == 0 && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_WAIT_TIMEOUT);
+        tc_fence_after_sync();
+        const uint32_t lane_base = tmem_d + (static_cast<uint32_t>(quarter * 32) << 16);
+        if (EPI == TC_EPI_RESIDUAL_ADD) {
+            uint32_t lo_bits[32], hi_bits[32];
+            tmem_ld_32x32(lane_base, lo_bits);               // columns 0-31
+            tmem_ld_32x32(lane_base + 32, hi_bits);          // columns 32-63
+            tmem_ld_wait();
+            if (ready && ok) {
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     const uint32_t* acc = half == 0 ? lo_bits : hi_bits;
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {            // 8 features = 16 bytes at a time
-                        const uint4 r8 = *reinterpret_cast<const uint4*>(p.residual_in + idx + half * 32 + v * 8);
+                        const uint4 r8 = *reinterpret_cast<const uint4*>(res + half * 32 + v * 8);
                         const uint32_t rw[4] = {r8.x, r8.y, r8.z, r8.w};
                         uint32_t ow[4];
 #pragma unroll
@@ -252,79 +340,78 @@ __global__ void __launch_bounds__(TC_THREADS, 1) proj_tc_kernel(const __grid_con
                             ow[e] = pack_bf16x2(r0 + __uint_as_float(acc[v * 8 + 2 * e]),
                                                 r1 + __uint_as_float(acc[v * 8 + 2 * e + 1]));
                         }
-                        *reinterpret_cast<uint4*>(p.residual_out + idx + half * 32 + v * 8) =
-                            make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                        *reinterpret_cast<uint4*>(dst + half * 32 + v * 8) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
                     }
                 }
-            } else {
-                const int ctx = p.context_lens[b];
-                const int d = p.d, half_d = d / 2;
-                const int i0 = 32 * blk;                     // first pair of this CTA
-                bool ok = ctx >= 0;
-                int page_idx = 0;
-                if (ok) {
-                    page_idx = ctx / p.page_size;
-                    if (ctx >= p.max_position || page_idx >= p.max_pages_per_seq) {
-                        if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
-                        ok = false;
-                    }
-                }
-                uint16_t* dst = nullptr;
-                const bool rotate = hh < p.Hq + p.Hkv;
-                if (ok) {
-                    if (hh < p.Hq) {
-                        dst = p.q_out + (static_cast<size_t>(b) * p.Hq + hh) * d;
-                    } else {
-                        const int page = p.block_table[static_cast<size_t>(b) * p.max_pages_per_seq + page_idx];
-                        if (page < 0 || page >= p.num_pages) {
-                            if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
-                            ok = false;
-                        } else {
-                            const bool is_k = hh < p.Hq + p.Hkv;
-                            const int h = is_k ? hh - p.Hq : hh - p.Hq - p.Hkv;
-                            dst = (is_k ? p.k_cache : p.v_cache) + static_cast<size_t>(page) * p.stride_page +
-                                  static_cast<size_t>(ctx - page_idx * p.page_size) * p.stride_token +
-                                  static_cast<size_t>(h) * p.stride_head;
-                        }
-                    }
-                }
-                if (ok) {
-                    const float* cos_row = p.rope_cos + static_cast<size_t>(ctx) * half_d + i0;
-                    const float* sin_row = p.rope_sin + static_cast<size_t>(ctx) * half_d + i0;
+            }
+        } else {
+            // Four groups of 8 pairs in a rolled loop (the rotation code is long; unrolled 32 times it
+            // would not stay in the instruction cache); the next group's angles are fetched a group ahead.
+            const int half_d = p.d / 2;
+#pragma unroll 1
+            for (int v = 0; v < 4; ++v) {
+                uint32_t lo[8], hi[8];
+                tmem_ld_32x8(lane_base + v * 8, lo);         // first halves of pairs 8 v .. 8 v + 7
+                tmem_ld_32x8(lane_base + 32 + v * 8, hi);    // their second halves
+                float c_cur[8], s_cur[8];
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {            // 8 pairs at a time
-                        uint16_t lo8[8], hi8[8];
-                        float c8[8], s8[8];
-                        if (rotate) {
-                            const float4 ca = *reinterpret_cast<const float4*>(cos_row + v * 8);
-                            const float4 cb = *reinterpret_cast<const float4*>(cos_row + v * 8 + 4);
-                            const float4 sa = *reinterpret_cast<const float4*>(sin_row + v * 8);
-                            const float4 sb = *reinterpret_cast<const float4*>(sin_row + v * 8 + 4);
-                            c8[0] = ca.x; c8[1] = ca.y; c8[2] = ca.z; c8[3] = ca.w;
-                            c8[4] = cb.x; c8[5] = cb.y; c8[6] = cb.z; c8[7] = cb.w;
-                            s8[0] = sa.x; s8[1] = sa.y; s8[2] = sa.z; s8[3] = sa.w;
-                            s8[4] = sb.x; s8[5] = sb.y; s8[6] = sb.z; s8[7] = sb.w;
-                        }
+                for (int e = 0; e < 8; ++e) {
+                    c_cur[e] = c_nxt[e];
+                    s_cur[e] = s_nxt[e];
+                }
+                if (cos_row != nullptr && v < 3) {
+                    const float4 ca = *reinterpret_cast<const float4*>(cos_row + (v + 1) * 8);
+                    const float4 cb = *reinterpret_cast<const float4*>(cos_row + (v + 1) * 8 + 4);
+                    const float4 sa = *reinterpret_cast<const float4*>(sin_row + (v + 1) * 8);
+                    const float4 sb = *reinterpret_cast<const float4*>(sin_row + (v + 1) * 8 + 4);
+                    c_nxt[0] = ca.x; c_nxt[1] = ca.y; c_nxt[2] = ca.z; c_nxt[3] = ca.w;
+                    c_nxt[4] = cb.x; c_nxt[5] = cb.y; c_nxt[6] = cb.z; c_nxt[7] = cb.w;
+                    s_nxt[0] = sa.x; s_nxt[1] = sa.y; s_nxt[2] = sa.z; s_nxt[3] = sa.w;
+                    s_nxt[4] = sb.x; s_nxt[5] = sb.y; s_nxt[6] = sb.z; s_nxt[7] = sb.w;
+                }
+                tmem_ld_wait();
+                if (ready && ok) {
+                    uint16_t lo8[8], hi8[8];
+                    float af[8], bf[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const uint32_t pk = pack_bf16x2(__uint_as_float(lo[e]), __uint_as_float(hi[e]));
+                        lo8[e] = static_cast<uint16_t>(pk & 0xFFFFu);
+                        hi8[e] = static_cast<uint16_t>(pk >> 16);
+                        af[e] = __uint_as_float(pk << 16);
+                        bf[e] = __uint_as_float(pk & 0xFFFF0000u);
+                    }
+                    if (rotate) {
+                        // all sixteen rotations without a branch, then the rare unproven ones again in fp64
+                        uint32_t unproven = 0;
 #pragma unroll
                         for (int e = 0; e < 8; ++e) {
-                            const uint32_t pk = pack_bf16x2(__uint_as_float(lo_bits[v * 8 + e]),
-                                                            __uint_as_float(hi_bits[v * 8 + e]));
-                            const uint16_t a = static_cast<uint16_t>(pk & 0xFFFFu), bb = static_cast<uint16_t>(pk >> 16);
-                            lo8[e] = rotate ? rope_first_half(a, bb, c8[e], s8[e]) : a;
-                            hi8[e] = rotate ? rope_second_half(a, bb, c8[e], s8[e]) : bb;
+                            bool p_lo, p_hi;
+                            lo8[e] = rope_diff_of_products_f32(af[e], c_cur[e], bf[e], s_cur[e], p_lo);
+                            hi8[e] = rope_diff_of_products_f32(bf[e], c_cur[e], af[e], -s_cur[e], p_hi);
+                            unproven |= (p_lo ? 0u : 1u << e) | (p_hi ? 0u : 256u << e);
                         }
-                        uint4 lo_v, hi_v;
-                        lo_v.x = lo8[0] | (static_cast<uint32_t>(lo8[1]) << 16);
-                        lo_v.y = lo8[2] | (static_cast<uint32_t>(lo8[3]) << 16);
-                        lo_v.z = lo8[4] | (static_cast<uint32_t>(lo8[5]) << 16);
-                        lo_v.w = lo8[6] | (static_cast<uint32_t>(lo8[7]) << 16);
-                        hi_v.x = hi8[0] | (static_cast<uint32_t>(hi8[1]) << 16);
-                        hi_v.y = hi8[2] | (static_cast<uint32_t>(hi8[3]) << 16);
-                        hi_v.z = hi8[4] | (static_cast<uint32_t>(hi8[5]) << 16);
-                        hi_v.w = hi8[6] | (static_cast<uint32_t>(hi8[7]) << 16);
-                        *reinterpret_cast<uint4*>(dst + i0 + v * 8) = lo_v;
-                        *reinterpret_cast<uint4*>(dst + i0 + half_d + v * 8) = hi_v;
+                        if (unproven != 0) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                if (unproven & (1u << e))
+                                    lo8[e] = rope_diff_of_products_f64(af[e], c_cur[e], bf[e], s_cur[e]);
+                                if (unproven & (256u << e))
+                                    hi8[e] = rope_diff_of_products_f64(bf[e], c_cur[e], af[e], -s_cur[e]);
+                            }
+                        }
                     }
+                    uint4 lo_v, hi_v;
+                    lo_v.x = lo8[0] | (static_cast<uint32_t>(lo8[1]) << 16);
+                    lo_v.y = lo8[2] | (static_cast<uint32_t>(lo8[3]) << 16);
+                    lo_v.z = lo8[4] | (static_cast<uint32_t>(lo8[5]) << 16);
+                    lo_v.w = lo8[6] | (static_cast<uint32_t>(lo8[7]) << 16);
+                    hi_v.x = hi8[0] | (static_cast<uint32_t>(hi8[1]) << 16);
+                    hi_v.y = hi8[2] | (static_cast<uint32_t>(hi8[3]) << 16);
+                    hi_v.z = hi8[4] | (static_cast<uint32_t>(hi8[5]) << 16);
+                    hi_v.w = hi8[6] | (static_cast<uint32_t>(hi8[7]) << 16);
+                    *reinterpret_cast<uint4*>(dst + i0 + v * 8) = lo_v;
+                    *reinterpret_cast<uint4*>(dst + i0 + half_d + v * 8) = hi_v;
                 }
             }
         }
@@ -355,6 +442,14 @@ cudaError_t launch_tc(const CUtensorMap& w_map, const CUtensorMap& x_map, const 
 }
 
 }  // namespace
+
+// Batch rows per CTA: the batch is cut into the fewest tiles of at most 128 rows, of equal size rounded
+// up to the 8-row swizzle period, so that no tile loads rows that do not exist.
+int proj_tc_batch_rows(int B) {
+    const int tiles = (B + TC_M - 1) / TC_M;
+    const int rows = ((B + tiles - 1) / tiles + 7) / 8 * 8;
+    return rows < TC_M ? rows : TC_M;
+}
 
 cudaError_t proj_tc_set_attributes(int smem_optin) {
     if (TC_SMEM_TOTAL > smem_optin) return cudaErrorInvalidConfiguration;
@@ -394,8 +489,9 @@ cudaError_t launch_qkv_rope_kv_append_tc(const CUtensorMap& w_map, const CUtenso
     p.Hq = Hq;
     p.Hkv = Hkv;
     p.d = d;
-    return launch_tc<TC_EPI_QKV_ROPE_APPEND>(w_map, x_map, p, dim3(d / 64, Hq + 2 * Hkv, (B + TC_M - 1) / TC_M),
-                                             stream);
+    p.x_rows = proj_tc_batch_rows(B);
+    return launch_tc<TC_EPI_QKV_ROPE_APPEND>(w_map, x_map, p,
+                                             dim3(d / 64, Hq + 2 * Hkv, (B + p.x_rows - 1) / p.x_rows), stream);
 }
 
 cudaError_t launch_oproj_residual_tc(const CUtensorMap& w_map, const CUtensorMap& x_map,
@@ -407,7 +503,8 @@ cudaError_t launch_oproj_residual_tc(const CUtensorMap& w_map, const CUtensorMap
     p.N = N;
     p.residual_in = static_cast<const uint16_t*>(residual_in);
     p.residual_out = static_cast<uint16_t*>(residual_out);
-    return launch_tc<TC_EPI_RESIDUAL_ADD>(w_map, x_map, p, dim3(1, N / 64, (B + TC_M - 1) / TC_M), stream);
+    p.x_rows = proj_tc_batch_rows(B);
+    return launch_tc<TC_EPI_RESIDUAL_ADD>(w_map, x_map, p, dim3(1, N / 64, (B + p.x_rows - 1) / p.x_rows), stream);
 }
 
 }  // namespace ac
