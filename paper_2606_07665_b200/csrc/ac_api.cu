@@ -28,7 +28,7 @@ struct Shape {
 };
 
 // Largest batch the warp-MMA projection kernels take; beyond it the tcgen05 kernels are used.
-constexpr int kWarpMmaMaxBatch = 32;
+constexpr int kWarpMmaMaxBatch = 16;
 
 int check_shape(const Shape& s) {
     if (s.B <= 0 || s.Hq <= 0 || s.Hkv <= 0 || s.d <= 0 || s.page_size <= 0 || s.num_pages <= 0)
@@ -335,11 +335,11 @@ int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out, 
     const cuuint64_t row_bytes = static_cast<cuuint64_t>(H) * 2;
     CUtensorMap w_map, x_map;
     if (B > kWarpMmaMaxBatch) {
-        // Batched decode: 128-row batch tiles on the tcgen05 path (boxes of 32 pairs x one K block).
+        // Batched decode: batch tiles of up to 128 rows on the tcgen05 path (boxes of 24 pairs x 2 K blocks).
         cuuint64_t wdims[5] = {64, static_cast<cuuint64_t>(d / 2), 2, static_cast<cuuint64_t>(Hq + 2 * Hkv),
                                static_cast<cuuint64_t>(H / 64)};
         cuuint64_t wstrides[4] = {row_bytes, row_bytes * (d / 2), row_bytes * d, 128};
-        cuuint32_t wbox[5] = {64, 32, 2, 1, 2};
+        cuuint32_t wbox[5] = {64, 24, 2, 1, static_cast<cuuint32_t>(proj_tc_k_blocks(B))};
         cuuint32_t es5[5] = {1, 1, 1, 1, 1};
         CUresult r = g_encode_tiled(&w_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(w_qkv),
                                     wdims, wstrides, wbox, es5, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -348,7 +348,7 @@ int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out, 
         if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
         cuuint64_t xdims[3] = {64, static_cast<cuuint64_t>(B), static_cast<cuuint64_t>(H / 64)};
         cuuint64_t xstrides[2] = {row_bytes, 128};
-        cuuint32_t xbox[3] = {64, static_cast<cuuint32_t>(proj_tc_batch_rows(B)), 2};
+        cuuint32_t xbox[3] = {64, static_cast<cuuint32_t>(proj_tc_batch_rows(B)), static_cast<cuuint32_t>(proj_tc_k_blocks(B))};
         cuuint32_t es3[3] = {1, 1, 1};
         r = g_encode_tiled(&x_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), xdims, xstrides,
                            xbox, es3, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -409,10 +409,10 @@ int ac_oproj_residual_rmsnorm(const void* attn_out, const void* w_o, int K, int 
     const cuuint64_t row_bytes = static_cast<cuuint64_t>(K) * 2;
     CUtensorMap w_map, x_map;
     cudaStream_t cs_tc = static_cast<cudaStream_t>(stream);
-    if (B > kWarpMmaMaxBatch && N % 64 == 0) {
-        cuuint64_t wdims[5] = {64, 32, 2, static_cast<cuuint64_t>(N / 64), static_cast<cuuint64_t>(K / 64)};
-        cuuint64_t wstrides[4] = {row_bytes, row_bytes * 32, row_bytes * 64, 128};
-        cuuint32_t wbox[5] = {64, 32, 2, 1, 2};
+    if (B > kWarpMmaMaxBatch) {
+        cuuint64_t wdims[5] = {64, 16, 2, static_cast<cuuint64_t>(N / 32), static_cast<cuuint64_t>(K / 64)};
+        cuuint64_t wstrides[4] = {row_bytes, row_bytes * 16, row_bytes * 32, 128};
+        cuuint32_t wbox[5] = {64, 16, 2, 1, static_cast<cuuint32_t>(proj_tc_k_blocks(B))};
         cuuint32_t es5[5] = {1, 1, 1, 1, 1};
         CUresult r = g_encode_tiled(&w_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(w_o), wdims,
                                     wstrides, wbox, es5, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -421,7 +421,7 @@ int ac_oproj_residual_rmsnorm(const void* attn_out, const void* w_o, int K, int 
         if (r != CUDA_SUCCESS) return fail_cuda(static_cast<int>(r));
         cuuint64_t xdims[3] = {64, static_cast<cuuint64_t>(B), static_cast<cuuint64_t>(K / 64)};
         cuuint64_t xstrides[2] = {row_bytes, 128};
-        cuuint32_t xbox[3] = {64, static_cast<cuuint32_t>(proj_tc_batch_rows(B)), 2};
+        cuuint32_t xbox[3] = {64, static_cast<cuuint32_t>(proj_tc_batch_rows(B)), static_cast<cuuint32_t>(proj_tc_k_blocks(B))};
         cuuint32_t es3[3] = {1, 1, 1};
         r = g_encode_tiled(&x_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(attn_out), xdims,
                            xstrides, xbox, es3, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,

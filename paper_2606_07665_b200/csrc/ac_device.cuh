@@ -169,24 +169,33 @@ __device__ __forceinline__ uint16_t f64_to_bf16_rne(double x) {
     return static_cast<uint16_t>(u >> 16);
 }
 
-// bf16_rne(fl64(x1 * y1 - x2 * y2)) for x1, x2 with bf16 precision (8-bit significands) and fp32 y1, y2:
-// both products are exact in fp64 (8 x 24 bits), the difference is rounded to fp64 once and then to
-// bf16 once.  That reference evaluation needs a dozen fp64-pipe instructions per output, so it is
-// kept for the rare hard cases only.  The common case runs in fp32: error-free products (product and
+// (a, b) = (x_i, x_{i+d/2}) as bf16 bits, c/s = cos/sin of the pair's angle.  Both products are exact
+// in fp64 (8-bit x 24-bit significands); __dmul_rn/__dadd_rn keep the three operations separate.
+__device__ __forceinline__ uint16_t rope_first_half(uint16_t a, uint16_t b, float c, float s) {
+    const double ad = static_cast<double>(bf16_bits_to_float(a));
+    const double bd = static_cast<double>(bf16_bits_to_float(b));
+    return f64_to_bf16_rne(__dsub_rn(__dmul_rn(ad, static_cast<double>(c)), __dmul_rn(bd, static_cast<double>(s))));
+}
+
+__device__ __forceinline__ uint16_t rope_second_half(uint16_t a, uint16_t b, float c, float s) {
+    const double ad = static_cast<double>(bf16_bits_to_float(a));
+    const double bd = static_cast<double>(bf16_bits_to_float(b));
+    return f64_to_bf16_rne(__dadd_rn(__dmul_rn(bd, static_cast<double>(c)), __dmul_rn(ad, static_cast<double>(s))));
+}
+
+// ---- the same rotation for callers that rotate thousands of values per CTA ------------------------
+//
+// bf16_rne(fl64(x1 * y1 - x2 * y2)) for x1, x2 with bf16 precision (8-bit significands) and fp32 y1, y2
+// is what the two functions above compute (first half: a c - b s; second half: b c - a (-s)).  That
+// evaluation costs a dozen fp64-pipe instructions per output, which a kernel that rotates a few
+// values per thread never notices and an epilogue that rotates 128 rows x 48 features does.  The
+// fp32 evaluation below gives the same bits whenever it can prove so: error-free products (product and
 // fma residual), an error-free difference of the high parts (TwoSum), and the small terms added on
 // top give r with |r - exact| < 0.501 ulp(r) provided the difference did not cancel more than ten bits
 // and nothing is near the fp32 range limits.  If r is then at least three fp32 ulps away from every
 // midpoint between adjacent bf16 values (low half-word not in 0x7FFE..0x8002), the exact value, its
-// fp64 rounding and r all round to the same bf16.
-__device__ __noinline__ inline uint16_t rope_diff_of_products_f64(float x1, float y1, float x2, float y2) {
-    // Kept out of line: it is rare, and callers unroll dozens of rotations.
-    return f64_to_bf16_rne(__dsub_rn(__dmul_rn(static_cast<double>(x1), static_cast<double>(y1)),
-                                     __dmul_rn(static_cast<double>(x2), static_cast<double>(y2))));
-}
-
-// The fp32 evaluation alone: returns the bf16 candidate and sets `proven` when the argument above holds
-// for it.  Callers that rotate many values evaluate a batch without branches and repair the (rare)
-// unproven ones afterwards with rope_diff_of_products_f64.
+// fp64 rounding and r all round to the same bf16.  Callers evaluate a batch without branches and
+// repair the (rare) unproven ones afterwards with rope_diff_of_products_f64.
 __device__ __forceinline__ uint16_t rope_diff_of_products_f32(float x1, float y1, float x2, float y2, bool& proven) {
     const float p1 = __fmul_rn(x1, y1);
     const float p1l = __fmaf_rn(x1, y1, -p1);            // exact: the product has at most 32 bits
@@ -203,20 +212,10 @@ __device__ __forceinline__ uint16_t rope_diff_of_products_f32(float x1, float y1
     return static_cast<uint16_t>((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
 }
 
-__device__ __forceinline__ uint16_t rope_diff_of_products(float x1, float y1, float x2, float y2) {
-    bool proven;
-    const uint16_t fast = rope_diff_of_products_f32(x1, y1, x2, y2, proven);
-    return proven ? fast : rope_diff_of_products_f64(x1, y1, x2, y2);
-}
-
-// (a, b) = (x_i, x_{i+d/2}) as bf16 bits, c/s = cos/sin of the pair's angle: a c - b s and b c + a s,
-// each evaluated exactly and rounded as described above.
-__device__ __forceinline__ uint16_t rope_first_half(uint16_t a, uint16_t b, float c, float s) {
-    return rope_diff_of_products(bf16_bits_to_float(a), c, bf16_bits_to_float(b), s);
-}
-
-__device__ __forceinline__ uint16_t rope_second_half(uint16_t a, uint16_t b, float c, float s) {
-    return rope_diff_of_products(bf16_bits_to_float(b), c, bf16_bits_to_float(a), -s);
+// Kept out of line: it is rare, and the callers unroll dozens of rotations.
+__device__ __noinline__ inline uint16_t rope_diff_of_products_f64(float x1, float y1, float x2, float y2) {
+    return f64_to_bf16_rne(__dsub_rn(__dmul_rn(static_cast<double>(x1), static_cast<double>(y1)),
+                                     __dmul_rn(static_cast<double>(x2), static_cast<double>(y2))));
 }
 
 }  // namespace acdev

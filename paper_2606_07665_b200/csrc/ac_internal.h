@@ -92,6 +92,7 @@ cudaError_t launch_rmsnorm_rows(const void* h, const void* weight, void* out, in
                                 cudaStream_t stream);
 cudaError_t proj_tc_set_attributes(int smem_optin);
 int proj_tc_batch_rows(int B);          // rows of the x box the tcgen05 kernels expect for batch B
+int proj_tc_k_blocks(int B);            // 64-element K blocks per TMA box (x and W) they expect for batch B
 cudaError_t launch_qkv_rope_kv_append_tc(const CUtensorMap& w_map, const CUtensorMap& x_map, void* q_out,
                                          void* k_cache, void* v_cache, int64_t stride_page,
                                          int64_t stride_token, int64_t stride_head,

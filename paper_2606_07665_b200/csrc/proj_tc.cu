@@ -2,21 +2,28 @@
 //
 // Same products and epilogues as qkv_prelude.cu (QKV projection + RoPE + KV append; output projection
 // + residual), for batches too large for the warp-MMA kernel's 32-row tiles: from a few dozen rows on
-// the contraction y[b, n] = sum_k x[b, k] W[n, k] stops being a weight stream and becomes a thin GEMM
-// whose operand traffic is dominated by re-reading x, so a 128-row batch tile per CTA (W streamed from
-// HBM once per 128 rows) and the UMMA pipe pay.
+// the contraction y[b, n] = sum_k x[b, k] W[n, k] stops being a weight stream and becomes a thin GEMM,
+// so the batch becomes the M dimension of a tcgen05.mma (up to 128 rows per CTA: W is streamed from
+// HBM once per 128 rows) with the accumulator in tensor memory.
 //
-// One CTA = 128 batch rows (M) x 64 output features (N: 32 rotary pairs, i.e. W rows i..i+31 and
-// i+d/2..i+d/2+31 of one head, or 64 consecutive rows for the output projection) x all of K.
-//   warp 0   producer: per 128-wide K chunk one 3-D TMA load of the x tile [128 rows x 2 x 64] (32 KB;
-//            rows beyond B are zero-filled by the bounds check) and one 5-D TMA load of the W tile
-//            [2 halves x 32 rows x 2 x 64] (16 KB), both as 128-byte-swizzled K-major blocks, into a
-//            4-stage ring (256 contiguous bytes of every W row per load);
-//   warp 1   allocates 64 TMEM columns, and its lane 0 issues eight tcgen05.mma (M128 N64 K16, bf16
-//            -> fp32) per chunk from shared-memory descriptors, then tcgen05.commit to hand the stage
-//            back to the producer, and a final commit to release the epilogue;
-//   warps 2-5 read the accumulator with tcgen05.ld (thread = one batch row, 64 columns), round to
-//            bf16, rotate / add the residual, and store.
+// What sets the pace is how fast one SM pulls its share of W out of DRAM through TMA (about 40 GB/s
+// per SM, whatever the ring depth), so the feature tiles are chosen to put a CTA on nearly every SM:
+//   QKV      48 features per CTA = 24 rotary pairs (W rows i..i+23 and i+d/2.. of one head).  A head
+//            has 64 pairs (d = 128), so three tiles start at pairs 0, 16 and 40: 144 CTAs for 48 head
+//            slots; the pairs that two tiles share are computed twice and stored twice with the same
+//            bits (12.5 % more weight traffic for 50 % more SMs).
+//   o_proj   32 consecutive output features per CTA (128 CTAs for N = 4096).
+// Per CTA:
+//   warp 0   producer: per 128-wide K chunk one 3-D TMA load of the x tile [x_rows x 2 x 64] and one
+//            5-D TMA load of the W tile, both as 128-byte-swizzled K-major blocks, into a ring that is
+//            as deep as shared memory allows (256 contiguous bytes of every W row per load);
+//   warp 1   allocates the TMEM columns, and its lane 0 issues eight tcgen05.mma (M128, K16, bf16 ->
+//            fp32) per chunk from shared-memory descriptors, then tcgen05.commit to hand the stage back
+//            to the producer, and a final commit to release the epilogue;
+//   the other warps are the epilogue, one warp per 32 batch rows and group of columns (thread = one
+//            batch row; 8 rotary pairs or 16 output features): they compute addresses and fetch angles
+//            or residuals while the main loop runs, then read the accumulator with tcgen05.ld, round
+//            to bf16, rotate / add the residual, and store.
 // Every wait is bounded; TMEM is released on every path.
 #include <math.h>
 
@@ -30,18 +37,26 @@ using namespace acdev;
 
 enum { TC_EPI_QKV_ROPE_APPEND = 0, TC_EPI_RESIDUAL_ADD = 1 };
 
-constexpr int TC_THREADS = 192;
 constexpr int TC_M = 128;                       // rows of the MMA tile: batch rows per CTA, at most
-constexpr int TC_N = 64;                        // output features per CTA
-constexpr int TC_KBLK = 2;                      // 64-element (128-byte) K blocks per stage
-constexpr int TC_KC = 64 * TC_KBLK;             // K elements per stage
 constexpr int TC_MAX_STAGES = 12;
-constexpr int TC_RING_BYTES = 216 * 1024;       // holds as many stages as fit: 4 at 128 batch rows, 8 at 40
-constexpr int TC_B_BLOCK = TC_N * 128;          // one swizzled [64 rows x 128 B] block of W: 8 KB
-constexpr int TC_B_BYTES = TC_KBLK * TC_B_BLOCK;
+constexpr int TC_RING_BYTES = 220 * 1024;       // holds as many stages as fit
 constexpr int TC_BAR_OFFSET = TC_RING_BYTES;
 constexpr int TC_SMEM_TOTAL = TC_BAR_OFFSET + (2 * TC_MAX_STAGES + 1) * 8 + 16 + 1024;
-constexpr uint32_t TC_TMEM_COLS = 64;
+
+template <int EPI>
+struct TcTile {
+    static constexpr int N = EPI == TC_EPI_QKV_ROPE_APPEND ? 48 : 32;        // features per CTA
+    static constexpr int GROUPS = EPI == TC_EPI_QKV_ROPE_APPEND ? 3 : 2;     // epilogue warps per 32 rows
+    static constexpr int THREADS = 64 + 128 * GROUPS;
+    static constexpr int B_BLOCK = N * 128;          // one swizzled [N rows x 128 B] block of W
+    static constexpr uint32_t TMEM_COLS = EPI == TC_EPI_QKV_ROPE_APPEND ? 64 : 32;   // a power of two >= N
+};
+
+// First rotary pair of QKV tile `blk` inside its head: 24-pair tiles at 0, 16, 40 (64 pairs per head)
+// or at 0, 8 (32 pairs per head); multiples of 8 so that every store is 16-byte aligned.
+__host__ __device__ inline int qkv_tile_first_pair(int half_d, int blk) {
+    return half_d == 64 ? (blk == 0 ? 0 : blk == 1 ? 16 : 40) : 8 * blk;
+}
 
 struct TcParams {
     uint16_t* q_out;
@@ -94,9 +109,9 @@ __device__ __forceinline__ uint64_t umma_desc_k_major_sw128(uint32_t smem_byte_a
     return desc;
 }
 
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 64.
-__device__ __forceinline__ uint32_t umma_idesc_bf16_m128_n64() {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((TC_N >> 3) << 17) | ((TC_M >> 4) << 24);
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n (a multiple of 16).
+__device__ __forceinline__ uint32_t umma_idesc_bf16_m128(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
@@ -117,21 +132,7 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
                  : "memory");
 }
 
-// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp gets lane (warp % 4) * 32 + i.
-__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
-
-// 32 lanes x 8 consecutive 32-bit columns.
+// 32 lanes x 8 consecutive 32-bit columns: thread i of the warp gets lane (warp % 4) * 32 + i.
 __device__ __forceinline__ void tmem_ld_32x8(uint32_t taddr, uint32_t (&r)[8]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
@@ -141,10 +142,13 @@ __device__ __forceinline__ void tmem_ld_32x8(uint32_t taddr, uint32_t (&r)[8]) {
 
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-template <int EPI>
-__global__ void __launch_bounds__(TC_THREADS, 1) proj_tc_kernel(const __grid_constant__ CUtensorMap w_map,
-                                                                const __grid_constant__ CUtensorMap x_map,
-                                                                const TcParams p) {
+// KBLK = 64-element (128-byte) K blocks per stage, 2 or 4 (a compile-time constant: the thread that
+// issues the MMAs is the critical path of the main loop, and every instruction in its loop shows).
+template <int EPI, int KBLK>
+__global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const __grid_constant__ CUtensorMap w_map,
+                                                                          const __grid_constant__ CUtensorMap x_map,
+                                                                          const TcParams p) {
+    using T = TcTile<EPI>;
     cudaTriggerProgrammaticLaunchCompletion();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_addr(smem_raw) + 1023u) & ~1023u;
@@ -156,20 +160,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) proj_tc_kernel(const __grid_con
     volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + TC_BAR_OFFSET +
                                                                             (2 * TC_MAX_STAGES + 1) * 8);
 
-    const int blk = blockIdx.x;          // block of 32 pairs inside the head (QKV) / unused (o_proj)
-    const int hh = blockIdx.y;           // head slot (QKV) / block of 64 output features (o_proj)
+    const int blk = blockIdx.x;          // pair tile inside the head (QKV) / unused (o_proj)
+    const int hh = blockIdx.y;           // head slot (QKV) / block of 32 output features (o_proj)
+    const int pair0 = EPI == TC_EPI_QKV_ROPE_APPEND ? qkv_tile_first_pair(p.d / 2, blk) : 0;
     // The x box holds x_rows rows per 64-element block; the MMA always reads 128.  Rows past x_rows are
     // whatever the ring holds: every accumulator row depends on its own x row only, and the epilogue
-    // skips them.  A stage is the x tile followed by the W tile.  The weights come from DRAM with
-    // microseconds of latency, so the ring is as deep as shared memory allows.
+    // skips them.  A stage is the x tile followed by the W tile.
     const int b0 = blockIdx.z * p.x_rows;
     const uint32_t a_block = static_cast<uint32_t>(p.x_rows) * 128u;
-    const uint32_t a_bytes = TC_KBLK * a_block;
-    const uint32_t stage_bytes = a_bytes + TC_B_BYTES;       // a multiple of 1024
+    const uint32_t a_bytes = KBLK * a_block;
+    const uint32_t stage_bytes = a_bytes + KBLK * T::B_BLOCK;        // a multiple of 1024
     const int stages = min(TC_MAX_STAGES, TC_RING_BYTES / static_cast<int>(stage_bytes));
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int n_chunks = (p.K + TC_KC - 1) / TC_KC;
+    const int n_chunks = (p.K + 64 * KBLK - 1) / (64 * KBLK);
 
     if (threadIdx.x == 0) {
         tma_prefetch_descriptor(&w_map);
@@ -181,7 +185,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) proj_tc_kernel(const __grid_con
         mbar_init(done_bar, 1);
         mbar_init_fence();
     }
-    if (warp == 1) tmem_alloc(tmem_slot, TC_TMEM_COLS);
+    if (warp == 1) tmem_alloc(tmem_slot, T::TMEM_COLS);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -202,13 +206,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) proj_tc_kernel(const __grid_con
                 }
                 const uint32_t dst = smem_base + stage * stage_bytes;
                 mbar_arrive_expect_tx(full_bar + stage * 8, stage_bytes);
-                tma_load_3d(dst, &x_map, full_bar + stage * 8, 0, b0, c * TC_KBLK, keep);
-                if (EPI == TC_EPI_QKV_ROPE_APPEND)
-                    tma_load_5d(dst + a_bytes, &w_map, full_bar + stage * 8, 0, 32 * blk, 0, hh, c * TC_KBLK,
-                                stream_once);
-                else
-                    tma_load_5d(dst + a_bytes, &w_map, full_bar + stage * 8, 0, 0, 0, hh, c * TC_KBLK,
-                                stream_once);
+                tma_load_3d(dst, &x_map, full_bar + stage * 8, 0, b0, c * KBLK, keep);
+                tma_load_5d(dst + a_bytes, &w_map, full_bar + stage * 8, 0, pair0, 0, hh, c * KBLK, stream_once);
                 if (++stage == stages) {
                     stage = 0;
                     ++round;
@@ -217,7 +216,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) proj_tc_kernel(const __grid_con
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16_m128_n64();
+            const uint32_t idesc = umma_idesc_bf16_m128(T::N);
             int stage = 0;
             uint32_t round = 0;
             for (int c = 0; c < n_chunks; ++c) {
@@ -228,9 +227,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) proj_tc_kernel(const __grid_con
                 tc_fence_after_sync();
                 const uint32_t a_addr = smem_base + stage * stage_bytes;
 #pragma unroll
-                for (int kb = 0; kb < TC_KBLK; ++kb) {
+                for (int kb = 0; kb < KBLK; ++kb) {
                     const uint64_t adesc = umma_desc_k_major_sw128(a_addr + kb * a_block);
-                    const uint64_t bdesc = umma_desc_k_major_sw128(a_addr + a_bytes + kb * TC_B_BLOCK);
+                    const uint64_t bdesc = umma_desc_k_major_sw128(a_addr + a_bytes + kb * T::B_BLOCK);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)           // 16 elements = 32 bytes = 2 descriptor units
                         umma_bf16(tmem_d, adesc + 2 * ks, bdesc + 2 * ks, idesc,
@@ -248,171 +247,146 @@ __global__ void __launch_bounds__(TC_THREADS, 1) proj_tc_kernel(const __grid_con
     if (timed_out && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_WAIT_TIMEOUT);
 
     if (warp >= 2) {
-        // ---- epilogue: thread = batch row, 64 accumulator columns -------------------------------------
-        // Everything that does not need the accumulator is done first, under the main loop: the row's
-        // position, its destination and (QKV) its rotary angles.
+        // ---- epilogue: thread = batch row; warp = 32 rows x one group of columns --------------------
+        // Everything that does not need the accumulator is done first, under the main loop.
         const int quarter = warp & 3;                        // TMEM lanes this warp may read
+        const int group = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;
         const int b = b0 + row;
         bool ok = row < p.x_rows && b < p.B;
-        uint16_t* dst = nullptr;
-        const uint16_t* res = nullptr;
-        bool rotate = false;
-        const float* cos_row = nullptr;                      // angles of this row's 32 pairs (QKV, q and k heads)
-        const float* sin_row = nullptr;
-        float c_nxt[8], s_nxt[8];                            // angles of the next group of 8 pairs
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            c_nxt[e] = 1.0f;
-            s_nxt[e] = 0.0f;
-        }
-        const int i0 = 32 * blk;                             // first pair of this CTA (QKV)
-        if (EPI == TC_EPI_RESIDUAL_ADD) {
-            if (ok) {
-                const size_t idx = static_cast<size_t>(b) * p.N + 64 * hh;
-                dst = p.residual_out + idx;
-                res = p.residual_in + idx;
-            }
-        } else if (ok) {
-            const int ctx = p.context_lens[b];
-            const int d = p.d, half_d = d / 2;
-            int page_idx = 0;
-            ok = ctx >= 0;
-            if (ok) {
-                page_idx = ctx / p.page_size;
-                if (ctx >= p.max_position || page_idx >= p.max_pages_per_seq) {
-                    if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
-                    ok = false;
-                }
-            }
-            rotate = hh < p.Hq + p.Hkv;
-            if (ok) {
-                if (hh < p.Hq) {
-                    dst = p.q_out + (static_cast<size_t>(b) * p.Hq + hh) * d;
-                } else {
-                    const int page = p.block_table[static_cast<size_t>(b) * p.max_pages_per_seq + page_idx];
-                    if (page < 0 || page >= p.num_pages) {
-                        if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
-                        ok = false;
-                    } else {
-                        const bool is_k = hh < p.Hq + p.Hkv;
-                        const int h = is_k ? hh - p.Hq : hh - p.Hq - p.Hkv;
-                        dst = (is_k ? p.k_cache : p.v_cache) + static_cast<size_t>(page) * p.stride_page +
-                              static_cast<size_t>(ctx - page_idx * p.page_size) * p.stride_token +
-                              static_cast<size_t>(h) * p.stride_head;
-                    }
-                }
-            }
-            if (ok && rotate) {
-                cos_row = p.rope_cos + static_cast<size_t>(ctx) * half_d + i0;
-                sin_row = p.rope_sin + static_cast<size_t>(ctx) * half_d + i0;
-                const float4 ca = *reinterpret_cast<const float4*>(cos_row), cb = *reinterpret_cast<const float4*>(cos_row + 4);
-                const float4 sa = *reinterpret_cast<const float4*>(sin_row), sb = *reinterpret_cast<const float4*>(sin_row + 4);
-                c_nxt[0] = ca.x; c_nxt[1] = ca.y; c_nxt[2] = ca.z; c_nxt[3] = ca.w;
-                c_nxt[4] = cb.x; c_nxt[5] = cb.y; c_nxt[6] = cb.z; c_nxt[7] = cb.w;
-                s_nxt[0] = sa.x; s_nxt[1] = sa.y; s_nxt[2] = sa.z; s_nxt[3] = sa.w;
-                s_nxt[4] = sb.x; s_nxt[5] = sb.y; s_nxt[6] = sb.z; s_nxt[7] = sb.w;
-            }
-        }
-
-        const bool ready = mbar_wait_bounded(done_bar, 0);
-        if (!ready && lane == 0 && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_WAIT_TIMEOUT);
-        tc_fence_after_sync();
         const uint32_t lane_base = tmem_d + (static_cast<uint32_t>(quarter * 32) << 16);
+
         if (EPI == TC_EPI_RESIDUAL_ADD) {
-            uint32_t lo_bits[32], hi_bits[32];
-            tmem_ld_32x32(lane_base, lo_bits);               // columns 0-31
-            tmem_ld_32x32(lane_base + 32, hi_bits);          // columns 32-63
+            // 16 output features: columns 16 group .. 16 group + 15
+            uint16_t* dst = nullptr;
+            uint4 res[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+            if (ok) {
+                const size_t idx = static_cast<size_t>(b) * p.N + T::N * hh + 16 * group;
+                dst = p.residual_out + idx;
+                res[0] = *reinterpret_cast<const uint4*>(p.residual_in + idx);
+                res[1] = *reinterpret_cast<const uint4*>(p.residual_in + idx + 8);
+            }
+            const bool ready = mbar_wait_bounded(done_bar, 0);
+            if (!ready && lane == 0 && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_WAIT_TIMEOUT);
+            tc_fence_after_sync();
+            uint32_t acc[2][8];
+            tmem_ld_32x8(lane_base + 16 * group, acc[0]);
+            tmem_ld_32x8(lane_base + 16 * group + 8, acc[1]);
             tmem_ld_wait();
             if (ready && ok) {
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const uint32_t* acc = half == 0 ? lo_bits : hi_bits;
+                for (int v = 0; v < 2; ++v) {                // 8 features = 16 bytes at a time
+                    const uint32_t rw[4] = {res[v].x, res[v].y, res[v].z, res[v].w};
+                    uint32_t ow[4];
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {            // 8 features = 16 bytes at a time
-                        const uint4 r8 = *reinterpret_cast<const uint4*>(res + half * 32 + v * 8);
-                        const uint32_t rw[4] = {r8.x, r8.y, r8.z, r8.w};
-                        uint32_t ow[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float r0 = __uint_as_float(rw[e] << 16);
-                            const float r1 = __uint_as_float(rw[e] & 0xFFFF0000u);
-                            ow[e] = pack_bf16x2(r0 + __uint_as_float(acc[v * 8 + 2 * e]),
-                                                r1 + __uint_as_float(acc[v * 8 + 2 * e + 1]));
-                        }
-                        *reinterpret_cast<uint4*>(dst + half * 32 + v * 8) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                    for (int e = 0; e < 4; ++e) {
+                        const float r0 = __uint_as_float(rw[e] << 16);
+                        const float r1 = __uint_as_float(rw[e] & 0xFFFF0000u);
+                        ow[e] = pack_bf16x2(r0 + __uint_as_float(acc[v][2 * e]), r1 + __uint_as_float(acc[v][2 * e + 1]));
                     }
+                    *reinterpret_cast<uint4*>(dst + v * 8) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
                 }
             }
         } else {
-            // Four groups of 8 pairs in a rolled loop (the rotation code is long; unrolled 32 times it
-            // would not stay in the instruction cache); the next group's angles are fetched a group ahead.
-            const int half_d = p.d / 2;
-#pragma unroll 1
-            for (int v = 0; v < 4; ++v) {
-                uint32_t lo[8], hi[8];
-                tmem_ld_32x8(lane_base + v * 8, lo);         // first halves of pairs 8 v .. 8 v + 7
-                tmem_ld_32x8(lane_base + 32 + v * 8, hi);    // their second halves
-                float c_cur[8], s_cur[8];
+            // 8 rotary pairs: first halves in columns 8 group .., second halves in columns 24 + 8 group ..
+            const int d = p.d, half_d = d / 2;
+            const int i0 = pair0 + 8 * group;                // first pair of this warp inside the head
+            uint16_t* dst = nullptr;
+            const bool rotate = hh < p.Hq + p.Hkv;           // v heads are stored as they are
+            float cs[8], sn[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                cs[e] = 1.0f;
+                sn[e] = 0.0f;
+            }
+            if (ok) {
+                const int ctx = p.context_lens[b];
+                int page_idx = 0;
+                ok = ctx >= 0;
+                if (ok) {
+                    page_idx = ctx / p.page_size;
+                    if (ctx >= p.max_position || page_idx >= p.max_pages_per_seq) {
+                        if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
+                        ok = false;
+                    }
+                }
+                if (ok) {
+                    if (hh < p.Hq) {
+                        dst = p.q_out + (static_cast<size_t>(b) * p.Hq + hh) * d;
+                    } else {
+                        const int page = p.block_table[static_cast<size_t>(b) * p.max_pages_per_seq + page_idx];
+                        if (page < 0 || page >= p.num_pages) {
+                            if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
+                            ok = false;
+                        } else {
+                            const bool is_k = hh < p.Hq + p.Hkv;
+                            const int h = is_k ? hh - p.Hq : hh - p.Hq - p.Hkv;
+                            dst = (is_k ? p.k_cache : p.v_cache) + static_cast<size_t>(page) * p.stride_page +
+                                  static_cast<size_t>(ctx - page_idx * p.page_size) * p.stride_token +
+                                  static_cast<size_t>(h) * p.stride_head;
+                        }
+                    }
+                }
+                if (ok && rotate) {
+                    const float* cos_row = p.rope_cos + static_cast<size_t>(ctx) * half_d + i0;
+                    const float* sin_row = p.rope_sin + static_cast<size_t>(ctx) * half_d + i0;
+                    const float4 ca = *reinterpret_cast<const float4*>(cos_row);
+                    const float4 cb = *reinterpret_cast<const float4*>(cos_row + 4);
+                    const float4 sa = *reinterpret_cast<const float4*>(sin_row);
+                    const float4 sb = *reinterpret_cast<const float4*>(sin_row + 4);
+                    cs[0] = ca.x; cs[1] = ca.y; cs[2] = ca.z; cs[3] = ca.w;
+                    cs[4] = cb.x; cs[5] = cb.y; cs[6] = cb.z; cs[7] = cb.w;
+                    sn[0] = sa.x; sn[1] = sa.y; sn[2] = sa.z; sn[3] = sa.w;
+                    sn[4] = sb.x; sn[5] = sb.y; sn[6] = sb.z; sn[7] = sb.w;
+                }
+            }
+            const bool ready = mbar_wait_bounded(done_bar, 0);
+            if (!ready && lane == 0 && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_WAIT_TIMEOUT);
+            tc_fence_after_sync();
+            uint32_t lo[8], hi[8];
+            tmem_ld_32x8(lane_base + 8 * group, lo);                 // first halves of pairs i0 .. i0 + 7
+            tmem_ld_32x8(lane_base + T::N / 2 + 8 * group, hi);      // their second halves
+            tmem_ld_wait();
+            if (ready && ok) {
+                uint16_t lo8[8], hi8[8];
+                float af[8], bf[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    c_cur[e] = c_nxt[e];
-                    s_cur[e] = s_nxt[e];
+                    const uint32_t pk = pack_bf16x2(__uint_as_float(lo[e]), __uint_as_float(hi[e]));
+                    lo8[e] = static_cast<uint16_t>(pk & 0xFFFFu);
+                    hi8[e] = static_cast<uint16_t>(pk >> 16);
+                    af[e] = __uint_as_float(pk << 16);
+                    bf[e] = __uint_as_float(pk & 0xFFFF0000u);
                 }
-                if (cos_row != nullptr && v < 3) {
-                    const float4 ca = *reinterpret_cast<const float4*>(cos_row + (v + 1) * 8);
-                    const float4 cb = *reinterpret_cast<const float4*>(cos_row + (v + 1) * 8 + 4);
-                    const float4 sa = *reinterpret_cast<const float4*>(sin_row + (v + 1) * 8);
-                    const float4 sb = *reinterpret_cast<const float4*>(sin_row + (v + 1) * 8 + 4);
-                    c_nxt[0] = ca.x; c_nxt[1] = ca.y; c_nxt[2] = ca.z; c_nxt[3] = ca.w;
-                    c_nxt[4] = cb.x; c_nxt[5] = cb.y; c_nxt[6] = cb.z; c_nxt[7] = cb.w;
-                    s_nxt[0] = sa.x; s_nxt[1] = sa.y; s_nxt[2] = sa.z; s_nxt[3] = sa.w;
-                    s_nxt[4] = sb.x; s_nxt[5] = sb.y; s_nxt[6] = sb.z; s_nxt[7] = sb.w;
-                }
-                tmem_ld_wait();
-                if (ready && ok) {
-                    uint16_t lo8[8], hi8[8];
-                    float af[8], bf[8];
+                if (rotate) {
+                    // all sixteen rotations without a branch, then the rare unproven ones again in fp64
+                    uint32_t unproven = 0;
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
-                        const uint32_t pk = pack_bf16x2(__uint_as_float(lo[e]), __uint_as_float(hi[e]));
-                        lo8[e] = static_cast<uint16_t>(pk & 0xFFFFu);
-                        hi8[e] = static_cast<uint16_t>(pk >> 16);
-                        af[e] = __uint_as_float(pk << 16);
-                        bf[e] = __uint_as_float(pk & 0xFFFF0000u);
+                        bool p_lo, p_hi;
+                        lo8[e] = rope_diff_of_products_f32(af[e], cs[e], bf[e], sn[e], p_lo);
+                        hi8[e] = rope_diff_of_products_f32(bf[e], cs[e], af[e], -sn[e], p_hi);
+                        unproven |= (p_lo ? 0u : 1u << e) | (p_hi ? 0u : 256u << e);
                     }
-                    if (rotate) {
-                        // all sixteen rotations without a branch, then the rare unproven ones again in fp64
-                        uint32_t unproven = 0;
+                    if (unproven != 0) {
 #pragma unroll
                         for (int e = 0; e < 8; ++e) {
-                            bool p_lo, p_hi;
-                            lo8[e] = rope_diff_of_products_f32(af[e], c_cur[e], bf[e], s_cur[e], p_lo);
-                            hi8[e] = rope_diff_of_products_f32(bf[e], c_cur[e], af[e], -s_cur[e], p_hi);
-                            unproven |= (p_lo ? 0u : 1u << e) | (p_hi ? 0u : 256u << e);
-                        }
-                        if (unproven != 0) {
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                if (unproven & (1u << e))
-                                    lo8[e] = rope_diff_of_products_f64(af[e], c_cur[e], bf[e], s_cur[e]);
-                                if (unproven & (256u << e))
-                                    hi8[e] = rope_diff_of_products_f64(bf[e], c_cur[e], af[e], -s_cur[e]);
-                            }
+                            if (unproven & (1u << e)) lo8[e] = rope_diff_of_products_f64(af[e], cs[e], bf[e], sn[e]);
+                            if (unproven & (256u << e)) hi8[e] = rope_diff_of_products_f64(bf[e], cs[e], af[e], -sn[e]);
                         }
                     }
-                    uint4 lo_v, hi_v;
-                    lo_v.x = lo8[0] | (static_cast<uint32_t>(lo8[1]) << 16);
-                    lo_v.y = lo8[2] | (static_cast<uint32_t>(lo8[3]) << 16);
-                    lo_v.z = lo8[4] | (static_cast<uint32_t>(lo8[5]) << 16);
-                    lo_v.w = lo8[6] | (static_cast<uint32_t>(lo8[7]) << 16);
-                    hi_v.x = hi8[0] | (static_cast<uint32_t>(hi8[1]) << 16);
-                    hi_v.y = hi8[2] | (static_cast<uint32_t>(hi8[3]) << 16);
-                    hi_v.z = hi8[4] | (static_cast<uint32_t>(hi8[5]) << 16);
-                    hi_v.w = hi8[6] | (static_cast<uint32_t>(hi8[7]) << 16);
-                    *reinterpret_cast<uint4*>(dst + i0 + v * 8) = lo_v;
-                    *reinterpret_cast<uint4*>(dst + i0 + half_d + v * 8) = hi_v;
                 }
+                uint4 lo_v, hi_v;
+                lo_v.x = lo8[0] | (static_cast<uint32_t>(lo8[1]) << 16);
+                lo_v.y = lo8[2] | (static_cast<uint32_t>(lo8[3]) << 16);
+                lo_v.z = lo8[4] | (static_cast<uint32_t>(lo8[5]) << 16);
+                lo_v.w = lo8[6] | (static_cast<uint32_t>(lo8[7]) << 16);
+                hi_v.x = hi8[0] | (static_cast<uint32_t>(hi8[1]) << 16);
+                hi_v.y = hi8[2] | (static_cast<uint32_t>(hi8[3]) << 16);
+                hi_v.z = hi8[4] | (static_cast<uint32_t>(hi8[5]) << 16);
+                hi_v.w = hi8[6] | (static_cast<uint32_t>(hi8[7]) << 16);
+                *reinterpret_cast<uint4*>(dst + i0) = lo_v;
+                *reinterpret_cast<uint4*>(dst + i0 + half_d) = hi_v;
             }
         }
     }
@@ -421,16 +395,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) proj_tc_kernel(const __grid_con
     __syncthreads();
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_d, TC_TMEM_COLS);
+        tmem_dealloc(tmem_d, T::TMEM_COLS);
     }
 }
 
-template <int EPI>
-cudaError_t launch_tc(const CUtensorMap& w_map, const CUtensorMap& x_map, const TcParams& p, dim3 grid,
-                      cudaStream_t stream) {
+template <int EPI, int KBLK>
+cudaError_t launch_tc_k(const CUtensorMap& w_map, const CUtensorMap& x_map, const TcParams& p, dim3 grid,
+                        cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
-    cfg.blockDim = dim3(TC_THREADS);
+    cfg.blockDim = dim3(TcTile<EPI>::THREADS);
     cfg.dynamicSmemBytes = TC_SMEM_TOTAL;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -438,7 +412,14 @@ cudaError_t launch_tc(const CUtensorMap& w_map, const CUtensorMap& x_map, const 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, proj_tc_kernel<EPI>, w_map, x_map, p);
+    return cudaLaunchKernelEx(&cfg, proj_tc_kernel<EPI, KBLK>, w_map, x_map, p);
+}
+
+template <int EPI>
+cudaError_t launch_tc(const CUtensorMap& w_map, const CUtensorMap& x_map, const TcParams& p, int kblk, dim3 grid,
+                      cudaStream_t stream) {
+    return kblk == 4 ? launch_tc_k<EPI, 4>(w_map, x_map, p, grid, stream)
+                     : launch_tc_k<EPI, 2>(w_map, x_map, p, grid, stream);
 }
 
 }  // namespace
@@ -451,13 +432,24 @@ int proj_tc_batch_rows(int B) {
     return rows < TC_M ? rows : TC_M;
 }
 
+// K blocks per stage: loads of 512 contiguous bytes per weight row stream measurably faster than loads
+// of 256, but only while at least three stages still fit beside the x tiles.
+int proj_tc_k_blocks(int B) { return proj_tc_batch_rows(B) <= 96 ? 4 : 2; }
+
 cudaError_t proj_tc_set_attributes(int smem_optin) {
     if (TC_SMEM_TOTAL > smem_optin) return cudaErrorInvalidConfiguration;
-    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TC_EPI_QKV_ROPE_APPEND>,
+    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<TC_EPI_QKV_ROPE_APPEND, 2>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(proj_tc_kernel<TC_EPI_RESIDUAL_ADD>,
-                                cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(proj_tc_kernel<TC_EPI_QKV_ROPE_APPEND, 4>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(proj_tc_kernel<TC_EPI_RESIDUAL_ADD, 2>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(proj_tc_kernel<TC_EPI_RESIDUAL_ADD, 4>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL);
+    return e;
 }
 
 cudaError_t launch_qkv_rope_kv_append_tc(const CUtensorMap& w_map, const CUtensorMap& x_map, void* q_out,
@@ -490,8 +482,9 @@ cudaError_t launch_qkv_rope_kv_append_tc(const CUtensorMap& w_map, const CUtenso
     p.Hkv = Hkv;
     p.d = d;
     p.x_rows = proj_tc_batch_rows(B);
-    return launch_tc<TC_EPI_QKV_ROPE_APPEND>(w_map, x_map, p,
-                                             dim3(d / 64, Hq + 2 * Hkv, (B + p.x_rows - 1) / p.x_rows), stream);
+    return launch_tc<TC_EPI_QKV_ROPE_APPEND>(w_map, x_map, p, proj_tc_k_blocks(B),
+                                             dim3(d == 128 ? 3 : 2, Hq + 2 * Hkv, (B + p.x_rows - 1) / p.x_rows),
+                                             stream);
 }
 
 cudaError_t launch_oproj_residual_tc(const CUtensorMap& w_map, const CUtensorMap& x_map,
@@ -504,7 +497,7 @@ cudaError_t launch_oproj_residual_tc(const CUtensorMap& w_map, const CUtensorMap
     p.residual_in = static_cast<const uint16_t*>(residual_in);
     p.residual_out = static_cast<uint16_t*>(residual_out);
     p.x_rows = proj_tc_batch_rows(B);
-    return launch_tc<TC_EPI_RESIDUAL_ADD>(w_map, x_map, p, dim3(1, N / 64, (B + p.x_rows - 1) / p.x_rows), stream);
+    return launch_tc<TC_EPI_RESIDUAL_ADD>(w_map, x_map, p, proj_tc_k_blocks(B), dim3(1, N / 32, (B + p.x_rows - 1) / p.x_rows), stream);
 }
 
 }  // namespace ac

@@ -6,8 +6,9 @@
 // the request's cache slot.  Nothing but the final results touches global memory.
 //
 // The kernel is bound by streaming W once from HBM.  One CTA owns 16 rotary pairs of one head: W rows
-// i .. i+15 and i+d/2 .. i+d/2+15 (32 rows), all of K, one tile of up to 32 batch rows; the grid is
-// (d/32, Hq+2Hkv, ceil(B/32)) -- 192 CTAs for a 32/8-head, d=128 layer.  A producer warp issues, per
+// i .. i+15 and i+d/2 .. i+d/2+15 (32 rows), all of K, one tile of 8 or 16 batch rows (larger batches
+// run on the tcgen05 kernels); the grid is (d/32, Hq+2Hkv, batch tiles) -- 192 CTAs for a 32/8-head,
+// d=128 layer.  A producer warp issues, per
 // 256-wide K chunk, ONE 5-D tensor-map load for the 32 x 256 weight tile (the two row blocks and the
 // four 64-element K blocks are box dimensions, so the 16 KB land as eight swizzled [16 x 128 B]
 // blocks) and one 3-D load for the x tile, into a ring of stages guarded by full/empty mbarriers.
@@ -43,7 +44,7 @@ struct QkvSmem {
     static constexpr int X_BLOCK_BYTES = BT * 128;                 // [BT batch rows x 64 elements]
     static constexpr int X_STAGE_BYTES = KBLOCKS * X_BLOCK_BYTES;
     static constexpr int STAGE_BYTES = W_STAGE_BYTES + X_STAGE_BYTES;
-    static constexpr int STAGES = BT <= 8 ? 5 : (BT <= 16 ? 4 : 3);
+    static constexpr int STAGES = BT <= 8 ? 5 : 4;
     static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
     static constexpr int TOTAL = BAR_OFFSET + 2 * STAGES * 8 + 1024;
     static_assert(QKV_WARPS * 32 * BT * 4 <= STAGES * STAGE_BYTES, "reduction buffer must fit");
@@ -294,7 +295,7 @@ cudaError_t launch_qkv(const CUtensorMap& w_map, const CUtensorMap& x_map, const
 }  // namespace
 
 cudaError_t qkv_set_attributes(int smem_optin) {
-    if (QkvSmem<32>::TOTAL > smem_optin) return cudaErrorInvalidConfiguration;
+    if (QkvSmem<16>::TOTAL > smem_optin) return cudaErrorInvalidConfiguration;
     cudaError_t e;
 #define AC_SET(BT_, EPI_)                                                                          \
     e = cudaFuncSetAttribute(qkv_rope_append_kernel<BT_, EPI_>,                                    \
@@ -302,15 +303,15 @@ cudaError_t qkv_set_attributes(int smem_optin) {
     if (e != cudaSuccess) return e;
     AC_SET(8, EPI_QKV_ROPE_APPEND)
     AC_SET(16, EPI_QKV_ROPE_APPEND)
-    AC_SET(32, EPI_QKV_ROPE_APPEND)
     AC_SET(8, EPI_RESIDUAL_ADD)
     AC_SET(16, EPI_RESIDUAL_ADD)
-    AC_SET(32, EPI_RESIDUAL_ADD)
 #undef AC_SET
     return cudaSuccess;
 }
 
-int qkv_batch_tile(int B) { return B <= 8 ? 8 : (B <= 16 ? 16 : 32); }
+// Batch rows per CTA tile.  The library sends batches above 16 rows to the tcgen05 kernels; this kernel
+// would still serve them, 16 rows per grid slice.
+int qkv_batch_tile(int B) { return B <= 8 ? 8 : 16; }
 
 cudaError_t launch_qkv_rope_kv_append(const CUtensorMap& w_map, const CUtensorMap& x_map, void* q_out,
                                       void* k_cache, void* v_cache, int64_t stride_page,
@@ -346,8 +347,7 @@ cudaError_t launch_qkv_rope_kv_append(const CUtensorMap& w_map, const CUtensorMa
     p.N = 0;
     const int bt = qkv_batch_tile(B);
     if (bt == 8) return launch_qkv<8, EPI_QKV_ROPE_APPEND>(w_map, x_map, p, stream);
-    if (bt == 16) return launch_qkv<16, EPI_QKV_ROPE_APPEND>(w_map, x_map, p, stream);
-    return launch_qkv<32, EPI_QKV_ROPE_APPEND>(w_map, x_map, p, stream);
+    return launch_qkv<16, EPI_QKV_ROPE_APPEND>(w_map, x_map, p, stream);
 }
 
 // ---- RMSNorm of whole rows (second launch of the output-projection fusion) -------------------------
@@ -411,8 +411,7 @@ cudaError_t launch_oproj_residual(const CUtensorMap& w_map, const CUtensorMap& x
     p.residual_out = static_cast<uint16_t*>(residual_out);
     const int bt = qkv_batch_tile(B);
     if (bt == 8) return launch_qkv<8, EPI_RESIDUAL_ADD>(w_map, x_map, p, stream);
-    if (bt == 16) return launch_qkv<16, EPI_RESIDUAL_ADD>(w_map, x_map, p, stream);
-    return launch_qkv<32, EPI_RESIDUAL_ADD>(w_map, x_map, p, stream);
+    return launch_qkv<16, EPI_RESIDUAL_ADD>(w_map, x_map, p, stream);
 }
 
 cudaError_t launch_rmsnorm_rows(const void* h, const void* weight, void* out, int B, int N, float eps,

@@ -32,13 +32,16 @@ def _close_bf16(got_bits, ref_bits, what):
     (5, 320, 4, 4, 128, 16),          # K not a multiple of the 256-wide stage: zero-filled tail
     (8, 1024, 8, 2, 64, 16),
     (12, 512, 28, 4, 128, 32),        # batch tile of 16 with empty rows
-    (31, 768, 8, 2, 128, 16),         # batch tile of 32
-    (40, 256, 4, 2, 64, 16),          # two batch tiles
+    (16, 512, 8, 2, 128, 16),         # largest batch on the warp-MMA kernel
+    (17, 320, 8, 2, 128, 16),         # smallest batch on the tcgen05 kernel; K not a multiple of its 256-wide stage
+    (31, 768, 8, 2, 128, 16),
+    (40, 256, 4, 2, 64, 16),          # head_dim 64: two overlapping 24-pair tiles per head
     (4, 4096, 32, 8, 128, 16),        # 8B-class layer: 6144 x 4096 weights
-    (33, 256, 4, 2, 128, 16),         # smallest batch on the tcgen05 path; rows 33..127 of the tile are padding
-    (100, 512, 8, 2, 64, 16),
+    (33, 256, 4, 2, 128, 16),
+    (96, 512, 8, 2, 128, 16),         # widest batch tile that still takes 256-wide stages
+    (100, 512, 8, 2, 64, 16),         # 104-row tile, 128-wide stages
     (128, 1024, 8, 2, 128, 32),       # exactly one 128-row tile
-    (200, 320, 4, 4, 128, 16),        # two tiles, K not a multiple of the stage count
+    (200, 320, 4, 4, 128, 16),        # two tiles of 104 rows, K not a multiple of the stage width
     (64, 4096, 32, 8, 128, 16),       # 8B-class layer, batched
 ])
 def test_qkv_prelude_matches_oracle(B, H, Hq, Hkv, d, ps):
@@ -89,9 +92,46 @@ def test_qkv_prelude_matches_oracle(B, H, Hq, Hkv, d, ps):
     print(f"[prelude] B={B} H={H}: exact fraction of v = {ev:.4f}")
 
 
+@pytest.mark.parametrize("B", [8, 100])
+def test_qkv_prelude_bit_exact_when_the_projection_is_exact(B):
+    """Small-integer x and W make every dot product an integer that fp32 and fp64 both hold exactly, so
+    the projected bf16 features equal the oracle's and the rotation that follows can be held to the
+    oracle bit for bit -- on the warp-MMA kernel (B = 8) and on the tcgen05 kernel (B = 100), whose
+    epilogue rotates in fp32 and falls back to fp64 for the values it cannot prove (about one in a
+    thousand of the 128 000 rotations here)."""
+    import torch
+    from paper_2606_07665_b200 import binding as ac
+    from paper_2606_07665_b200 import build, runner
+    build.build()
+    torch.cuda.set_device(0)
+    ac.ac_init(0)
+    H, Hq, Hkv, d, ps = 256, 8, 2, 128, 16
+    rng = np.random.default_rng(4242 + B)
+    lens = rng.integers(0, 1500, size=B).tolist()
+    w = W.make_workload("prelude_exact", 300 + B, B=B, Hq=Hq, Hkv=Hkv, d=d, page_size=ps,
+                        num_pages=B * (1500 // ps + 2) + 4, context_lens=lens, rope_base=10000.0)
+    x = W.f32_to_bf16_bits(rng.integers(-2, 3, size=(B, H)).astype(np.float32))
+    wq = W.f32_to_bf16_bits(rng.integers(-2, 3, size=((Hq + 2 * Hkv) * d, H)).astype(np.float32))
+    q_ref, k_ref, v_ref = O.oracle_qkv_rope_kv_append(x, wq, w.k_cache, w.v_cache, w.block_table,
+                                                      w.context_lens, w.rope_cos, w.rope_sin, ps, Hq, Hkv, d)
+    st = runner.DecodeStep(w, num_splits=1)
+    ac.ac_qkv_rope_kv_append(torch.from_numpy(x.view(np.int16)).cuda(), torch.from_numpy(wq.view(np.int16)).cuda(),
+                             H, st.q_rot, st.k_cache, st.v_cache, st.stride_page, st.stride_token,
+                             st.stride_head, st.block_table, w.max_pages_per_seq, st.context_lens,
+                             st.rope_cos, st.rope_sin, w.max_position, B, Hq, Hkv, d, ps, w.num_pages,
+                             st.status_flag)
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) == 0
+    assert np.array_equal(runner.bits_of(st.q_rot), q_ref)
+    k_gpu, v_gpu = st.cache_bits()
+    assert np.array_equal(k_gpu, k_ref)
+    assert np.array_equal(v_gpu, v_ref)
+
+
 @pytest.mark.parametrize("B,K,N", [(1, 256, 64), (5, 320, 96), (8, 1024, 512), (13, 512, 256), (31, 768, 128),
                                    (40, 256, 64), (4, 4096, 4096), (33, 128, 64), (100, 512, 192), (128, 1024, 256),
-                                   (200, 320, 128), (40, 256, 96), (64, 4096, 4096)])
+                                   (200, 320, 128), (40, 256, 96), (64, 4096, 4096), (16, 512, 128), (17, 320, 96),
+                                   (96, 1024, 256)])
 def test_oproj_residual_rmsnorm_matches_oracle(B, K, N):
     import torch
     from paper_2606_07665_b200 import binding as ac
