@@ -169,10 +169,10 @@ int ac_rope_kv_append_ex(const void* q_in, void* q_out, const void* k_new, const
  * The projection is not bit-reproducible against an fp64 evaluation (fp32 accumulation order): its
  * bf16 results can differ from the correctly rounded ones by one unit in the last place; the
  * rotation and the stores are exact given those results.  Errors and status bits as
- * ac_rope_kv_append.  Up to 32 batch rows run on a warp-level MMA kernel that streams w_qkv once
- * from HBM; larger batches run on a tcgen05 kernel (batch tiles of 128 rows as the M dimension of
- * the instruction, accumulators in tensor memory) that streams w_qkv once per 128 rows.  Both give
- * the same results up to fp32 accumulation order. */
+ * ac_rope_kv_append.  Up to 16 batch rows run on a warp-level MMA kernel that streams w_qkv once
+ * from HBM; larger batches run on a tcgen05 kernel (batch tiles of up to 128 rows as the M dimension
+ * of the instruction, accumulators in tensor memory) that streams w_qkv once per 128 rows.  Both
+ * give the same results up to fp32 accumulation order. */
 int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out,
                           void* k_cache, void* v_cache,
                           int64_t stride_page, int64_t stride_token, int64_t stride_head,
@@ -192,7 +192,7 @@ int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out,
  * in its epilogue, then the row norm (it needs all N features of a row); the second starts under the
  * first one's tail.  The norm is exact given h (fp64 sum of squares, correctly rounded sqrt and
  * division); h can differ from the correctly rounded value by one bf16 step (fp32 accumulation).
- * As for ac_qkv_rope_kv_append, B > 32 with N % 64 == 0 runs the product on the tcgen05 kernel. */
+ * As for ac_qkv_rope_kv_append, B > 16 runs the product on the tcgen05 kernel. */
 int ac_oproj_residual_rmsnorm(const void* attn_out, const void* w_o, int K, int N,
                               const void* residual_in, void* residual_out,
                               const void* norm_weight, float norm_eps, void* normed_out,
