@@ -353,11 +353,12 @@ cudaError_t launch_qkv_rope_kv_append(const CUtensorMap& w_map, const CUtensorMa
 // ---- RMSNorm of whole rows (second launch of the output-projection fusion) -------------------------
 namespace {
 
-// NORM_SLICES CTAs per row: each recomputes the row's sum of squares in fp64 (exact for bf16 inputs
+// gridDim.x CTAs per row: each recomputes the row's sum of squares in fp64 (exact for bf16 inputs
 // of moderate range, so every CTA gets the same value; the row is a few KB and sits in L2) and
 // normalises its own slice: y = bf16(bf16(h / sqrt(mean + eps)) * w), the arithmetic of the per-head
-// norm of the prelude.
-constexpr int NORM_SLICES = 8;
+// norm of the prelude.  Few rows are cut into up to eight slices so that the launch still covers the
+// GPU; many rows need no slicing, and recomputing the sum eight times would only cost time.
+constexpr int NORM_MAX_SLICES = 8;
 
 __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const uint16_t* __restrict__ h,
                                                            const uint16_t* __restrict__ weight,
@@ -387,7 +388,7 @@ __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const uint16_t* __res
     const double r = __ddiv_rn(1.0, __dsqrt_rn(__dadd_rn(__ddiv_rn(total, static_cast<double>(N)),
                                                          static_cast<double>(eps))));
     uint16_t* orow = out + static_cast<size_t>(blockIdx.y) * N;
-    const int per = (N + NORM_SLICES - 1) / NORM_SLICES;
+    const int per = (N + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
     const int lo_i = blockIdx.x * per;
     const int hi_i = min(N, lo_i + per);
     for (int i = lo_i + threadIdx.x; i < hi_i; i += 256) {
@@ -417,7 +418,9 @@ cudaError_t launch_oproj_residual(const CUtensorMap& w_map, const CUtensorMap& x
 cudaError_t launch_rmsnorm_rows(const void* h, const void* weight, void* out, int B, int N, float eps,
                                 cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(NORM_SLICES, B);
+    int slices = (2 * 148 + B - 1) / B;                 // about two CTAs per SM in total
+    slices = slices < 1 ? 1 : (slices > NORM_MAX_SLICES ? NORM_MAX_SLICES : slices);
+    cfg.gridDim = dim3(slices, B);
     cfg.blockDim = dim3(256);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
