@@ -99,6 +99,17 @@ int ac_sm_count(void);
 int ac_decode_plan(int B, int Hq, int Hkv, int d, int page_size, int max_context_len, int sm_count,
                    int* num_splits_out, int* split_tokens_out, size_t* workspace_bytes_out);
 
+/* The same plan for a batch whose row lengths the caller knows (a scheduler builds context_lens on
+ * the host anyway).  token_counts_host[b] = tokens row b attends over this step (cached + new; <= 0
+ * for an inactive row), a HOST array of B entries; max_context_len >= every entry bounds the chunk
+ * grid as in ac_decode_plan (counts above it are clipped).  Splits that lie beyond a row's end launch
+ * CTAs that exit at once, so a ragged batch can afford more and shorter splits than its longest row
+ * alone suggests: the estimate counts only the CTAs that have tokens, the longest of them, and the
+ * batch's total bytes.  Same outputs and errors as ac_decode_plan; any plan gives the same results. */
+int ac_decode_plan_for_lengths(const int32_t* token_counts_host, int B, int Hq, int Hkv, int d,
+                               int page_size, int max_context_len, int sm_count,
+                               int* num_splits_out, int* split_tokens_out, size_t* workspace_bytes_out);
+
 /* Tokens per split the attention kernel uses for a given (max_context_len, num_splits): the smallest
  * multiple of 64 whose num_splits-fold covers max_context_len.  Host only, pure. */
 int ac_split_tokens(int max_context_len, int num_splits);

@@ -22,6 +22,7 @@ AC_FLAG_POSITION_OOB = 2
 AC_FLAG_WAIT_TIMEOUT = 4
 
 EXPORTS = ("ac_init", "ac_status_string", "ac_last_cuda_error", "ac_sm_count", "ac_decode_plan",
+           "ac_decode_plan_for_lengths",
            "ac_split_tokens", "ac_workspace_bytes", "ac_rope_kv_append", "ac_paged_decode_attn",
            "ac_splitkv_merge", "ac_decode_step_host", "ac_paged_decode_attn_static_scratch",
            "ac_fused_workspace_bytes", "ac_fused_workspace_reset", "ac_paged_decode_attn_fused_merge",
@@ -71,6 +72,9 @@ def lib():
         L.ac_sm_count.restype = c_int
         L.ac_decode_plan.argtypes = [c_int] * 7 + [POINTER(c_int), POINTER(c_int), POINTER(c_size_t)]
         L.ac_decode_plan.restype = c_int
+        L.ac_decode_plan_for_lengths.argtypes = ([c_void_p] + [c_int] * 7 +
+                                                 [POINTER(c_int), POINTER(c_int), POINTER(c_size_t)])
+        L.ac_decode_plan_for_lengths.restype = c_int
         L.ac_split_tokens.argtypes = [c_int, c_int]
         L.ac_split_tokens.restype = c_int
         L.ac_workspace_bytes.argtypes = [c_int] * 4
@@ -162,6 +166,18 @@ def ac_decode_plan(B, Hq, Hkv, d, page_size, max_context_len, sm_count=0):
     ns, st, wb = c_int(0), c_int(0), c_size_t(0)
     _check(lib().ac_decode_plan(B, Hq, Hkv, d, page_size, max_context_len, sm_count,
                                 ctypes.byref(ns), ctypes.byref(st), ctypes.byref(wb)), "ac_decode_plan")
+    return ns.value, st.value, wb.value
+
+
+def ac_decode_plan_for_lengths(token_counts, Hq, Hkv, d, page_size, max_context_len, sm_count=0):
+    """token_counts: host sequence of B ints (tokens each row attends over; <= 0 = inactive row).
+    Returns (num_splits, split_tokens, workspace_bytes)."""
+    counts = (ctypes.c_int32 * len(token_counts))(*[int(t) for t in token_counts])
+    ns, st, wb = c_int(0), c_int(0), c_size_t(0)
+    _check(lib().ac_decode_plan_for_lengths(ctypes.cast(counts, c_void_p), len(token_counts), Hq, Hkv, d,
+                                            page_size, max_context_len, sm_count, ctypes.byref(ns),
+                                            ctypes.byref(st), ctypes.byref(wb)),
+           "ac_decode_plan_for_lengths")
     return ns.value, st.value, wb.value
 
 

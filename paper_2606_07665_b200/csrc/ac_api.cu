@@ -184,8 +184,11 @@ size_t ac_workspace_bytes(int B, int Hq, int d, int num_splits) {
     return static_cast<size_t>(B) * Hq * num_splits * (static_cast<size_t>(d) + 1) * sizeof(float);
 }
 
-int ac_decode_plan(int B, int Hq, int Hkv, int d, int page_size, int max_context_len, int sm_count,
-                   int* num_splits_out, int* split_tokens_out, size_t* workspace_bytes_out) {
+// The plan proper.  token_counts == nullptr: every row is taken to attend over max_context_len
+// tokens; otherwise token_counts[b] = tokens row b attends over (<= 0: the row launches no work).
+static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_context_len, int sm_count,
+                       const int32_t* token_counts, int* num_splits_out, int* split_tokens_out,
+                       size_t* workspace_bytes_out) {
     if (num_splits_out == nullptr || split_tokens_out == nullptr || workspace_bytes_out == nullptr)
         return AC_ERR_NULL;
     Shape s{B, Hq, Hkv, d, page_size, 1};
@@ -200,29 +203,71 @@ int ac_decode_plan(int B, int Hq, int Hkv, int d, int page_size, int max_context
     //  * At least one wave of (request, KV head) pairs: do not split, unless contexts are long --
     //    then cut them into chunks of at most 4096 tokens so that ragged batches balance.
     //  * Fewer pairs than slots: scan the split counts and take the one with the smallest
-    //    estimated time, all rows assumed at max_context_len.
+    //    estimated time.  Without the rows' lengths every row counts as max_context_len tokens; with
+    //    them, a split that lies beyond a row's end costs nothing (its CTA exits at once), so a ragged
+    //    batch can take more, shorter splits before it spills into a second wave.
     const double slots = 2.0 * sm_count;
     const double hbm = 6.5e12 * sm_count / 148.0;      // bytes/s the whole GPU streams
     const double cta_rate = 33e9;                       // bytes/s one CTA streams on its own
     const double wave_cost = 3e-6;
-    const long long pairs = static_cast<long long>(B) * Hkv;
+    long long active_rows = B;
+    double total_tokens = static_cast<double>(B) * max_context_len;
+    if (token_counts != nullptr) {
+        active_rows = 0;
+        total_tokens = 0.0;
+        for (int b = 0; b < B; ++b)
+            if (token_counts[b] > 0) {
+                ++active_rows;
+                total_tokens += token_counts[b] < max_context_len ? token_counts[b] : max_context_len;
+            }
+        if (active_rows == 0) active_rows = 1;
+    }
+    const long long pairs = active_rows * Hkv;
     long long S = 1;
     if (pairs >= static_cast<long long>(slots)) {
         S = (static_cast<long long>(max_context_len) + 4095) / 4096;
     } else {
-        const int s_max = max_context_len / 256 > 1 ? max_context_len / 256 : 1;
+        int s_max = max_context_len / 256 > 1 ? max_context_len / 256 : 1;
+        if (s_max > 4096) s_max = 4096;
+        if (token_counts != nullptr && static_cast<long long>(s_max) * B > 4000000ll) {
+            s_max = static_cast<int>(4000000ll / B);      // bound the host work of the scan
+            if (s_max < 1) s_max = 1;
+        }
         double best = 0.0;
-        for (int cand = 1; cand <= s_max && cand <= 4096; ++cand) {
+        for (int cand = 1; cand <= s_max; ++cand) {
             const int chunk = split_tokens_for(max_context_len, cand);
             if (static_cast<long long>(chunk) * (cand - 1) >= max_context_len) continue;   // empty split
-            const double n = static_cast<double>(pairs) * cand;
-            const double c = static_cast<double>(chunk) * d * 4.0;          // K+V bytes of one CTA
+            double n = static_cast<double>(pairs) * cand;                // CTAs that have tokens
+            double longest = chunk;                                       // tokens of the longest CTA
+            if (token_counts != nullptr) {
+                long long pieces = 0;
+                int most = 0;
+                for (int b = 0; b < B; ++b) {
+                    int t = token_counts[b];
+                    if (t <= 0) continue;
+                    if (t > max_context_len) t = max_context_len;
+                    pieces += (t + chunk - 1) / chunk;
+                    const int m = t < chunk ? t : chunk;
+                    if (m > most) most = m;
+                }
+                n = static_cast<double>(pieces) * Hkv;
+                longest = most;
+            }
+            const double bytes_per_token = d * 4.0;                      // K + V of one KV head
             const double waves = ceil(n / slots);
-            const double last = n - (waves - 1.0) * slots;
-            double t = (waves - 1.0) * slots * c / hbm;
-            const double t_last_bw = last * c / hbm, t_last_cta = c / cta_rate;
-            t += (t_last_bw > t_last_cta ? t_last_bw : t_last_cta) + waves * wave_cost;
-            if (cand > 1) t += 2.0 * B * Hq * cand * (d + 1.0) * 4.0 / hbm + 1e-6;
+            double t;
+            if (token_counts == nullptr) {
+                const double c = longest * bytes_per_token;
+                const double last = n - (waves - 1.0) * slots;
+                t = (waves - 1.0) * slots * c / hbm;
+                const double t_last_bw = last * c / hbm, t_last_cta = c / cta_rate;
+                t += (t_last_bw > t_last_cta ? t_last_bw : t_last_cta) + waves * wave_cost;
+            } else {
+                const double t_bw = total_tokens * Hkv * bytes_per_token / hbm;
+                const double t_cta = longest * bytes_per_token / cta_rate;
+                t = (t_bw > t_cta ? t_bw : t_cta) + waves * wave_cost;
+            }
+            if (cand > 1) t += 2.0 * active_rows * Hq * cand * (d + 1.0) * 4.0 / hbm + 1e-6;
             if (best == 0.0 || t < best) {
                 best = t;
                 S = cand;
@@ -246,6 +291,20 @@ int ac_decode_plan(int B, int Hq, int Hkv, int d, int page_size, int max_context
     *split_tokens_out = split_tokens_for(max_context_len, static_cast<int>(S));
     *workspace_bytes_out = ac_workspace_bytes(B, Hq, d, static_cast<int>(S));
     return AC_OK;
+}
+
+int ac_decode_plan(int B, int Hq, int Hkv, int d, int page_size, int max_context_len, int sm_count,
+                   int* num_splits_out, int* split_tokens_out, size_t* workspace_bytes_out) {
+    return plan_splits(B, Hq, Hkv, d, page_size, max_context_len, sm_count, nullptr, num_splits_out,
+                       split_tokens_out, workspace_bytes_out);
+}
+
+int ac_decode_plan_for_lengths(const int32_t* token_counts_host, int B, int Hq, int Hkv, int d,
+                               int page_size, int max_context_len, int sm_count, int* num_splits_out,
+                               int* split_tokens_out, size_t* workspace_bytes_out) {
+    if (token_counts_host == nullptr) return AC_ERR_NULL;
+    return plan_splits(B, Hq, Hkv, d, page_size, max_context_len, sm_count, token_counts_host,
+                       num_splits_out, split_tokens_out, workspace_bytes_out);
 }
 
 int ac_rope_kv_append_ex(const void* q_in, void* q_out, const void* k_new, const void* v_new,

@@ -80,8 +80,10 @@ class DecodeStep:
         if self.window > 0:
             span = min(span, self.window + 63)         # tokens a row can attend over, as the kernel counts
         if num_splits is None:
-            num_splits, _, _ = ac.ac_decode_plan(self.B, self.Hq, self.Hkv, self.d, self.ps, span,
-                                                 ac.ac_sm_count())
+            # the lengths are on the host (the scheduler built context_lens from them): plan with them
+            counts = [min(int(n) + 1, span) if n >= 0 else 0 for n in self.w.context_lens]
+            num_splits, _, _ = ac.ac_decode_plan_for_lengths(counts, self.Hq, self.Hkv, self.d, self.ps,
+                                                             span, ac.ac_sm_count())
         self.num_splits = int(num_splits)
         self.split_tokens = ac.ac_split_tokens(span, self.num_splits)
         # sized for either merge flavour: partials, then the fused path's arrival counters

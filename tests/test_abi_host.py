@@ -67,6 +67,42 @@ def test_plan_properties(ac, B, Hq, Hkv, d, ps, maxlen):
         assert S > 1                                              # small batches are split across SMs
 
 
+def test_plan_for_lengths(ac):
+    import numpy as np
+    # every row at the maximum: the same plan as without lengths
+    for B, Hq, Hkv, d, ps, maxlen in [(1, 32, 8, 128, 16, 4097), (8, 28, 4, 128, 32, 2049), (4, 64, 8, 128, 16, 131073),
+                                      (64, 32, 8, 128, 16, 8193), (256, 28, 4, 128, 32, 2049)]:
+        assert ac.ac_decode_plan_for_lengths([maxlen] * B, Hq, Hkv, d, ps, maxlen, 148) == \
+            ac.ac_decode_plan(B, Hq, Hkv, d, ps, maxlen, 148)
+    # a ragged batch: splits beyond a row's end cost nothing, so the plan may split finer -- never coarser --
+    # and still leaves no split empty for the longest row
+    rng = np.random.default_rng(5)
+    for B, Hkv in [(32, 4), (16, 2), (8, 4), (48, 2)]:
+        lens = rng.integers(513, 2050, size=B).tolist()
+        maxlen = max(lens)
+        S0, _, _ = ac.ac_decode_plan(B, 4 * Hkv, Hkv, 128, 16, maxlen, 148)
+        S1, st1, wb1 = ac.ac_decode_plan_for_lengths(lens, 4 * Hkv, Hkv, 128, 16, maxlen, 148)
+        assert S1 >= S0
+        assert st1 == ac.ac_split_tokens(maxlen, S1) and st1 * (S1 - 1) < maxlen
+        assert wb1 == ac.ac_workspace_bytes(B, 4 * Hkv, 128, S1)
+        pieces = sum(-(-n // st1) for n in lens) * Hkv
+        assert S1 == 1 or st1 >= 256
+        assert S1 == S0 or pieces <= 2 * 148                      # the finer plan still fits one wave
+    # inactive rows launch nothing: they count neither as pairs nor as bytes
+    lens = [2000, 1800, 0, -1, 0, 0, 0, 0]
+    assert ac.ac_decode_plan_for_lengths(lens, 32, 8, 128, 16, 2000, 148)[0] == \
+        ac.ac_decode_plan_for_lengths(lens[:2], 32, 8, 128, 16, 2000, 148)[0]
+    # the graph-sweep bucket of 32 requests: three splits of 704 tokens instead of two of 1024
+    from paper_2606_07665_b200 import workloads as W
+    w = W.graph_sweep(32)
+    counts = [int(n) + 1 for n in w.context_lens]
+    assert ac.ac_decode_plan_for_lengths(counts, w.Hq, w.Hkv, w.d, w.page_size, w.max_context_len, 148)[:2] == (3, 704)
+    L = ac.lib()
+    ns, st, wb = ctypes.c_int(), ctypes.c_int(), ctypes.c_size_t()
+    assert L.ac_decode_plan_for_lengths(None, 4, 8, 2, 64, 16, 512, 148, ctypes.byref(ns), ctypes.byref(st),
+                                        ctypes.byref(wb)) == 1
+
+
 def test_plan_rejects_bad_shapes(ac):
     L = ac.lib()
     ns, st, wb = ctypes.c_int(), ctypes.c_int(), ctypes.c_size_t()
