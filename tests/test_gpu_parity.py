@@ -641,3 +641,48 @@ def test_workload_long_context_sampled_heads(rt, fused_step):
             gots.append(got[b, hq])
     check_out(np.array(gots), np.array(refs), "long_context sampled heads")
     assert np.isfinite(got).all()
+
+
+# ---------------------------------------------------------------------------------------------
+# Seeded random configurations: shapes, lengths, page sizes, layouts, splits, windows and launch
+# flavours drawn together, so that combinations nobody wrote down by hand are exercised as well.
+# ---------------------------------------------------------------------------------------------
+
+def _random_case(seed):
+    rng = np.random.default_rng(9000 + seed)
+    d = int(rng.choice([64, 128]))
+    Hkv = int(rng.choice([1, 2, 3, 4, 8]))
+    G = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 12, 16]))
+    ps = int(rng.choice([16, 32, 48, 64, 128]))
+    B = int(rng.integers(1, 10))
+    top = int(rng.choice([40, 300, 1500, 5000]))
+    lens = rng.integers(0, top + 1, size=B)
+    # sprinkle the boundaries: empty cache, one token, exact page and tile multiples
+    for b in range(B):
+        r = rng.random()
+        if r < 0.08:
+            lens[b] = 0
+        elif r < 0.16:
+            lens[b] = ps * int(rng.integers(1, 4)) - int(rng.integers(0, 2))
+        elif r < 0.24:
+            lens[b] = 16 * int(rng.integers(1, 9)) - 1
+    inactive = tuple(int(b) for b in range(B) if rng.random() < 0.12)
+    if len(inactive) == B:
+        inactive = inactive[1:]
+    pages = int(sum((int(n) + 1 + ps - 1) // ps for n in lens)) + int(rng.integers(2, 40))
+    w = W.make_workload(f"random{seed}", 9000 + seed, B=B, Hq=G * Hkv, Hkv=Hkv, d=d, page_size=ps,
+                        num_pages=pages, context_lens=lens.tolist(), rope_base=float(rng.choice([1e4, 5e5])),
+                        inactive_rows=inactive, peak_fraction=float(rng.choice([0.0, 0.02])))
+    max_len = int(lens.max()) + 1
+    splits = None if rng.random() < 0.3 else int(rng.integers(1, max(2, min(9, max_len // 64 + 2))))
+    layout = str(rng.choice(["token_major", "head_major"]))
+    fused = [False, True, "step"][int(rng.integers(0, 3))]
+    window = 0 if rng.random() < 0.6 else int(rng.integers(1, max_len + 40))
+    return w, splits, layout, fused, window
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_configurations_match_oracle(rt, seed):
+    w, splits, layout, fused, window = _random_case(seed)
+    run_and_compare(rt, w, num_splits=splits, layout=layout, fused=fused, window=window,
+                    check_cache=True)
