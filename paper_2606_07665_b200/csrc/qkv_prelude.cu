@@ -100,8 +100,11 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
         mbar_init_fence();
     }
     __syncthreads();
-    // x is produced by the kernel before this one; W and the tables are not.
-    cudaGridDependencySynchronize();
+    // x is produced by the kernel before this one; W is not.  The producer thread therefore sends the
+    // weight loads of the first ring fill on their way BEFORE it waits for that kernel (launched with
+    // programmatic stream serialization this CTA may be resident while the predecessor still runs),
+    // and everybody else waits here.
+    if (warp != QKV_WARPS) cudaGridDependencySynchronize();
 
     bool timed_out = false;
     float acc[2][NT][4];
@@ -117,9 +120,19 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
         if (lane == 0) {
             const uint64_t stream_once = l2_policy_evict_first();
             const uint64_t keep = l2_policy_evict_last();
-            for (int c = 0; c < n_chunks; ++c) {
+            const int first_fill = n_chunks < STAGES ? n_chunks : STAGES;
+            for (int c = 0; c < first_fill; ++c) {          // weights of the first ring fill
+                mbar_arrive_expect_tx(full_bar + c * 8, L::STAGE_BYTES);
+                tma_load_5d(smem_base + c * L::STAGE_BYTES, &w_map, full_bar + c * 8, 0, 16 * blk, 0, hh,
+                            c * KBLOCKS, stream_once);
+            }
+            cudaGridDependencySynchronize();
+            for (int c = 0; c < first_fill; ++c)             // their x tiles
+                tma_load_3d(smem_base + c * L::STAGE_BYTES + W_STAGE_BYTES, &x_map, full_bar + c * 8, 0, b0,
+                            c * KBLOCKS, keep);
+            for (int c = first_fill; c < n_chunks; ++c) {
                 const int stage = c % STAGES;
-                if (c >= STAGES && !mbar_wait_bounded(empty_bar + stage * 8, ((c / STAGES) - 1) & 1)) {
+                if (!mbar_wait_bounded(empty_bar + stage * 8, ((c / STAGES) - 1) & 1)) {
                     timed_out = true;
                     break;
                 }
@@ -128,6 +141,8 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
                 tma_load_5d(dst, &w_map, full_bar + stage * 8, 0, 16 * blk, 0, hh, c * KBLOCKS, stream_once);
                 tma_load_3d(dst + W_STAGE_BYTES, &x_map, full_bar + stage * 8, 0, b0, c * KBLOCKS, keep);
             }
+        } else {
+            cudaGridDependencySynchronize();               // the producer warp's other lanes
         }
     } else {
         // ---- consumers: warp w takes k-steps 2w and 2w+1 of every chunk ------------------------------
