@@ -686,3 +686,13 @@ def test_random_configurations_match_oracle(rt, seed):
     w, splits, layout, fused, window = _random_case(seed)
     run_and_compare(rt, w, num_splits=splits, layout=layout, fused=fused, window=window,
                     check_cache=True)
+
+
+def test_maximum_batch(rt):
+    """B = 65535, the largest batch the ABI accepts (grid.y limit): every row gets its own CTA."""
+    B = 65535
+    rng = np.random.default_rng(B)
+    lens = rng.integers(0, 21, size=B).tolist()
+    w = W.make_workload("max_batch", B, B=B, Hq=2, Hkv=1, d=64, page_size=16,
+                        num_pages=sum((n + 16) // 16 for n in lens) + 8, context_lens=lens, rope_base=10000.0)
+    run_and_compare(rt, w, fused="step")
