@@ -197,9 +197,11 @@ static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_con
     if (max_context_len <= 0) return AC_ERR_SHAPE;
     if (sm_count <= 0) sm_count = g_last_sm_count > 0 ? g_last_sm_count : 148;
 
-    // Two CTAs are resident per SM ("slots").  Measured on B200: one CTA streams at most ~35 GB/s
-    // (its ring holds 96 KB against ~2.5 us of load latency), a wave of CTAs costs ~3 us of
-    // ramp-up/epilogue that overlaps poorly, and every extra split adds partial-result traffic.
+    // Two CTAs are resident per SM ("slots").  Measured on B200: one CTA on its own streams ~45-57
+    // GB/s once its ring is full (96 KB in flight against ~2 us of load latency); charged with its
+    // own ramp that is ~33 GB/s over a short chunk, the figure fitted to sweeps of the split count.
+    // A wave of CTAs costs ~3 us of ramp-up/epilogue that overlaps poorly, and every extra split adds
+    // partial-result traffic.
     //  * At least one wave of (request, KV head) pairs: do not split, unless contexts are long --
     //    then cut them into chunks of at most 4096 tokens so that ragged batches balance.
     //  * Fewer pairs than slots: scan the split counts and take the one with the smallest
