@@ -238,7 +238,11 @@ int ac_paged_decode_attn(const void* q_rot, const void* k_cache, const void* v_c
  * (the "fused cross-CTA merging" of family (iv); Supplementary Implementation Notes: "a fused
  * fence-based merge that removes a separate reduction kernel").  Each CTA publishes its partial,
  * fences, and takes a ticket from a per-(request, KV head) arrival counter; the holder of the last
- * ticket merges and resets the counter.  No CTA ever waits for another.
+ * ticket merges and resets the counter.  No CTA ever waits for another.  When a pair's splits number
+ * at most 16 and the whole grid is resident at once, the launch instead makes each pair's splits one
+ * thread-block cluster: every CTA stages its partial in its own shared memory and the CTA of split 0
+ * reads them from there (distributed shared memory, two hardware cluster barriers; no partials in
+ * global memory, no ticket); the workspace contract is the same either way.
  *
  * Arguments as ac_paged_decode_attn, except: out is always written; for num_splits > 1 the workspace
  * must hold ac_fused_workspace_bytes(B,Hq,Hkv,d,num_splits) bytes = the partials followed by int32

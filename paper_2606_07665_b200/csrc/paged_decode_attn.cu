@@ -83,7 +83,35 @@ struct AttnParams {
     const int32_t* row_order;     // optional [B] permutation: grid row y serves request row_order[y]
     int longest_first;            // 1: grid row y serves the request with the y-th longest context
     int window;                   // > 0: attend over the last `window` tokens of each row only
+    int cluster_merge;            // 1: the splits of a (request, KV head) are one thread-block cluster and
+                                  //    split 0 merges them out of the others' shared memory
 };
+
+// ---- thread-block cluster helpers (fused merge through distributed shared memory) ------------------
+__device__ __forceinline__ uint32_t cluster_map_shared(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;                   // address of the same shared-memory location in CTA `rank` of the cluster
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float4 cluster_load_f32x4(uint32_t cluster_addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(cluster_addr)
+                 : "memory");
+    return v;
+}
+__device__ __forceinline__ float cluster_load_f32(uint32_t cluster_addr) {
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
+    return v;
+}
+// Hardware barrier over the threads of the cluster (not a spin).  Every CTA of a cluster-merge launch
+// executes exactly two of them, on every path.
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
 template <int D, bool WIDE, bool ROPE>
 __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
@@ -189,6 +217,12 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
         } else {
             uint16_t* o = p.out + (static_cast<size_t>(b) * p.Hq + h * G) * D;
             for (int e = threadIdx.x; e < G * D; e += THREADS) o[e] = 0;
+        }
+        if (p.cluster_merge != 0 && S > 1) {
+            // Cluster merge: keep step with the two cluster barriers of the CTAs that have tokens
+            // (this CTA stages nothing and nobody reads its shared memory).
+            cluster_sync_all();
+            cluster_sync_all();
         }
         return;
     }
@@ -543,6 +577,17 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     float* wm = wo + WROWS * WSTRIDE;                                           // [WROWS]
     float* wl = wm + WROWS;                                                     // [WROWS]
     static_assert((WROWS * WSTRIDE + 2 * WROWS) * 4 <= L::RING_BYTES, "merge scratch must fit in a ring");
+    // Cluster merge: this CTA's normalised result is staged behind the warps' scratch, eight query rows
+    // per ring (rows 0-7 in ring 0, rows 8-15 in ring 1): [8][D] fp32, then the 8 log-sum-exps.
+    constexpr int STAGE_OFF = (WROWS * WSTRIDE + 2 * WROWS) * 4;
+    static_assert(STAGE_OFF % 16 == 0 && STAGE_OFF + 8 * D * 4 + 8 * 4 <= L::RING_BYTES, "staged result must fit");
+    auto staged_o = [&](int row, int col) {       // byte offset from smem_base
+        return static_cast<uint32_t>((row >> 3) * L::RING_BYTES + STAGE_OFF + ((row & 7) * D + col) * 4);
+    };
+    auto staged_lse = [&](int row) {
+        return static_cast<uint32_t>((row >> 3) * L::RING_BYTES + STAGE_OFF + 8 * D * 4 + (row & 7) * 4);
+    };
+    const bool cluster_merge = p.cluster_merge != 0 && S > 1;
 #pragma unroll
     for (int r = 0; r < ROWS; ++r) {
         float l = l_run[r];
@@ -581,6 +626,9 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
         const size_t hq = static_cast<size_t>(b) * p.Hq + h * G + row;
         if (S == 1) {
             p.out[hq * D + col] = static_cast<uint16_t>(pack_bf16x2(val, 0.0f) & 0xFFFFu);
+        } else if (cluster_merge) {
+            *reinterpret_cast<float*>(smem_gen + staged_o(row, col)) = val;
+            if (col == 0) *reinterpret_cast<float*>(smem_gen + staged_lse(row)) = (M + log2f(den)) * LN2;
         } else {
             p.partial_o[(hq * S + split) * D + col] = val;
             if (col == 0) p.partial_lse[hq * S + split] = (M + log2f(den)) * LN2;
@@ -588,6 +636,51 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     }
 
     if (S == 1 || !p.fused_merge) return;
+
+    if (cluster_merge) {
+        // ---- fused merge inside a cluster: split 0 reads the other splits' staged results out of
+        // their shared memory.  No global round trip, no ticket; CTAs whose split has no tokens pass
+        // through the same two barriers and nothing else.
+        const int n_active = (n_tokens - window_base + p.split_tokens - 1) / p.split_tokens;   // <= 16
+        cluster_sync_all();                              // every staged result is written and visible
+        if (split == 0) {
+            constexpr int D4 = D / 4;
+            const size_t hq0 = static_cast<size_t>(b) * p.Hq + h * G;
+            for (int e = threadIdx.x; e < G * D4; e += THREADS) {
+                const int row = e / D4;
+                const int c4 = e - row * D4;
+                const uint32_t o_addr = smem_base + staged_o(row, c4 * 4);
+                const uint32_t l_addr = smem_base + staged_lse(row);
+                float4 v[16];
+                float l[16];
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {           // all loads first: one round trip
+                    const bool on = u < n_active;
+                    l[u] = on ? cluster_load_f32(cluster_map_shared(l_addr, u)) : -INFINITY;
+                    v[u] = on ? cluster_load_f32x4(cluster_map_shared(o_addr, u)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                float M = -INFINITY;
+#pragma unroll
+                for (int u = 0; u < 16; ++u) M = fmaxf(M, l[u]);
+                float den = 0.0f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {
+                    const float wgt = __expf(l[u] - M);  // 0 for the padding entries
+                    acc.x = fmaf(wgt, v[u].x, acc.x);
+                    acc.y = fmaf(wgt, v[u].y, acc.y);
+                    acc.z = fmaf(wgt, v[u].z, acc.z);
+                    acc.w = fmaf(wgt, v[u].w, acc.w);
+                    den += wgt;
+                }
+                const float inv = 1.0f / den;
+                *reinterpret_cast<uint2*>(p.out + (hq0 + row) * D + c4 * 4) =
+                    make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
+            }
+        }
+        cluster_sync_all();                              // nobody's shared memory goes away before it was read
+        return;
+    }
 
     // ---- fused merge: the CTA that arrives last for this (request, KV head) combines the splits ----
     // Publish this CTA's partials, take a ticket, and let the holder of the last ticket do the merge.
@@ -654,9 +747,12 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     }
 }
 
+constexpr int kClusterMergeMaxSplits = 16;           // largest (non-portable) cluster size
+
 template <int D, bool WIDE, bool ROPE>
-cudaError_t launch_one(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnParams& p, int B,
+cudaError_t launch_one(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnParams& p_in, int B,
                        cudaStream_t stream) {
+    AttnParams p = p_in;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.Hkv, B, p.num_splits);
     cfg.blockDim = dim3(THREADS);
@@ -665,11 +761,36 @@ cudaError_t launch_one(const CUtensorMap& k_map, const CUtensorMap& v_map, const
     // Programmatic dependent launch: this kernel may start while the preceding kernel of the
     // stream is still running; it calls cudaGridDependencySynchronize() before touching anything
     // that kernel produces.
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;    // the splits of a (request, KV head)
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = static_cast<unsigned>(p.num_splits);
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    if (p.cluster_merge) {
+        // A cluster is placed inside one GPC, so fewer clusters than CTA slots / cluster size may be
+        // resident at once (9-CTA clusters: 28 on a 148-SM part, not 32).  The cluster merge is used
+        // only when every cluster of the grid is resident together; the answer per split count is
+        // asked of the runtime once and remembered (benign race: every thread stores the same value).
+        static int max_clusters[kMaxDevices][kClusterMergeMaxSplits + 1];     // 0 = not asked yet
+        int dev = 0;
+        cudaGetDevice(&dev);
+        int& known = max_clusters[dev < kMaxDevices ? dev : 0][p.num_splits];
+        if (known == 0) {
+            int n = 0;
+            cfg.numAttrs = 2;
+            const cudaError_t qe = cudaOccupancyMaxActiveClusters(&n, paged_decode_attn_kernel<D, WIDE, ROPE>, &cfg);
+            if (qe != cudaSuccess) {
+                cudaGetLastError();
+                n = 0;
+            }
+            known = n > 0 ? n : -1;
+        }
+        if (static_cast<long long>(B) * p.Hkv > known) p.cluster_merge = 0;
+    }
+    cfg.numAttrs = p.cluster_merge ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, paged_decode_attn_kernel<D, WIDE, ROPE>, k_map, v_map, p);
 }
 
@@ -684,6 +805,12 @@ cudaError_t attn_set_attributes(int smem_optin) {
     if (e != cudaSuccess) return e;                                                                \
     e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, true>,                               \
                              cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D_>::TOTAL);        \
+    if (e != cudaSuccess) return e;                                                                \
+    e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, false>,                              \
+                             cudaFuncAttributeNonPortableClusterSizeAllowed, 1);                   \
+    if (e != cudaSuccess) return e;                                                                \
+    e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, true>,                               \
+                             cudaFuncAttributeNonPortableClusterSizeAllowed, 1);                   \
     if (e != cudaSuccess) return e;
     AC_SET(128, false)
     AC_SET(128, true)
@@ -734,6 +861,11 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
     sms = device_state(dev).sm_count;
     p.longest_first = (B > 1 && B <= kLongestFirstMaxBatch &&
                        static_cast<long long>(B) * Hkv * num_splits > 2ll * sms) ? 1 : 0;
+    // Merge inside a cluster when the splits of a (request, KV head) fit in one cluster and the whole
+    // grid is resident at once (clusters are scheduled as a unit; in a grid several waves deep that
+    // would cost more at the tail than the merge saves).
+    p.cluster_merge = (p.fused_merge && num_splits >= 2 && num_splits <= kClusterMergeMaxSplits &&
+                       static_cast<long long>(B) * Hkv * num_splits <= 2ll * sms) ? 1 : 0;
     p.q = static_cast<const uint16_t*>(q_rot);
     p.block_table = block_table;
     p.context_lens = context_lens;
