@@ -861,11 +861,13 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
     sms = device_state(dev).sm_count;
     p.longest_first = (B > 1 && B <= kLongestFirstMaxBatch &&
                        static_cast<long long>(B) * Hkv * num_splits > 2ll * sms) ? 1 : 0;
-    // Merge inside a cluster when the splits of a (request, KV head) fit in one cluster and the whole
-    // grid is resident at once (clusters are scheduled as a unit; in a grid several waves deep that
-    // would cost more at the tail than the merge saves).
+    // Merge inside a cluster when the splits of a (request, KV head) fit in one cluster and the grid
+    // has no more CTAs than the GPU has SMs.  Clusters are scheduled as a unit inside one GPC: on a
+    // fuller GPU some of them wait for a second wave even where the occupancy query says they all
+    // fit (32 clusters of 8 CTAs measured 53 us against 35 us with the ticket merge), which costs far
+    // more than the merge saves; small grids are where the merge's latency matters anyway.
     p.cluster_merge = (p.fused_merge && num_splits >= 2 && num_splits <= kClusterMergeMaxSplits &&
-                       static_cast<long long>(B) * Hkv * num_splits <= 2ll * sms) ? 1 : 0;
+                       static_cast<long long>(B) * Hkv * num_splits <= sms) ? 1 : 0;
     p.q = static_cast<const uint16_t*>(q_rot);
     p.block_table = block_table;
     p.context_lens = context_lens;
