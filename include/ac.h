@@ -90,7 +90,7 @@ int ac_sm_count(void);
  * (request, KV head) pairs alone fill the GPU and contexts are short, chunks of at most 4096 tokens
  * when contexts are long, and otherwise the split count with the smallest estimated time from a
  * small cost model (bandwidth of one CTA, waves of CTAs, partial-result traffic); splits are never
- * shorter than 256 tokens.  max_context_len = the largest number of tokens any row attends over in this bucket
+ * shorter than 256 tokens, or 128 where the grid is small enough for the merge inside a cluster.  max_context_len = the largest number of tokens any row attends over in this bucket
  * (cached + new).  Outputs: *num_splits_out >= 1, *split_tokens_out = tokens per split (a multiple
  * of 64; split s of row b covers tokens [s*split_tokens, min((s+1)*split_tokens, n_b)) ), and
  * *workspace_bytes_out = bytes of fp32 workspace the attention + merge calls need for that plan

@@ -229,7 +229,9 @@ static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_con
     if (pairs >= static_cast<long long>(slots)) {
         S = (static_cast<long long>(max_context_len) + 4095) / 4096;
     } else {
-        int s_max = max_context_len / 256 > 1 ? max_context_len / 256 : 1;
+        // Splits are at least 256 tokens long -- 128 where the merge is the cheap one inside a cluster
+        // (small grids, where nothing but latency is at stake).
+        int s_max = (max_context_len + 63) / 64;            // the chunk-length test below does the limiting
         if (s_max > 4096) s_max = 4096;
         if (token_counts != nullptr && static_cast<long long>(s_max) * B > 4000000ll) {
             s_max = static_cast<int>(4000000ll / B);      // bound the host work of the scan
@@ -239,6 +241,8 @@ static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_con
         for (int cand = 1; cand <= s_max; ++cand) {
             const int chunk = split_tokens_for(max_context_len, cand);
             if (static_cast<long long>(chunk) * (cand - 1) >= max_context_len) continue;   // empty split
+            const bool in_cluster = cand <= kClusterMergeMaxSplits && pairs * cand <= sm_count;
+            if (cand > 1 && chunk < (in_cluster ? 128 : 256)) continue;
             double n = static_cast<double>(pairs) * cand;                // CTAs that have tokens
             double longest = chunk;                                       // tokens of the longest CTA
             if (token_counts != nullptr) {
@@ -269,7 +273,8 @@ static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_con
                 const double t_cta = longest * bytes_per_token / cta_rate;
                 t = (t_bw > t_cta ? t_bw : t_cta) + waves * wave_cost;
             }
-            if (cand > 1) t += 2.0 * active_rows * Hq * cand * (d + 1.0) * 4.0 / hbm + 1e-6;
+            if (cand > 1)            // partials out and back in plus the ticket round trip, or two cluster barriers
+                t += in_cluster ? 0.3e-6 : 2.0 * active_rows * Hq * cand * (d + 1.0) * 4.0 / hbm + 1.6e-6;
             if (best == 0.0 || t < best) {
                 best = t;
                 S = cand;

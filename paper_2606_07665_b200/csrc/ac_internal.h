@@ -11,6 +11,9 @@
 namespace ac {
 
 constexpr int kMaxDevices = 64;
+// Fused merge inside a thread-block cluster: used when a (request, KV head)'s splits number at most
+// this many and the grid has no more CTAs than the GPU has SMs (the plan prices it accordingly).
+constexpr int kClusterMergeMaxSplits = 16;
 
 struct DeviceState {
     bool ready = false;

@@ -747,8 +747,6 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     }
 }
 
-constexpr int kClusterMergeMaxSplits = 16;           // largest (non-portable) cluster size
-
 template <int D, bool WIDE, bool ROPE>
 cudaError_t launch_one(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnParams& p_in, int B,
                        cudaStream_t stream) {
