@@ -17,9 +17,11 @@
 //   warp 0   producer: per 128-wide K chunk one 3-D TMA load of the x tile [x_rows x 2 x 64] and one
 //            5-D TMA load of the W tile, both as 128-byte-swizzled K-major blocks, into a ring that is
 //            as deep as shared memory allows (256 contiguous bytes of every W row per load);
-//   warp 1   allocates the TMEM columns, and its lane 0 issues eight tcgen05.mma (M128, K16, bf16 ->
-//            fp32) per chunk from shared-memory descriptors, then tcgen05.commit to hand the stage back
-//            to the producer, and a final commit to release the epilogue;
+//   warp 1   allocates the TMEM columns; its lane 0 and lane 0 of the last warp issue the tcgen05.mma
+//            (M128, K16, bf16 -> fp32, eight or sixteen per chunk) from shared-memory descriptors, the
+//            first the even chunks into one accumulator, the second the odd chunks into another, then
+//            tcgen05.commit to hand the stage back to the producer, and a final commit each to release
+//            the epilogue, which adds the two accumulators;
 //   the other warps are the epilogue, one warp per 32 batch rows and group of columns (thread = one
 //            batch row; 8 rotary pairs or 16 output features): they compute addresses and fetch angles
 //            or residuals while the main loop runs, then read the accumulator with tcgen05.ld, round
@@ -47,9 +49,11 @@ template <int EPI>
 struct TcTile {
     static constexpr int N = EPI == TC_EPI_QKV_ROPE_APPEND ? 48 : 32;        // features per CTA
     static constexpr int GROUPS = EPI == TC_EPI_QKV_ROPE_APPEND ? 3 : 2;     // epilogue warps per 32 rows
-    static constexpr int THREADS = 64 + 128 * GROUPS;
+    static constexpr int THREADS = 64 + 128 * GROUPS + 32;       // the last warp holds the second MMA issuer
+    static constexpr int MMA2_WARP = 2 + 4 * GROUPS;
     static constexpr int B_BLOCK = N * 128;          // one swizzled [N rows x 128 B] block of W
-    static constexpr uint32_t TMEM_COLS = EPI == TC_EPI_QKV_ROPE_APPEND ? 64 : 32;   // a power of two >= N
+    static constexpr uint32_t ACC_COLS = EPI == TC_EPI_QKV_ROPE_APPEND ? 64 : 32;    // a power of two >= N
+    static constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;                              // two accumulators
 };
 
 // First rotary pair of QKV tile `blk` inside its head: 24-pair tiles at 0, 16, 40 (64 pairs per head)
@@ -182,7 +186,7 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
             mbar_init(full_bar + s * 8, 1);
             mbar_init(empty_bar + s * 8, 1);
         }
-        mbar_init(done_bar, 1);
+        mbar_init(done_bar, 2);                              // one arrival per MMA-issuing thread
         mbar_init_fence();
     }
     if (warp == 1) tmem_alloc(tmem_slot, T::TMEM_COLS);
@@ -214,9 +218,16 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
                 }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || warp == T::MMA2_WARP) {
+        // Two threads issue the MMAs, one the even chunks into the first accumulator, one the odd chunks
+        // into the second (the epilogue adds them): a thread is held ~75 cycles per tcgen05.mma however
+        // narrow the tile, several times the tensor pipe's own time here.  BOTH threads wait for EVERY
+        // chunk's full barrier, in order: a thread that skipped the barriers of the other's chunks could
+        // run a whole phase ahead of a stage, which a one-bit parity wait cannot tell from being on time.
         if (lane == 0) {
+            const int which = warp == 1 ? 0 : 1;
             const uint32_t idesc = umma_idesc_bf16_m128(T::N);
+            const uint32_t acc = tmem_d + which * T::ACC_COLS;
             int stage = 0;
             uint32_t round = 0;
             for (int c = 0; c < n_chunks; ++c) {
@@ -224,29 +235,30 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
                     timed_out = true;
                     break;
                 }
-                tc_fence_after_sync();
-                const uint32_t a_addr = smem_base + stage * stage_bytes;
+                if ((c & 1) == which) {
+                    tc_fence_after_sync();
+                    const uint32_t a_addr = smem_base + stage * stage_bytes;
 #pragma unroll
-                for (int kb = 0; kb < KBLK; ++kb) {
-                    const uint64_t adesc = umma_desc_k_major_sw128(a_addr + kb * a_block);
-                    const uint64_t bdesc = umma_desc_k_major_sw128(a_addr + a_bytes + kb * T::B_BLOCK);
+                    for (int kb = 0; kb < KBLK; ++kb) {
+                        const uint64_t adesc = umma_desc_k_major_sw128(a_addr + kb * a_block);
+                        const uint64_t bdesc = umma_desc_k_major_sw128(a_addr + a_bytes + kb * T::B_BLOCK);
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)           // 16 elements = 32 bytes = 2 descriptor units
-                        umma_bf16(tmem_d, adesc + 2 * ks, bdesc + 2 * ks, idesc,
-                                  (c > 0 || kb > 0 || ks > 0) ? 1u : 0u);
+                        for (int ks = 0; ks < 4; ++ks)       // 16 elements = 32 bytes = 2 descriptor units
+                            umma_bf16(acc, adesc + 2 * ks, bdesc + 2 * ks, idesc, (c > 1 || kb > 0 || ks > 0) ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar + stage * 8);      // the stage is free once these MMAs have read it
                 }
-                umma_commit(empty_bar + stage * 8);          // the stage is free once these MMAs have read it
                 if (++stage == stages) {
                     stage = 0;
                     ++round;
                 }
             }
-            umma_commit(done_bar);                           // accumulator complete (or as far as we got)
+            umma_commit(done_bar);                           // this thread's accumulator is complete (or as far as it got)
         }
     }
     if (timed_out && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_WAIT_TIMEOUT);
 
-    if (warp >= 2) {
+    if (warp >= 2 && warp < T::MMA2_WARP) {
         // ---- epilogue: thread = batch row; warp = 32 rows x one group of columns --------------------
         // Everything that does not need the accumulator is done first, under the main loop.
         const int quarter = warp & 3;                        // TMEM lanes this warp may read
@@ -269,10 +281,19 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
             const bool ready = mbar_wait_bounded(done_bar, 0);
             if (!ready && lane == 0 && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_WAIT_TIMEOUT);
             tc_fence_after_sync();
-            uint32_t acc[2][8];
+            uint32_t acc[2][8], odd[2][8];
             tmem_ld_32x8(lane_base + 16 * group, acc[0]);
             tmem_ld_32x8(lane_base + 16 * group + 8, acc[1]);
+            tmem_ld_32x8(lane_base + T::ACC_COLS + 16 * group, odd[0]);           // the odd chunks' sums
+            tmem_ld_32x8(lane_base + T::ACC_COLS + 16 * group + 8, odd[1]);
             tmem_ld_wait();
+            if (n_chunks > 1) {                              // a single chunk leaves the second accumulator unwritten
+#pragma unroll
+                for (int v = 0; v < 2; ++v)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        acc[v][e] = __float_as_uint(__uint_as_float(acc[v][e]) + __uint_as_float(odd[v][e]));
+            }
             if (ready && ok) {
 #pragma unroll
                 for (int v = 0; v < 2; ++v) {                // 8 features = 16 bytes at a time
@@ -343,10 +364,19 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
             const bool ready = mbar_wait_bounded(done_bar, 0);
             if (!ready && lane == 0 && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_WAIT_TIMEOUT);
             tc_fence_after_sync();
-            uint32_t lo[8], hi[8];
+            uint32_t lo[8], hi[8], lo_odd[8], hi_odd[8];
             tmem_ld_32x8(lane_base + 8 * group, lo);                 // first halves of pairs i0 .. i0 + 7
             tmem_ld_32x8(lane_base + T::N / 2 + 8 * group, hi);      // their second halves
+            tmem_ld_32x8(lane_base + T::ACC_COLS + 8 * group, lo_odd);                // the odd chunks' sums
+            tmem_ld_32x8(lane_base + T::ACC_COLS + T::N / 2 + 8 * group, hi_odd);
             tmem_ld_wait();
+            if (n_chunks > 1) {                              // a single chunk leaves the second accumulator unwritten
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    lo[e] = __float_as_uint(__uint_as_float(lo[e]) + __uint_as_float(lo_odd[e]));
+                    hi[e] = __float_as_uint(__uint_as_float(hi[e]) + __uint_as_float(hi_odd[e]));
+                }
+            }
             if (ready && ok) {
                 uint16_t lo8[8], hi8[8];
                 float af[8], bf[8];
@@ -432,9 +462,10 @@ int proj_tc_batch_rows(int B) {
     return rows < TC_M ? rows : TC_M;
 }
 
-// K blocks per stage: loads of 512 contiguous bytes per weight row stream measurably faster than loads
-// of 256, but only while at least three stages still fit beside the x tiles.
-int proj_tc_k_blocks(int B) { return proj_tc_batch_rows(B) <= 96 ? 4 : 2; }
+// K blocks per stage: 256-wide stages (sixteen MMAs per barrier round trip, 512 contiguous bytes per
+// weight row and load) are faster, but only while at least five of them fit beside the x tiles -- with
+// two threads issuing MMAs two stages are being read at any time, and the rest must cover the loads.
+int proj_tc_k_blocks(int B) { return proj_tc_batch_rows(B) <= 40 ? 4 : 2; }
 
 cudaError_t proj_tc_set_attributes(int smem_optin) {
     if (TC_SMEM_TOTAL > smem_optin) return cudaErrorInvalidConfiguration;
