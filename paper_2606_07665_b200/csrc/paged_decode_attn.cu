@@ -7,9 +7,9 @@
 // 128-byte swizzle, so ldmatrix reads are free of bank conflicts.  (Issuing a tensor load costs the
 // issuing thread on the order of 100 ns, so the number of loads per tile matters: splitting head_dim
 // into the innermost 64 elements and an outer block index keeps the swizzle span at 128 bytes while
-// still fetching the whole 256-byte rows with one instruction.)  Every warp runs its own ring of STAGES tiles with one mbarrier per stage and takes
-// tiles warp, warp+WARPS, ... of the CTA's token range; there is no CTA-wide synchronisation in the
-// main loop.  The physical page id of a tile is fetched from the block table one tile ahead of the
+// still fetching the whole 256-byte rows with one instruction.)  Every warp runs its own ring of
+// STAGES tiles with one mbarrier per stage and takes tiles warp, warp+WARPS, ... of the CTA's token
+// range; there is no CTA-wide synchronisation in the main loop.  The physical page id of a tile is fetched from the block table one tile ahead of the
 // TMA issue that needs it.  KV bytes are read once, so the loads carry an evict-first L2 policy.
 //
 // Arithmetic.  The Hq/Hkv query heads of the group are the rows of a 16-row MMA tile (rows >= group
@@ -19,6 +19,10 @@
 // warp-shuffle reductions across the four lanes that share a row.  At the end the warps' partial
 // (max, sum, O) are combined through shared memory and the CTA writes either the final bf16 row
 // (one split) or its normalised fp32 partial plus the natural-log log-sum-exp (several splits).
+// With the fused merge the splits of a (request, KV head) are combined inside this kernel: by the CTA
+// that arrives last (ticket on a global counter, partials through global memory), or, for grids of
+// at most one CTA per SM, by the CTA of split 0 of a thread-block cluster that reads the other splits'
+// results out of their shared memory.
 //
 // With a group of 4-8 query rows the path needs G flop per KV byte; at HBM speed that exceeds what
 // the fp32 pipes deliver for G >= 7, which is why the products run on the tensor pipe even though
