@@ -334,7 +334,8 @@ int ac_splitkv_merge(const void* workspace, int num_splits, const int32_t* conte
  * end-to-end timing): copies q/k_new/v_new/block_table/context_lens from the *_host buffers (pinned
  * memory recommended) into the caller's device buffers of the same name, resets the arrival
  * counters, enqueues ac_decode_step_fused for the given num_splits (workspace_bytes >=
- * ac_fused_workspace_bytes), and copies the bf16 result from out into out_host.  When the host
+ * ac_fused_workspace_bytes), and delivers the bf16 result in out AND out_host (when out_host is pinned
+ * memory the GPU can address, the kernel's final stores go to both; otherwise a copy from out follows).  When the host
  * buffers are pinned memory the GPU can address and their sizes are multiples of 16 bytes, the five
  * inputs are gathered (and the counters cleared) by ONE small kernel reading host memory directly
  * instead of five copy-engine transfers; otherwise each buffer gets its own cudaMemcpyAsync.  Everything is asynchronous on `stream`; the caller

@@ -641,14 +641,15 @@ int ac_decode_step_fused(const void* q_in, void* q_rot_out, const void* k_new, c
                                    num_pages, max_context_len, status_flag, stream, nullptr);
 }
 
-int ac_decode_step_fused_ex(const void* q_in, void* q_rot_out, const void* k_new, const void* v_new,
-                            void* k_cache, void* v_cache, int64_t stride_page, int64_t stride_token,
-                            int64_t stride_head, const int32_t* block_table, int max_pages_per_seq,
-                            const int32_t* context_lens, const float* rope_cos, const float* rope_sin,
-                            int max_position, float softmax_scale, int num_splits, void* workspace,
-                            size_t workspace_bytes, void* out, int B, int Hq, int Hkv, int d,
-                            int page_size, int num_pages, int max_context_len, int32_t* status_flag,
-                            void* stream, const ac_attn_options* options) {
+// The fused step with an optional mirror of the result (a second destination for every store to out).
+static int decode_step_fused_impl(const void* q_in, void* q_rot_out, const void* k_new, const void* v_new,
+                                  void* k_cache, void* v_cache, int64_t stride_page, int64_t stride_token,
+                                  int64_t stride_head, const int32_t* block_table, int max_pages_per_seq,
+                                  const int32_t* context_lens, const float* rope_cos, const float* rope_sin,
+                                  int max_position, float softmax_scale, int num_splits, void* workspace,
+                                  size_t workspace_bytes, void* out, int B, int Hq, int Hkv, int d,
+                                  int page_size, int num_pages, int max_context_len, int32_t* status_flag,
+                                  void* stream, const ac_attn_options* options, void* out_mirror) {
     const int window = options != nullptr ? options->window : 0;
     const int32_t* row_order = options != nullptr ? options->row_order : nullptr;
     if (!q_in || !k_new || !v_new || !rope_cos || !rope_sin) return AC_ERR_NULL;
@@ -670,10 +671,26 @@ int ac_decode_step_fused_ex(const void* q_in, void* q_rot_out, const void* k_new
     rope.rope_sin = rope_sin;
     rope.max_position = max_position;
     rope.num_pages = num_pages;
+    rope.out_mirror = out_mirror;
     return attn_common(q_in, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
                        max_pages_per_seq, context_lens, 1, softmax_scale, num_splits, workspace,
                        workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages, max_context_len,
                        status_flag, stream, true, &rope, window, row_order);
+}
+
+int ac_decode_step_fused_ex(const void* q_in, void* q_rot_out, const void* k_new, const void* v_new,
+                            void* k_cache, void* v_cache, int64_t stride_page, int64_t stride_token,
+                            int64_t stride_head, const int32_t* block_table, int max_pages_per_seq,
+                            const int32_t* context_lens, const float* rope_cos, const float* rope_sin,
+                            int max_position, float softmax_scale, int num_splits, void* workspace,
+                            size_t workspace_bytes, void* out, int B, int Hq, int Hkv, int d,
+                            int page_size, int num_pages, int max_context_len, int32_t* status_flag,
+                            void* stream, const ac_attn_options* options) {
+    return decode_step_fused_impl(q_in, q_rot_out, k_new, v_new, k_cache, v_cache, stride_page, stride_token,
+                                  stride_head, block_table, max_pages_per_seq, context_lens, rope_cos,
+                                  rope_sin, max_position, softmax_scale, num_splits, workspace,
+                                  workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages, max_context_len,
+                                  status_flag, stream, options, nullptr);
 }
 
 int ac_paged_decode_attn_ex(const void* q_rot, const void* k_cache, const void* v_cache,
@@ -775,12 +792,24 @@ int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* 
             (e = cudaMemcpyAsync(context_lens, context_lens_host, len_bytes, cudaMemcpyHostToDevice, cs)) != cudaSuccess)
             return fail_cuda(static_cast<int>(e));
     }
-    st = ac_decode_step_fused(q, nullptr, k_new, v_new, k_cache, v_cache, stride_page, stride_token,
-                              stride_head, block_table, max_pages_per_seq, context_lens, rope_cos,
-                              rope_sin, max_position, softmax_scale, num_splits, workspace,
-                              workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages, max_context_len,
-                              status_flag, stream);
-    if (st != AC_OK) return st;
+    // The result goes to out and, when out_host is pinned memory the GPU can address (16-byte aligned),
+    // straight to out_host as well: the kernel's final stores are mirrored there, which saves the
+    // device-to-host copy and the two stream hand-overs around it.  Otherwise a copy follows.
+    void* mirror = nullptr;
+    {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, out_host) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
+            attr.devicePointer != nullptr && aligned16(attr.devicePointer))
+            mirror = attr.devicePointer;
+        else
+            cudaGetLastError();
+    }
+    st = decode_step_fused_impl(q, nullptr, k_new, v_new, k_cache, v_cache, stride_page, stride_token,
+                                stride_head, block_table, max_pages_per_seq, context_lens, rope_cos,
+                                rope_sin, max_position, softmax_scale, num_splits, workspace,
+                                workspace_bytes, out, B, Hq, Hkv, d, page_size, num_pages, max_context_len,
+                                status_flag, stream, nullptr, mirror);
+    if (st != AC_OK || mirror != nullptr) return st;
     e = cudaMemcpyAsync(out_host, out, q_bytes, cudaMemcpyDeviceToHost, cs);
     return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
 }

@@ -48,6 +48,7 @@ struct FusedRopeArgs {
     const float* rope_cos;
     const float* rope_sin;
     int max_position, num_pages;
+    void* out_mirror;         // optional: a second copy of the bf16 result, e.g. in host memory the GPU can write
 };
 
 // Prelude variants of the RoPE + append kernel (validated by the ABI layer).

@@ -75,6 +75,7 @@ struct AttnParams {
     float* partial_o;             // [B, Hq, S, D]   (S > 1)
     float* partial_lse;           // [B, Hq, S]      (S > 1)
     uint16_t* out;                // [B, Hq, D] bf16 (S == 1)
+    uint16_t* out_mirror;         // optional second destination of every store to `out` (nullptr: none)
     int32_t* status_flag;
     int32_t* arrivals;            // [B, Hkv] arrival counters, zero on entry (fused merge only)
     float scale_log2;             // softmax scale * log2(e)
@@ -215,12 +216,18 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
             if (!p.fused_merge && threadIdx.x < G)
                 p.partial_lse[(static_cast<size_t>(b) * p.Hq + h * G + threadIdx.x) * S + split] = -INFINITY;
             if (p.fused_merge && split == 0) {   // a row with no tokens at all: its output is +0
-                uint16_t* o = p.out + (static_cast<size_t>(b) * p.Hq + h * G) * D;
-                for (int e = threadIdx.x; e < G * D; e += THREADS) o[e] = 0;
+                const size_t o = (static_cast<size_t>(b) * p.Hq + h * G) * D;
+                for (int e = threadIdx.x; e < G * D; e += THREADS) {
+                    p.out[o + e] = 0;
+                    if (p.out_mirror != nullptr) p.out_mirror[o + e] = 0;
+                }
             }
         } else {
-            uint16_t* o = p.out + (static_cast<size_t>(b) * p.Hq + h * G) * D;
-            for (int e = threadIdx.x; e < G * D; e += THREADS) o[e] = 0;
+            const size_t o = (static_cast<size_t>(b) * p.Hq + h * G) * D;
+            for (int e = threadIdx.x; e < G * D; e += THREADS) {
+                p.out[o + e] = 0;
+                if (p.out_mirror != nullptr) p.out_mirror[o + e] = 0;
+            }
         }
         if (p.cluster_merge != 0 && S > 1) {
             // Cluster merge: keep step with the two cluster barriers of the CTAs that have tokens
@@ -629,7 +636,9 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
         const float val = num / den;
         const size_t hq = static_cast<size_t>(b) * p.Hq + h * G + row;
         if (S == 1) {
-            p.out[hq * D + col] = static_cast<uint16_t>(pack_bf16x2(val, 0.0f) & 0xFFFFu);
+            const uint16_t bits = static_cast<uint16_t>(pack_bf16x2(val, 0.0f) & 0xFFFFu);
+            p.out[hq * D + col] = bits;
+            if (p.out_mirror != nullptr) p.out_mirror[hq * D + col] = bits;
         } else if (cluster_merge) {
             *reinterpret_cast<float*>(smem_gen + staged_o(row, col)) = val;
             if (col == 0) *reinterpret_cast<float*>(smem_gen + staged_lse(row)) = (M + log2f(den)) * LN2;
@@ -678,8 +687,9 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
                     den += wgt;
                 }
                 const float inv = 1.0f / den;
-                *reinterpret_cast<uint2*>(p.out + (hq0 + row) * D + c4 * 4) =
-                    make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
+                const uint2 bits = make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
+                *reinterpret_cast<uint2*>(p.out + (hq0 + row) * D + c4 * 4) = bits;
+                if (p.out_mirror != nullptr) *reinterpret_cast<uint2*>(p.out_mirror + (hq0 + row) * D + c4 * 4) = bits;
             }
         }
         cluster_sync_all();                              // nobody's shared memory goes away before it was read
@@ -746,8 +756,9 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
             }
         }
         const float inv = 1.0f / den;
-        *reinterpret_cast<uint2*>(p.out + (hq0 + row) * D + c4 * 4) =
-            make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
+        const uint2 bits = make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
+        *reinterpret_cast<uint2*>(p.out + (hq0 + row) * D + c4 * 4) = bits;
+        if (p.out_mirror != nullptr) *reinterpret_cast<uint2*>(p.out_mirror + (hq0 + row) * D + c4 * 4) = bits;
     }
 }
 
@@ -840,7 +851,9 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
     p.stride_page = p.stride_token = p.stride_head = 0;
     p.rope_cos = p.rope_sin = nullptr;
     p.max_position = p.num_pages = 0;
+    p.out_mirror = nullptr;
     if (rope != nullptr) {
+        p.out_mirror = static_cast<uint16_t*>(rope->out_mirror);
         p.q_rot_out = static_cast<uint16_t*>(rope->q_rot_out);
         p.k_new = static_cast<const uint16_t*>(rope->k_new);
         p.v_new = static_cast<const uint16_t*>(rope->v_new);

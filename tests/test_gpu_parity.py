@@ -465,15 +465,23 @@ def test_batch_of_only_inactive_rows(rt, fused):
     (dict(B=3, Hq=8, Hkv=2, context_lens=[200, 37, 333], num_pages=96), 2),        # sizes not 16-byte multiples
     (dict(B=1, Hq=8, Hkv=2, context_lens=[77], num_pages=16), 2),
 ])
-def test_decode_step_from_host_buffers(rt, kw, splits):
+@pytest.mark.parametrize("pinned", [True, False])
+def test_decode_step_from_host_buffers(rt, kw, splits, pinned):
+    # pinned: inputs gathered by one kernel, result stored straight into the host buffer by the
+    # attention kernel; pageable: one copy per buffer in, one copy out.  Same results either way.
     import torch
     from paper_2606_07665_b200 import binding as ac
     w = small(57, **kw)
     q_rot, k_after, v_after, out_ref = O.oracle_decode_step(w)
     st = rt.DecodeStep(w, num_splits=splits)
-    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+
+    def pin(a):
+        t = torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else np.ascontiguousarray(a))
+        return t.pin_memory() if pinned else t.clone()
+
     h_q, h_k, h_v, h_bt, h_len = pin(w.q), pin(w.k_new), pin(w.v_new), pin(w.block_table), pin(w.context_lens)
-    h_out = torch.full((w.B, w.Hq, w.d), 0x7FC0, dtype=torch.int16).pin_memory()
+    h_out = torch.full((w.B, w.Hq, w.d), 0x7FC0, dtype=torch.int16)
+    h_out = h_out.pin_memory() if pinned else h_out
     # device staging buffers start with garbage: everything must come from the host buffers
     for t in (st.q_in, st.k_new, st.v_new):
         t.fill_(0x7FC0)
@@ -491,6 +499,7 @@ def test_decode_step_from_host_buffers(rt, kw, splits):
         assert int(st.status_flag.item()) == 0
         got = W.bf16_bits_to_f32(h_out.numpy().view(np.uint16)).astype(np.float64)
         check_out(got, out_ref, f"host step rep {rep}")
+        assert np.array_equal(rt.bits_of(st.out), h_out.numpy().view(np.uint16))    # device copy holds the same bits
         k_gpu, v_gpu = st.cache_bits()
         assert np.array_equal(k_gpu, k_after) and np.array_equal(v_gpu, v_after)
 
