@@ -241,7 +241,9 @@ static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_con
         for (int cand = 1; cand <= s_max; ++cand) {
             const int chunk = split_tokens_for(max_context_len, cand);
             if (static_cast<long long>(chunk) * (cand - 1) >= max_context_len) continue;   // empty split
-            const bool in_cluster = cand <= kClusterMergeMaxSplits && pairs * cand <= sm_count;
+            // the launch decides by the grid it is given: all B rows count, active or not
+            const bool in_cluster = cand <= kClusterMergeMaxSplits &&
+                                    static_cast<long long>(B) * Hkv * cand <= sm_count;
             if (cand > 1 && chunk < (in_cluster ? 128 : 256)) continue;
             double n = static_cast<double>(pairs) * cand;                // CTAs that have tokens
             double longest = chunk;                                       // tokens of the longest CTA
