@@ -626,3 +626,79 @@ def test_tiny_workload_oracle_result_is_frozen():
             assert np.allclose(va, vb, rtol=1e-12, atol=0), (a, b)
         else:
             assert a == b
+
+
+# ---------------------------------------------------------------------------------------------
+# Structural properties of softmax attention that hold for any inputs (they pin the oracle against
+# the mathematics, not against another implementation)
+# ---------------------------------------------------------------------------------------------
+
+def _dense_case(seed, n_tokens=23, Hq=4, Hkv=2, d=8, ps=4):
+    """One request whose cache is filled by the generator; returns bits ready for the attention oracle."""
+    w = tiny_case(seed=seed, B=1, Hq=Hq, Hkv=Hkv, d=d, ps=ps, lens=(n_tokens,), pool=2 * (n_tokens // ps + 2))
+    q_rot, k_after, v_after = O.oracle_rope_kv_append(w.q, w.k_new, w.v_new, w.k_cache, w.v_cache,
+                                                      w.block_table, w.context_lens, w.rope_cos,
+                                                      w.rope_sin, w.page_size)
+    return w, q_rot, k_after, v_after
+
+
+def test_output_is_a_convex_combination_of_the_values():
+    # every output coordinate lies between the smallest and the largest value of that coordinate
+    # among the attended tokens of the head's KV head, and equals neither unless all are equal
+    w, q_rot, k, v = _dense_case(21)
+    out = O.oracle_paged_decode_attn(q_rot, k, v, w.block_table, w.context_lens, w.page_size)
+    n = int(w.context_lens[0]) + 1
+    G = w.Hq // w.Hkv
+    for hq in range(w.Hq):
+        vals = O.gather_kv(v, w.block_table[0], n, w.page_size, hq // G)
+        assert (out[0, hq] > vals.min(axis=0)).all() and (out[0, hq] < vals.max(axis=0)).all()
+
+
+def test_token_order_inside_the_cache_does_not_matter():
+    # attention is a sum over tokens: storing the same (k, v) pairs in a different token order gives
+    # the same output up to fp64 summation order
+    w, q_rot, k, v = _dense_case(22)
+    out = O.oracle_paged_decode_attn(q_rot, k, v, w.block_table, w.context_lens, w.page_size)
+    n = int(w.context_lens[0]) + 1
+    perm = np.random.default_rng(5).permutation(n)
+    k2, v2 = k.copy(), v.copy()
+    ps = w.page_size
+    for new_t, old_t in enumerate(perm):
+        po, so = w.block_table[0, old_t // ps], old_t % ps
+        pn, sn = w.block_table[0, new_t // ps], new_t % ps
+        k2[pn, sn], v2[pn, sn] = k[po, so], v[po, so]
+    out2 = O.oracle_paged_decode_attn(q_rot, k2, v2, w.block_table, w.context_lens, w.page_size)
+    assert np.allclose(out, out2, rtol=1e-13, atol=1e-15)
+
+
+def test_duplicating_every_token_changes_nothing_but_the_lse():
+    # softmax over a multiset with every element twice has the same weights ratio: the output is
+    # unchanged and the log-sum-exp grows by exactly ln 2
+    w, q_rot, k, v = _dense_case(23, n_tokens=11)
+    n = int(w.context_lens[0]) + 1
+    out, lse = O.oracle_paged_decode_attn(q_rot, k, v, w.block_table, w.context_lens, w.page_size,
+                                          return_lse=True)
+    ps = w.page_size
+    pages2 = (2 * n + ps - 1) // ps
+    k2 = np.zeros((pages2, ps) + k.shape[2:], k.dtype)
+    v2 = np.zeros_like(k2)
+    for t in range(2 * n):
+        src = t % n
+        k2[t // ps, t % ps] = k[w.block_table[0, src // ps], src % ps]
+        v2[t // ps, t % ps] = v[w.block_table[0, src // ps], src % ps]
+    bt2 = np.arange(pages2, dtype=np.int32)[None, :]
+    out2, lse2 = O.oracle_paged_decode_attn(q_rot, k2, v2, bt2, np.array([2 * n], np.int32), ps,
+                                            new_tokens=0, return_lse=True)
+    assert np.allclose(out, out2, rtol=1e-13, atol=1e-15)
+    assert np.allclose(lse2 - lse, math.log(2.0), rtol=0, atol=1e-13)
+
+
+def test_scaling_q_by_a_power_of_two_equals_scaling_the_softmax_scale():
+    # scores are bilinear in q: doubling q (exact in bf16) is the same as doubling softmax_scale
+    w, q_rot, k, v = _dense_case(24)
+    q2 = W.f32_to_bf16_bits(W.bf16_bits_to_f32(q_rot) * np.float32(2.0))
+    d = w.d
+    a = O.oracle_paged_decode_attn(q2, k, v, w.block_table, w.context_lens, w.page_size)
+    b = O.oracle_paged_decode_attn(q_rot, k, v, w.block_table, w.context_lens, w.page_size,
+                                   softmax_scale=2.0 / math.sqrt(d))
+    assert np.allclose(a, b, rtol=1e-13, atol=1e-15)
