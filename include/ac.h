@@ -28,10 +28,11 @@
  *   - The kernels are launched with programmatic stream serialization and signal launch completion
  *     early, so that in a chain of calls each kernel's set-up overlaps the tail of the one before.
  *     Before synchronising on the preceding kernel the attention kernels read only context_lens,
- *     block_table and cache tiles below the one holding slot context_lens[b] - 1.  This is invisible
- *     unless the kernel enqueued directly before one of these calls BOTH writes context_lens or
- *     block_table AND itself signals programmatic launch completion before finishing; such a
- *     producer must not signal early (copies and ordinary kernels are always safe).
+ *     block_table and cache tiles below the one holding slot context_lens[b] - 1, and the projection
+ *     kernels only their weights.  This is invisible unless the kernel enqueued directly before one
+ *     of these calls BOTH writes context_lens, block_table or those weights AND itself signals
+ *     programmatic launch completion before finishing; such a producer must not signal early
+ *     (copies and ordinary kernels are always safe).
  *   - Tensors q/k/v/cache/out are bf16 (16-bit patterns); rope tables and partials are fp32;
  *     block_table and context_lens are int32.  The innermost dimension (head_dim) is contiguous.
  *   - Return value: AC_OK (0) or an ac_status > 0.  On any non-zero return nothing was launched.
