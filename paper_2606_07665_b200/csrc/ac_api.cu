@@ -472,7 +472,7 @@ int ac_oproj_residual_rmsnorm(const void* attn_out, const void* w_o, int K, int 
     int dev;
     int st = current_ready_device(&dev);
     if (st != AC_OK) return st;
-    // W_o [N, K] as (64 elements, row inside a 16-row half, half, 32-row block, 64-element K block);
+    // W_o [N, K] as (64 elements, row inside a 16-row block, -, 16-row block, 64-element K block);
     // attn_out [B, K] as (64 elements, batch row, 64-element K block).
     const cuuint64_t row_bytes = static_cast<cuuint64_t>(K) * 2;
     CUtensorMap w_map, x_map;
@@ -501,9 +501,10 @@ int ac_oproj_residual_rmsnorm(const void* attn_out, const void* w_o, int K, int 
         return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
     }
     {
-        cuuint64_t dims[5] = {64, 16, 2, static_cast<cuuint64_t>(N / 32), static_cast<cuuint64_t>(K / 64)};
-        cuuint64_t strides[4] = {row_bytes, row_bytes * 16, row_bytes * 32, 128};
-        cuuint32_t box[5] = {64, 16, 2, 1, 4};
+        // 16 consecutive rows per CTA (the third dimension is a dummy of extent 1)
+        cuuint64_t dims[5] = {64, 16, 1, static_cast<cuuint64_t>(N / 16), static_cast<cuuint64_t>(K / 64)};
+        cuuint64_t strides[4] = {row_bytes, row_bytes * 16, row_bytes * 16, 128};
+        cuuint32_t box[5] = {64, 16, 1, 1, 4};
         cuuint32_t es[5] = {1, 1, 1, 1, 1};
         CUresult r = g_encode_tiled(&w_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(w_o), dims,
                                     strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,

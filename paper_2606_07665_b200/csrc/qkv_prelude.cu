@@ -18,7 +18,7 @@
 // the epilogue rounds, rotates and scatters.
 //
 // The same weight-streaming body also serves the output projection (kernel family (v)): there a CTA
-// owns 32 consecutive output features and the epilogue adds the residual row and rounds once; the
+// owns 16 consecutive output features and the epilogue adds the residual row and rounds once; the
 // RMSNorm that follows needs all H features of a row and runs as a second, dependent launch.
 #include <math.h>
 
@@ -37,17 +37,22 @@ constexpr int QKV_THREADS = (QKV_WARPS + 1) * 32;
 constexpr int KC = 256;                               // K elements per stage
 constexpr int KBLOCKS = KC / 64;                      // 128-byte column blocks per stage
 constexpr int W_BLOCK_BYTES = 16 * 128;               // one swizzled [16 rows x 64 elements] block
-constexpr int W_STAGE_BYTES = KBLOCKS * 2 * W_BLOCK_BYTES;     // 16 KB: [kblock][half][row][64]
+// Row blocks of 16 weight rows per CTA: 2 for the QKV projection (the first and second halves of 16
+// rotary pairs), 1 for the output projection (16 consecutive features; 256 CTAs for N = 4096, so that
+// most SMs stream for two CTAs -- 128 CTAs of 32 features left 20 SMs idle and the rest at the rate
+// of a single CTA).
+__host__ __device__ constexpr int row_blocks(int epi) { return epi == 1 ? 1 : 2; }
 
-template <int BT>
+template <int BT, int RB>
 struct QkvSmem {
+    static constexpr int W_STAGE_BYTES = KBLOCKS * RB * W_BLOCK_BYTES;   // [kblock][row block][row][64]
     static constexpr int X_BLOCK_BYTES = BT * 128;                 // [BT batch rows x 64 elements]
     static constexpr int X_STAGE_BYTES = KBLOCKS * X_BLOCK_BYTES;
     static constexpr int STAGE_BYTES = W_STAGE_BYTES + X_STAGE_BYTES;
-    static constexpr int STAGES = BT <= 8 ? 5 : 4;
+    static constexpr int STAGES = RB == 1 ? (BT <= 8 ? 8 : 6) : (BT <= 8 ? 5 : 4);
     static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
     static constexpr int TOTAL = BAR_OFFSET + 2 * STAGES * 8 + 1024;
-    static_assert(QKV_WARPS * 32 * BT * 4 <= STAGES * STAGE_BYTES, "reduction buffer must fit");
+    static_assert(QKV_WARPS * 16 * RB * BT * 4 <= STAGES * STAGE_BYTES, "reduction buffer must fit");
 };
 
 struct QkvParams {
@@ -72,7 +77,10 @@ template <int BT, int EPI>
 __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
     const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map,
     const QkvParams p) {
-    using L = QkvSmem<BT>;
+    constexpr int RB = row_blocks(EPI);
+    constexpr int TROWS = 16 * RB;                    // weight rows (output features) per CTA
+    constexpr int W_STAGE_BYTES = QkvSmem<BT, RB>::W_STAGE_BYTES;
+    using L = QkvSmem<BT, RB>;
     constexpr int STAGES = L::STAGES;
     constexpr int NT = BT / 8;                        // 8-wide batch tiles of the MMA
 
@@ -107,9 +115,9 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
     if (warp != QKV_WARPS) cudaGridDependencySynchronize();
 
     bool timed_out = false;
-    float acc[2][NT][4];
+    float acc[RB][NT][4];
 #pragma unroll
-    for (int rb = 0; rb < 2; ++rb)
+    for (int rb = 0; rb < RB; ++rb)
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -164,10 +172,10 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
                 const int ks = 2 * warp + u;                      // k-step (16 elements) inside the chunk
                 const int kb = ks >> 2;                           // 64-element block
                 const int ch = (ks & 3) * 2;                      // first 16-byte chunk of the k-step
-                uint32_t a[2][4];
+                uint32_t a[RB][4];
 #pragma unroll
-                for (int rb = 0; rb < 2; ++rb) {
-                    const uint32_t addr = wbase + (kb * 2 + rb) * W_BLOCK_BYTES + a_row_off +
+                for (int rb = 0; rb < RB; ++rb) {
+                    const uint32_t addr = wbase + (kb * RB + rb) * W_BLOCK_BYTES + a_row_off +
                                           (((ch + a_chunk) ^ r8) << 4);
                     ldmatrix_x4(a[rb][0], a[rb][1], a[rb][2], a[rb][3], addr);
                 }
@@ -179,7 +187,7 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
                     (void)bq2;
                     (void)bq3;
 #pragma unroll
-                    for (int rb = 0; rb < 2; ++rb)
+                    for (int rb = 0; rb < RB; ++rb)
                         mma_bf16_16816(acc[rb][0][0], acc[rb][0][1], acc[rb][0][2], acc[rb][0][3], a[rb][0],
                                        a[rb][1], a[rb][2], a[rb][3], bq0, bq1);
                 } else {
@@ -190,7 +198,7 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
                         uint32_t bq0, bq1, bq2, bq3;
                         ldmatrix_x4(bq0, bq1, bq2, bq3, addr);
 #pragma unroll
-                        for (int rb = 0; rb < 2; ++rb) {
+                        for (int rb = 0; rb < RB; ++rb) {
                             mma_bf16_16816(acc[rb][2 * np][0], acc[rb][2 * np][1], acc[rb][2 * np][2],
                                            acc[rb][2 * np][3], a[rb][0], a[rb][1], a[rb][2], a[rb][3], bq0, bq1);
                             mma_bf16_16816(acc[rb][2 * np + 1][0], acc[rb][2 * np + 1][1], acc[rb][2 * np + 1][2],
@@ -207,14 +215,14 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
 
     // ---- reduce the warps' partial sums through shared memory ----------------------------------------
     __syncthreads();                                   // every load has landed and been consumed
-    float* red = reinterpret_cast<float*>(smem_gen);   // [QKV_WARPS][32 rows][BT]
+    float* red = reinterpret_cast<float*>(smem_gen);   // [QKV_WARPS][TROWS][BT]
     if (warp < QKV_WARPS) {
         const int g = lane >> 2, t = lane & 3;
 #pragma unroll
-        for (int rb = 0; rb < 2; ++rb)
+        for (int rb = 0; rb < RB; ++rb)
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-                float* base = red + (warp * 32 + rb * 16) * BT + nt * 8 + 2 * t;
+                float* base = red + (warp * TROWS + rb * 16) * BT + nt * 8 + 2 * t;
                 *reinterpret_cast<float2*>(base + g * BT) = make_float2(acc[rb][nt][0], acc[rb][nt][1]);
                 *reinterpret_cast<float2*>(base + (g + 8) * BT) = make_float2(acc[rb][nt][2], acc[rb][nt][3]);
             }
@@ -223,15 +231,15 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
 
     if (EPI == EPI_RESIDUAL_ADD) {
         // ---- epilogue of the output projection: h = bf16(residual + y), one rounding ----------------
-        for (int item = threadIdx.x; item < 32 * BT; item += QKV_THREADS) {
-            const int r = item / BT;                   // row inside the 32-feature block
+        for (int item = threadIdx.x; item < TROWS * BT; item += QKV_THREADS) {
+            const int r = item / BT;                   // row inside the CTA's block of features
             const int n = item - r * BT;
             const int b = b0 + n;
             if (b >= p.B) continue;
             float y = 0.0f;
 #pragma unroll
-            for (int w = 0; w < QKV_WARPS; ++w) y += red[(w * 32 + r) * BT + n];
-            const size_t idx = static_cast<size_t>(b) * p.N + 32 * hh + r;
+            for (int w = 0; w < QKV_WARPS; ++w) y += red[(w * TROWS + r) * BT + n];
+            const size_t idx = static_cast<size_t>(b) * p.N + TROWS * hh + r;
             const float res = bf16_bits_to_float(p.residual_in[idx]);
             p.residual_out[idx] = static_cast<uint16_t>(pack_bf16x2(res + y, 0.0f) & 0xFFFFu);
         }
@@ -250,8 +258,8 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
         float y_lo = 0.0f, y_hi = 0.0f;
 #pragma unroll
         for (int w = 0; w < QKV_WARPS; ++w) {
-            y_lo += red[(w * 32 + j) * BT + n];
-            y_hi += red[(w * 32 + 16 + j) * BT + n];
+            y_lo += red[(w * TROWS + j) * BT + n];
+            y_hi += red[(w * TROWS + 16 + j) * BT + n];
         }
         const uint32_t packed = pack_bf16x2(y_lo, y_hi);
         uint16_t lo = static_cast<uint16_t>(packed & 0xFFFFu), hi = static_cast<uint16_t>(packed >> 16);
@@ -294,10 +302,10 @@ template <int BT, int EPI>
 cudaError_t launch_qkv(const CUtensorMap& w_map, const CUtensorMap& x_map, const QkvParams& p,
                        cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = EPI == EPI_RESIDUAL_ADD ? dim3(1, p.N / 32, (p.B + BT - 1) / BT)
+    cfg.gridDim = EPI == EPI_RESIDUAL_ADD ? dim3(1, p.N / (16 * row_blocks(EPI)), (p.B + BT - 1) / BT)
                                           : dim3(p.d / 32, p.Hq + 2 * p.Hkv, (p.B + BT - 1) / BT);
     cfg.blockDim = dim3(QKV_THREADS);
-    cfg.dynamicSmemBytes = QkvSmem<BT>::TOTAL;
+    cfg.dynamicSmemBytes = QkvSmem<BT, row_blocks(EPI)>::TOTAL;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -310,11 +318,13 @@ cudaError_t launch_qkv(const CUtensorMap& w_map, const CUtensorMap& x_map, const
 }  // namespace
 
 cudaError_t qkv_set_attributes(int smem_optin) {
-    if (QkvSmem<16>::TOTAL > smem_optin) return cudaErrorInvalidConfiguration;
+    if (QkvSmem<16, 2>::TOTAL > smem_optin || QkvSmem<16, 1>::TOTAL > smem_optin)
+        return cudaErrorInvalidConfiguration;
     cudaError_t e;
 #define AC_SET(BT_, EPI_)                                                                          \
     e = cudaFuncSetAttribute(qkv_rope_append_kernel<BT_, EPI_>,                                    \
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, QkvSmem<BT_>::TOTAL);    \
+                             cudaFuncAttributeMaxDynamicSharedMemorySize,                          \
+                             QkvSmem<BT_, row_blocks(EPI_)>::TOTAL);                               \
     if (e != cudaSuccess) return e;
     AC_SET(8, EPI_QKV_ROPE_APPEND)
     AC_SET(16, EPI_QKV_ROPE_APPEND)
