@@ -500,6 +500,33 @@ def time_warm_replays(st, torch, reps=50):
     return a.elapsed_time(b) * 1e3 / reps
 
 
+def time_kernels_alone(w, device, runner, torch, reps=10):
+    """Median us of each kernel of the three-call path on its own (one event pair per launch, the
+    launches of a kind back to back with a synchronise in between): ac_rope_kv_append,
+    ac_paged_decode_attn (partials only) and ac_splitkv_merge."""
+    st = runner.DecodeStep(w, device=device, fused_step=False, fused_merge=False)
+    stream = torch.cuda.current_stream()
+    out = {}
+    for name, call in (("ac_rope_kv_append", st.rope_kv_append), ("ac_paged_decode_attn", st.attention),
+                       ("ac_splitkv_merge", st.merge)):
+        call()
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(reps):
+            a = torch.cuda.Event(enable_timing=True)
+            b = torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            call()
+            b.record(stream)
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b) * 1e3)
+        out[name + "_us"] = round(statistics.median(times), 2)
+    out["num_splits"] = st.num_splits
+    out["note"] = "each call timed alone between events, own launch (host launch path included)"
+    del st
+    return out
+
+
 def time_single_graph_call(st, torch, reps=30):
     """us per call when every call is its own graph launch (host launch overhead included), L2
     flushed between calls: write a buffer 4x L2, then read it so its dirty lines are written back."""
@@ -602,6 +629,7 @@ def run_ours(args):
                     "status_flag": info["status_flag"]})
                 del s2, ww
                 torch.cuda.empty_cache()
+            kernels_alone = time_kernels_alone(w, device, runner, torch)
             prelude = time_prelude_fusion(torch, device)
             for r in prelude:
                 r["frac_of_hbm_peak"] = round(r["weight_gbs"] / peak, 4)
@@ -615,6 +643,7 @@ def run_ours(args):
             cpu = None
             prelude = []
             block = []
+            kernels_alone = None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -639,7 +668,7 @@ def run_ours(args):
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
             "gpu_launches": args.steps * launches_per_step,
             "clocks": clocks, "status_flag": flag, "workloads": others,
-            "prelude_fusion": prelude, "attention_block": block,
+            "kernels_alone": kernels_alone, "prelude_fusion": prelude, "attention_block": block,
         }
         print(json.dumps(line))
     if world > 1:
