@@ -156,6 +156,17 @@ def oracle_sample_seconds(w, budget_s: float = 12.0):
     return bytes_total, t_total, desc
 
 
+def cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def cpu_threads_used() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -190,7 +201,8 @@ def run_reference(args):
         "config": {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "head_dim": w.d,
                    "page_size": w.page_size, "seed": w.seed,
                    "note": "ms_per_step is the sample's rate extrapolated to the whole step"},
-        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
+                         "cpu_model": cpu_model(), "host_cores": len(os.sched_getaffinity(0))},
         "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -638,7 +650,8 @@ def run_ours(args):
                 r["frac_of_hbm_peak"] = round(r["gbs"] / peak, 4)
             cpu_bytes, cpu_s, cpu_desc = oracle_sample_seconds(w, 12.0)
             cpu = {"value": cpu_bytes / cpu_s / 1e9, "unit": UNIT, "cores": cpu_threads_used(),
-                   "kind": "oracle", "sample": cpu_desc}
+                   "kind": "oracle", "sample": cpu_desc, "cpu_model": cpu_model(),
+                   "host_cores": len(os.sched_getaffinity(0))}
         else:
             cpu = None
             prelude = []
