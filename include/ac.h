@@ -29,10 +29,12 @@
  *     early, so that in a chain of calls each kernel's set-up overlaps the tail of the one before.
  *     Before synchronising on the preceding kernel the attention kernels read only context_lens,
  *     block_table and cache tiles below the one holding slot context_lens[b] - 1, and the projection
- *     kernels only their weights.  This is invisible unless the kernel enqueued directly before one
- *     of these calls BOTH writes context_lens, block_table or those weights AND itself signals
- *     programmatic launch completion before finishing; such a producer must not signal early
- *     (copies and ordinary kernels are always safe).
+ *     kernels only their weights.  The attention and RoPE kernels signal only after their own
+ *     synchronisation, so no kernel that writes the cache can still be running two launches back:
+ *     consecutive steps on one cache need nothing between them.  The early reads are invisible
+ *     unless the kernel enqueued directly before one of these calls BOTH writes context_lens,
+ *     block_table or those weights AND itself signals programmatic launch completion before
+ *     finishing; such a producer must not signal early (copies and ordinary kernels are always safe).
  *   - Tensors q/k/v/cache/out are bf16 (16-bit patterns); rope tables and partials are fp32;
  *     block_table and context_lens are int32.  The innermost dimension (head_dim) is contiguous.
  *   - Return value: AC_OK (0) or an ac_status > 0.  On any non-zero return nothing was launched.
@@ -68,7 +70,8 @@ typedef enum {
 
 /* Bits the kernels OR into the optional device word `status_flag` (never cleared by the library). */
 #define AC_FLAG_PAGE_OOB 1     /* a block-table entry used for the append was outside [0, num_pages) */
-#define AC_FLAG_POSITION_OOB 2 /* context_lens[b] >= max_position or its page index >= max_pages_per_seq */
+#define AC_FLAG_POSITION_OOB 2 /* context_lens[b] >= max_position or its page index >= max_pages_per_seq; in the
+                                  single-launch step also context_lens[b] + 1 > the tokens the split grid covers */
 #define AC_FLAG_WAIT_TIMEOUT 4 /* a bounded wait on a shared-memory barrier gave up */
 
 /* Once per device, outside any stream capture, with no other call of this library running on that
@@ -272,8 +275,10 @@ int ac_paged_decode_attn_fused_merge(const void* q_rot, const void* k_cache, con
  *
  * q_in is the un-rotated query [B,Hq,d]; q_rot_out (optional, may be NULL) receives the rotated
  * rows and must not alias q_in.  Workspace as for ac_paged_decode_attn_fused_merge (counters zero on
- * entry when num_splits > 1).  A row whose position is outside the rope table or whose page id is
- * outside the pool sets the status bits and appends nothing; its output is then unspecified. */
+ * entry when num_splits > 1).  A row whose position is outside the rope table or the block-table row,
+ * whose page id is outside the pool, or whose context_lens[b] + 1 exceeds what the launch's split
+ * grid covers (max_context_len too small for it: the new token's slot then lies in no CTA's range)
+ * sets the status bits, appends nothing and writes no q_rot_out; its output is then unspecified. */
 int ac_decode_step_fused(const void* q_in, void* q_rot_out, const void* k_new, const void* v_new,
                          void* k_cache, void* v_cache,
                          int64_t stride_page, int64_t stride_token, int64_t stride_head,
@@ -377,9 +382,10 @@ int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* 
  * bf16 rows to out [B,Hq,d].
  *
  * Limits and rules
- *   - B * Hq * num_splits * (d + 1) * 4 bytes must not exceed AC_STATIC_SCRATCH_BYTES, otherwise
- *     AC_ERR_SCRATCH_LIMIT is returned and nothing is launched.  Lower num_splits, or use
- *     ac_paged_decode_attn with your own workspace.
+ *   - For num_splits > 1, B * Hq * num_splits * (d + 1) * 4 bytes must not exceed
+ *     AC_STATIC_SCRATCH_BYTES, otherwise AC_ERR_SCRATCH_LIMIT is returned and nothing is launched.
+ *     Lower num_splits, or use ac_paged_decode_attn with your own workspace.  A single split uses
+ *     no scratch (the attention kernel writes `out` itself), so no size limit applies to it.
  *   - ac_init must have succeeded on the current device.  The first call on each device also looks
  *     up the array's device address (once; later calls reuse it): make that first call outside any
  *     stream capture.

@@ -271,8 +271,7 @@ def ac_decode_step_fused(q_in, q_rot_out, k_new, v_new, k_cache, v_cache, stride
         stride_token, stride_head, _ptr(block_table), max_pages_per_seq, _ptr(context_lens),
         _ptr(rope_cos), _ptr(rope_sin), max_position, softmax_scale, num_splits, _ptr(workspace),
         workspace_bytes, _ptr(out), B, Hq, Hkv, d, page_size, num_pages, max_context_len,
-        _ptr(status_flag), _stream(stream)), "ac_decode_step_fused", "ac_paged_decode_attn_ex", "ac_decode_step_fused_ex",
-           "ac_rope_kv_append_ex", "ac_qkv_rope_kv_append", "ac_oproj_residual_rmsnorm")
+        _ptr(status_flag), _stream(stream)), "ac_decode_step_fused")
 
 
 def _options(window: int = 0, fused_merge: bool = False, row_order=None):

@@ -51,10 +51,21 @@ extern "C" int ac_paged_decode_attn_static_scratch(
     const int32_t* context_lens, int new_tokens, float softmax_scale, int num_splits, void* out, int B,
     int Hq, int Hkv, int d, int page_size, int num_pages, int max_context_len, int32_t* status_flag,
     void* stream) {
+    // Every check that the two inner calls would make on `out`, B, Hq, d and num_splits is made here
+    // first, so that an error can only come back before anything has been enqueued.
     if (!out) return AC_ERR_NULL;
     if (B <= 0 || Hq <= 0 || d <= 0 || num_splits <= 0) return AC_ERR_SHAPE;
-    // The partials are needed even for a single split here (the merge then just converts to bf16),
-    // so the size rule is the plain product, not ac_workspace_bytes (which is 0 for one split).
+    if (d != 64 && d != 128) return AC_ERR_UNSUPPORTED;
+    if (B > 65535 || num_splits > 65535) return AC_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(out) & 15u) return AC_ERR_ALIGN;
+    if (num_splits == 1) {
+        // One split: the existing entry point writes the final rows to `out` directly and touches
+        // no scratch at all, so the size limit does not apply.
+        return ac_paged_decode_attn(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head,
+                                    block_table, max_pages_per_seq, context_lens, new_tokens,
+                                    softmax_scale, 1, nullptr, 0, out, B, Hq, Hkv, d, page_size,
+                                    num_pages, max_context_len, status_flag, stream);
+    }
     const unsigned long long need = static_cast<unsigned long long>(B) * Hq * num_splits *
                                     (static_cast<unsigned long long>(d) + 1) * sizeof(float);
     if (need > AC_STATIC_SCRATCH_BYTES) return AC_ERR_SCRATCH_LIMIT;
@@ -71,19 +82,11 @@ extern "C" int ac_paged_decode_attn_static_scratch(
     // log-sum-exp slot of its own split (a number, or -inf for a split with no tokens) before the
     // merge reads it, and the merge never reads the partial_o of a split whose slot is -inf.  What
     // an earlier call left behind is therefore either overwritten or ignored.
-    int st;
-    if (num_splits == 1) {
-        // One split: the existing entry point writes the final rows to `out` directly and touches
-        // no scratch at all.
-        return ac_paged_decode_attn(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head,
-                                    block_table, max_pages_per_seq, context_lens, new_tokens,
-                                    softmax_scale, 1, nullptr, 0, out, B, Hq, Hkv, d, page_size,
-                                    num_pages, max_context_len, status_flag, stream);
-    }
-    st = ac_paged_decode_attn(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head,
-                              block_table, max_pages_per_seq, context_lens, new_tokens, softmax_scale,
-                              num_splits, scratch, static_cast<size_t>(need), out, B, Hq, Hkv, d,
-                              page_size, num_pages, max_context_len, status_flag, stream);
+    const int st = ac_paged_decode_attn(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head,
+                                        block_table, max_pages_per_seq, context_lens, new_tokens,
+                                        softmax_scale, num_splits, scratch, static_cast<size_t>(need), out,
+                                        B, Hq, Hkv, d, page_size, num_pages, max_context_len, status_flag,
+                                        stream);
     if (st != AC_OK) return st;
     return ac_splitkv_merge(scratch, num_splits, context_lens, out, B, Hq, d, stream);
 }

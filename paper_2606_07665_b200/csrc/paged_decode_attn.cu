@@ -169,11 +169,6 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     const int G = p.Hq / p.Hkv;
     const int S = p.num_splits;
 
-    // Let the next kernel of the stream (launched with the programmatic-serialization attribute, as
-    // the kernels of this library are) become resident as soon as this grid's last CTAs are: its
-    // set-up and first loads then fill the SM slots that free up during this grid's tail.
-    cudaTriggerProgrammaticLaunchCompletion();
-
     // Everything up to the first read of q or of a cache slot that the preceding kernel may have
     // written is independent of that kernel, so with a programmatic dependent launch it overlaps the
     // preceding kernel's execution.  The preceding kernel is either the RoPE + append kernel of this
@@ -193,7 +188,8 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     for (int s = 0; s < STAGES; ++s) page_first[s] = load_page_id(s);
 
     int n_tokens = ctx < 0 ? 0 : ctx + p.new_tokens;
-    n_tokens = min(n_tokens, p.max_pages_per_seq * p.page_size);
+    const long long table_tokens = static_cast<long long>(p.max_pages_per_seq) * p.page_size;
+    if (n_tokens > table_tokens) n_tokens = static_cast<int>(table_tokens);
     // Sliding window: the row attends over tokens [tok_lo, n_tokens).  The splits partition the range
     // that starts at tok_lo rounded down to a multiple of 64; tiles wholly below tok_lo are skipped
     // and the first tile masks its leading tokens.
@@ -208,10 +204,23 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     }
     const int tok_end = min(window_base + (split + 1) * p.split_tokens, n_tokens);
 
+    // Programmatic launch completion is signalled only AFTER this CTA has synchronised on the
+    // preceding kernel (dependency_sync below).  The next kernel of the stream (launched with the
+    // programmatic-serialization attribute, as the kernels of this library are) then becomes resident
+    // while this grid is still running -- its set-up and first loads fill the SM slots that free up
+    // during this grid's tail -- but never before the kernel ahead of this one has completed: at most
+    // two kernels of a chain are in flight, so what a kernel reads before its own synchronisation can
+    // only be stale with respect to its direct predecessor, which is what the tile limit below
+    // (first_dependent_tile) accounts for.
+    auto dependency_sync = [&]() {
+        cudaGridDependencySynchronize();
+        cudaTriggerProgrammaticLaunchCompletion();
+    };
+
     if (tok_begin >= tok_end) {
         // Nothing to attend over in this split.  The buffers written here may still be in use by
         // the preceding kernel (a merge of the previous step, say), so wait for it first.
-        cudaGridDependencySynchronize();
+        dependency_sync();
         if (S > 1) {
             if (!p.fused_merge && threadIdx.x < G)
                 p.partial_lse[(static_cast<size_t>(b) * p.Hq + h * G + threadIdx.x) * S + split] = -INFINITY;
@@ -271,7 +280,12 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     // Fused step: the rotary angles of this CTA's query rows depend only on ctx; fetch them now so
     // that they are in registers when q itself can be read (after the dependency is met).
     constexpr int QP = ROPE ? (16 * (D / 2) + THREADS - 1) / THREADS : 1;   // rotary pairs per thread
-    const bool rope_ok = ROPE && ctx < p.max_position;
+    // The new token can be appended only if its position has a rope-table row, a block-table entry
+    // and a tile in this launch's split grid (max_context_len too small for the row otherwise).
+    const bool rope_ok = ROPE && ctx < p.max_position &&
+                         ctx < table_tokens &&
+                         static_cast<long long>(ctx) <
+                             window_base + static_cast<long long>(S) * p.split_tokens;
     float q_cos[QP], q_sin[QP];
     if (ROPE) {
         const float* cos_row = p.rope_cos + static_cast<size_t>(ctx) * (D / 2);
@@ -294,7 +308,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     for (int s = 0; s < STAGES; ++s) {
         if (s < n_my) {
             if (!dependency_met && tile_begin + warp + s * WARPS >= first_dependent_tile) {
-                cudaGridDependencySynchronize();
+                dependency_sync();
                 dependency_met = true;
             }
             if (lane == 0) issue(s, page_first[s]);
@@ -302,7 +316,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
         }
     }
     int page_next = issued < n_my ? load_page_id(issued) : 0;
-    if (!dependency_met) cudaGridDependencySynchronize();      // q was written by the preceding kernel
+    if (!dependency_met) dependency_sync();                    // q was written by the preceding kernel
     uint16_t q_raw_lo[QP], q_raw_hi[QP];
     if (ROPE) {
         const uint16_t* qsrc = p.q + (static_cast<size_t>(b) * p.Hq + h * G) * D;
@@ -453,6 +467,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
             timed_out = true;
             break;
         }
+        bool wrote_stage = false;                              // ordinary stores went into this stage
         const int tok0 = tile_token0(j);
         const int n_valid = tok_end - tok0;                    // >= 1; < 16 only on the last tile
         const int lo_valid = tok_lo - tok0;                    // > 0 only on the first tile of a window
@@ -473,6 +488,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
             }
             if (lane * 4 < D)
                 *reinterpret_cast<uint2*>(smem_gen + (vbase - smem_base) + tile_byte(lane * 4)) = v_new4;
+            wrote_stage = true;
             __syncwarp();
         }
 
@@ -518,6 +534,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
                     *dstz = make_uint4(0u, 0u, 0u, 0u);
                 }
             }
+            wrote_stage = true;
             __syncwarp();
         }
 
@@ -564,6 +581,9 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
         }
 
         // ---- refill this stage -----------------------------------------------------------------
+        // Ordinary (generic-proxy) stores into the stage -- the patch of the new token, the cleared V
+        // rows of a ragged tile -- are ordered before the TMA (async-proxy) write that refills it.
+        if (wrote_stage) fence_proxy_async_shared();
         __syncwarp();
         if (issued < n_my) {
             const int page = page_next;
@@ -654,7 +674,8 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
         // ---- fused merge inside a cluster: split 0 reads the other splits' staged results out of
         // their shared memory.  No global round trip, no ticket; CTAs whose split has no tokens pass
         // through the same two barriers and nothing else.
-        const int n_active = (n_tokens - window_base + p.split_tokens - 1) / p.split_tokens;   // <= 16
+        // splits with tokens, <= 16 (a row longer than the split grid covers still has S of them)
+        const int n_active = min(S, (n_tokens - window_base + p.split_tokens - 1) / p.split_tokens);
         cluster_sync_all();                              // every staged result is written and visible
         if (split == 0) {
             constexpr int D4 = D / 4;
@@ -700,7 +721,8 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     // Publish this CTA's partials, take a ticket, and let the holder of the last ticket do the merge.
     // Nobody waits for anybody: CTAs that are not last simply exit.
     __shared__ int s_is_last;
-    const int n_active = (n_tokens - window_base + p.split_tokens - 1) / p.split_tokens;   // splits with tokens
+    // splits with tokens (a row longer than the split grid covers still has S of them)
+    const int n_active = min(S, (n_tokens - window_base + p.split_tokens - 1) / p.split_tokens);
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {

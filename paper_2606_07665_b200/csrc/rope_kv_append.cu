@@ -29,12 +29,14 @@ __global__ void __launch_bounds__(128) rope_kv_append_kernel(
     int max_pages_per_seq, const int32_t* __restrict__ context_lens,
     const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, int max_position, int B,
     int Hq, int Hkv, int page_size, int num_pages, int32_t* status_flag) {
-    // Let a dependent kernel (the attention launch that follows) begin its own set-up right away; it
-    // synchronises on this grid's completion before reading anything written here.  This kernel
-    // itself may have been launched early, under the tail of the previous attention kernel, whose
-    // inputs (the rotated q buffer, the cache) it overwrites: wait for that kernel first.
-    cudaTriggerProgrammaticLaunchCompletion();
+    // This kernel may have been launched early, under the tail of the previous attention kernel, whose
+    // inputs (the rotated q buffer, the cache) it overwrites: wait for that kernel first.  Only then
+    // is the dependent kernel (the attention launch that follows) let in to begin its own set-up; it
+    // synchronises on this grid's completion before reading anything written here.  Signalling after
+    // the wait keeps a chain of launches at most two kernels deep, which is what the attention
+    // kernel's early tile loads rely on.
     cudaGridDependencySynchronize();
+    cudaTriggerProgrammaticLaunchCompletion();
     constexpr int HALF = D / 2;
     constexpr int THREADS_PER_VEC = HALF / 8;            // 8 (D=128) or 4 (D=64)
     const int heads = Hq + Hkv;
@@ -117,8 +119,8 @@ __global__ void __launch_bounds__(128) rope_kv_append_ex_kernel(
     const float* __restrict__ rope_sin, int max_position, int B, int Hq, int Hkv, int page_size,
     int num_pages, int32_t* status_flag, int rotary_dim, int interleaved,
     const uint16_t* __restrict__ q_norm_w, const uint16_t* __restrict__ k_norm_w, float norm_eps) {
+    cudaGridDependencySynchronize();               // as in the plain kernel: wait, then let the next one in
     cudaTriggerProgrammaticLaunchCompletion();
-    cudaGridDependencySynchronize();
     constexpr int EPL = D / 32;                           // elements per lane: 4 (D=128) or 2 (D=64)
     __shared__ uint16_t s_vec[4][D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
