@@ -15,6 +15,12 @@ L2 (how a serving loop runs the kernels: one graph per batch-size bucket coverin
 plus the time of a call that is its own graph launch with L2 flushed before it.  With N > 1 every rank runs an independent
 replica on its own GPU (the path has no exchange step); value is the sum over ranks.
 
+Timing: the block of K = ``--steps`` steps is repeated until about one second of device time has
+been timed (``timed_blocks`` blocks, each between its own pair of CUDA events, no host
+synchronisation in between) and the MEDIAN block is reported, so that the clock sampler sees the GPU
+under sustained load even when K steps take a few milliseconds; ``us_x_sm_mhz`` = us per step x
+median SM clock makes runs at different clocks comparable.
+
 ``--impl reference`` times the CPU oracle, as it stands, on a bounded sample of the same workload.
 """
 from __future__ import annotations
@@ -40,6 +46,9 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0          # datasheet figure, for context only (the roofline uses the measured copy peak)
 L2_FLUSH_BYTES = 512 << 20
+# the five configurations the benchmark spec names (the serving sweep counts once per bucket)
+BASELINE_CONFIGS = ("tiny", "single_request", "continuous_batching", "long_context") + tuple(
+    f"graph_sweep_b{b}" for b in W.GRAPH_SWEEP_BATCHES)
 
 
 # ---------------------------------------------------------------------------------------------
@@ -93,7 +102,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
             out = ""
-        sm, smax, reasons = [], [], set()
+        sm, smax, power, reasons = [], [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
         for line in out.splitlines():
             parts = [p.strip() for p in line.split(",")]
@@ -104,12 +113,19 @@ class ClockSampler:
                 smax.append(float(parts[1]))
             except ValueError:
                 continue
+            try:
+                power.append(float(parts[2]))
+            except ValueError:
+                pass
             for n, v in zip(names, parts[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None,
+        # "under load": samples taken while the board drew more than half of its highest reading
+        busy = [c for c, w in zip(sm, power) if power and w >= 0.5 * max(power)] if len(power) == len(sm) else sm
+        return {"sm_mhz": statistics.median(busy) if busy else (statistics.median(sm) if sm else None),
                 "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "samples_under_load": len(busy),
+                "power_w_max": max(power) if power else None, "reasons": sorted(reasons)}
 
 
 def dist_env():
@@ -122,6 +138,29 @@ def dist_env():
 # ---------------------------------------------------------------------------------------------
 # CPU oracle timing (reported baseline; also the --impl reference arm)
 # ---------------------------------------------------------------------------------------------
+
+def oracle_rows(w, budget_s: float = 1.5):
+    """The oracle timed on workload ``w`` twice: BLAS limited to one thread, and as it stands (all the
+    threads BLAS takes).  Each row: GB/s of K/V covered, threads, and what the sample was."""
+    rows = []
+    try:
+        from threadpoolctl import threadpool_limits
+    except Exception:
+        threadpool_limits = None
+    for label in ("1 thread", "all cores"):
+        if label == "1 thread":
+            if threadpool_limits is None:
+                continue
+            with threadpool_limits(limits=1):
+                b, t, desc = oracle_sample_seconds(w, budget_s)
+            threads = 1
+        else:
+            b, t, desc = oracle_sample_seconds(w, budget_s)
+            threads = cpu_threads_used()
+        rows.append({"threads": threads, "value": round(b / t / 1e9, 4), "unit": UNIT, "kind": "oracle",
+                     "seconds": round(t, 3), "sample": desc})
+    return rows
+
 
 def oracle_sample_seconds(w, budget_s: float = 12.0):
     """Times the oracle on (request, KV head) pairs of ``w`` until about ``budget_s`` of CPU work.
@@ -232,41 +271,57 @@ def aggregate_throughput(kv_bytes_per_rank, ms_slowest_rank, world):
 # GPU arm
 # ---------------------------------------------------------------------------------------------
 
+TIMED_REGION_MS = 1000.0          # repeat the K-step block until about this much device time is timed
+
+
+def blocks_for(ms_per_block: float, target_ms: float = TIMED_REGION_MS) -> int:
+    return int(max(1, min(2000, -(-target_ms // max(ms_per_block, 1e-3)))))
+
+
 def time_headline(st, steps, warmup, torch):
-    """K steps back to back between one pair of CUDA events on the launching stream.
+    """Blocks of K steps back to back, each block between its own pair of CUDA events on the launching
+    stream, repeated until about a second has been timed; returns the median block.
 
     With the single-launch fused step the step IS the dominant kernel, so its average launch
-    duration is the bracketed time / K (no event is recorded between launches: an event node between
+    duration is the block time / K (no event is recorded between launches: an event node between
     two kernels would undo the programmatic overlap of their tail and ramp).  With separate launches
     an event pair around every attention launch gives that kernel's own duration.
+    Returns (ms per step, ms per attention launch, number of blocks timed).
     """
     stream = torch.cuda.current_stream()
+    w0 = torch.cuda.Event(enable_timing=True)
+    w1 = torch.cuda.Event(enable_timing=True)
+    w0.record(stream)
     for _ in range(warmup):
         st.step(stream)
+    w1.record(stream)
     torch.cuda.synchronize()
-    t0 = torch.cuda.Event(enable_timing=True)
-    t1 = torch.cuda.Event(enable_timing=True)
+    n_blocks = blocks_for(w0.elapsed_time(w1) / max(1, warmup) * steps)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_blocks + 1)]
     if st.fused_step:
-        t0.record(stream)
-        for _ in range(steps):
-            st.decode_step_fused(stream)
-        t1.record(stream)
+        marks[0].record(stream)
+        for blk in range(n_blocks):
+            for _ in range(steps):
+                st.decode_step_fused(stream)
+            marks[blk + 1].record(stream)
         torch.cuda.synchronize()
-        per_step = t0.elapsed_time(t1) / steps
-        return per_step, per_step
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
-    t0.record(stream)
-    for i in range(steps):
-        st.rope_kv_append(stream)
-        ev[i][0].record(stream)
-        st.attention(stream)
-        ev[i][1].record(stream)
-        st.merge(stream)
-    t1.record(stream)
+        per_step = statistics.median(marks[i].elapsed_time(marks[i + 1]) for i in range(n_blocks)) / steps
+        return per_step, per_step, n_blocks
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps * n_blocks)]
+    marks[0].record(stream)
+    for blk in range(n_blocks):
+        for i in range(steps):
+            st.rope_kv_append(stream)
+            ev[blk * steps + i][0].record(stream)
+            st.attention(stream)
+            ev[blk * steps + i][1].record(stream)
+            st.merge(stream)
+        marks[blk + 1].record(stream)
     torch.cuda.synchronize()
-    total_ms = t0.elapsed_time(t1)
-    attn_ms = [a.elapsed_time(b) for a, b in ev]
-    return total_ms / steps, sum(attn_ms) / len(attn_ms)
+    block_ms = [marks[i].elapsed_time(marks[i + 1]) for i in range(n_blocks)]
+    mid = sorted(range(n_blocks), key=lambda i: block_ms[i])[n_blocks // 2]          # the median block
+    attn_ms = [a.elapsed_time(b) for a, b in ev[mid * steps:(mid + 1) * steps]]
+    return block_ms[mid] / steps, sum(attn_ms) / len(attn_ms), n_blocks
 
 
 def time_e2e(st, steps, warmup, torch):
@@ -291,19 +346,25 @@ def time_e2e(st, steps, warmup, torch):
                                st.B, st.Hq, st.Hkv, st.d, st.ps, st.num_pages, st.max_context_len,
                                st.status_flag, stream)
 
+    w0 = torch.cuda.Event(enable_timing=True)
+    w1 = torch.cuda.Event(enable_timing=True)
+    w0.record(stream)
     for _ in range(warmup):
         one()
+    w1.record(stream)
     torch.cuda.synchronize()
-    t0 = torch.cuda.Event(enable_timing=True)
-    t1 = torch.cuda.Event(enable_timing=True)
-    t0.record(stream)
-    for _ in range(steps):
-        one()
-    t1.record(stream)
+    n_blocks = blocks_for(w0.elapsed_time(w1) / max(1, warmup) * steps, 300.0)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_blocks + 1)]
+    marks[0].record(stream)
+    for blk in range(n_blocks):
+        for _ in range(steps):
+            one()
+        marks[blk + 1].record(stream)
     torch.cuda.synchronize()
     h2d = sum(t.numel() * t.element_size() for t in (h_q, h_k, h_v, h_bt, h_len))
     d2h = h_out.numel() * h_out.element_size()
-    return t0.elapsed_time(t1) / steps, h2d, d2h
+    ms = statistics.median(marks[i].elapsed_time(marks[i + 1]) for i in range(n_blocks)) / steps
+    return ms, h2d, d2h
 
 
 L2_BYTES = 126 << 20
@@ -494,6 +555,65 @@ def time_attention_block(torch, device, batches=(1, 8, 32), replicas=8, replays=
     return rows
 
 
+def time_read_stream(torch, device, nbytes=4 << 30, reps=10):
+    """GB/s of a plain coalesced read-only pass over a 4 GiB device buffer (the library's probe kernel,
+    16-byte streaming loads, nothing written): best and median of `reps` passes after three warm-ups.
+    Context for the roofline fractions, whose denominator is a copy (read + write) measurement."""
+    from paper_2606_07665_b200 import binding as ac
+    buf = torch.empty(nbytes // 4, dtype=torch.int32, device=device)
+    buf.fill_(0x01010101)
+    sink = torch.zeros(2, dtype=torch.int64, device=device)
+    stream = torch.cuda.current_stream()
+    for _ in range(3):
+        ac.ac_hbm_read_probe(buf, nbytes, sink, stream)
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(reps):
+        a = torch.cuda.Event(enable_timing=True)
+        b = torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        ac.ac_hbm_read_probe(buf, nbytes, sink, stream)
+        b.record(stream)
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b))
+    del buf
+    torch.cuda.empty_cache()
+    return {"best_gbs": round(nbytes / min(times) / 1e6, 1), "median_gbs": round(nbytes / statistics.median(times) / 1e6, 1),
+            "bytes": nbytes, "kernel": "hbm_read_probe_kernel"}
+
+
+def time_rope_variants(torch, device, batch=256, reps=50):
+    """us per call of ac_rope_kv_append_ex with the prelude variants switched on (per-head Q/K RMSNorm,
+    partial rotary, interleaved pairing) on a graph-sweep-shaped batch, one launch per event pair."""
+    from paper_2606_07665_b200 import runner
+    w = W.graph_sweep(batch)
+    R = 64
+    w.rope_cos, w.rope_sin = W.rope_table(w.max_position, R, w.rope_base)
+    st = runner.DecodeStep(w, device=device, fused_merge=False)
+    rng = np.random.default_rng(5)
+    nw = torch.from_numpy(W.f32_to_bf16_bits((1 + 0.1 * rng.standard_normal(w.d)).astype(np.float32)).view(np.int16)).to(device)
+    stream = torch.cuda.current_stream()
+    rows = []
+    for label, kw in (("qk_norm+partial_rotary_64+interleaved", dict(rotary_dim=R, interleaved=True, q_norm_weight=nw, k_norm_weight=nw, norm_eps=1e-6)),
+                      ("partial_rotary_64", dict(rotary_dim=R))):
+        for _ in range(3):
+            st.rope_kv_append_ex(stream, **kw)
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(reps):
+            a = torch.cuda.Event(enable_timing=True)
+            b = torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            st.rope_kv_append_ex(stream, **kw)
+            b.record(stream)
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b) * 1e3)
+        rows.append({"kernel": "rope_kv_append_ex_kernel", "variant": label, "B": batch,
+                     "us_per_call_own_launch": round(statistics.median(times), 2),
+                     "status_flag": int(st.status_flag.item())})
+    return rows
+
+
 def time_warm_replays(st, torch, reps=50):
     """us per call when the same captured step is replayed back to back with nothing else touching the
     GPU: K/V of workloads that fit in L2 stay resident there (the warm figure next to the cold ones)."""
@@ -580,6 +700,10 @@ def run_ours(args):
     ac.ac_init(local)
     peak, peak_kind = measured_peak()
 
+    if args.rope_variants_only:
+        if rank == 0:
+            print(json.dumps({"rope_variants": time_rope_variants(torch, device, reps=5)}))
+        return
     if args.prelude_only:
         if rank == 0:
             print(json.dumps({"prelude_fusion": time_prelude_fusion(torch, device, batches=(args.prelude_batch,),
@@ -599,13 +723,14 @@ def run_ours(args):
     barrier()
     if rank == 0:
         sampler.start()
-    ms_step, ms_attn = time_headline(st, args.steps, args.warmup, torch)
+    ms_step, ms_attn, timed_blocks = time_headline(st, args.steps, args.warmup, torch)
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
     ms_e2e, h2d, d2h = time_e2e(st, args.steps, args.warmup, torch)
     barrier()
+    clocks = sampler.stop() if rank == 0 else None       # sampled over both timed regions
     flag = int(st.status_flag.item())
     launches_per_step = st.launches_per_step
+    timed_num_splits = st.num_splits
 
     ms_step, ms_attn, ms_e2e = max_over_ranks([ms_step, ms_attn, ms_e2e], world, device)
 
@@ -638,10 +763,13 @@ def run_ours(args):
                     "us_per_call_own_graph_launch_l2_flushed": round(alone_us, 2),
                     "us_per_call_own_graph_launch_warm": round(warm_us, 2),
                     "fits_in_l2": bool(ww.kv_bytes < L2_BYTES),
-                    "status_flag": info["status_flag"]})
+                    "status_flag": info["status_flag"],
+                    "cpu_baseline": oracle_rows(ww) if name in BASELINE_CONFIGS else None})
                 del s2, ww
                 torch.cuda.empty_cache()
             kernels_alone = time_kernels_alone(w, device, runner, torch)
+            read_stream = time_read_stream(torch, device)
+            rope_variants = time_rope_variants(torch, device)
             prelude = time_prelude_fusion(torch, device)
             for r in prelude:
                 r["frac_of_hbm_peak"] = round(r["weight_gbs"] / peak, 4)
@@ -651,46 +779,52 @@ def run_ours(args):
             cpu_bytes, cpu_s, cpu_desc = oracle_sample_seconds(w, 12.0)
             cpu = {"value": cpu_bytes / cpu_s / 1e9, "unit": UNIT, "cores": cpu_threads_used(),
                    "kind": "oracle", "sample": cpu_desc, "cpu_model": cpu_model(),
-                   "host_cores": len(os.sched_getaffinity(0))}
+                   "host_cores": len(os.sched_getaffinity(0)),
+                   "rows": oracle_rows(w, 4.0)}
         else:
             cpu = None
             prelude = []
             block = []
             kernels_alone = None
+            read_stream = None
+            rope_variants = []
+        sm_mhz = clocks.get("sm_mhz") if clocks else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms_step, "timed_blocks": timed_blocks,
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "head_dim": w.d,
                        "page_size": w.page_size, "context_len": int(w.context_lens.max()),
-                       "num_pages": w.num_pages, "seed": w.seed, "num_splits": runner_splits(w, ac),
+                       "num_pages": w.num_pages, "seed": w.seed, "num_splits": timed_num_splits,
                        "kv_bytes_per_step": kv, "l2": "inputs larger than L2 (no flush)",
+                       "timing": f"median of {timed_blocks} blocks of {args.steps} steps, ~{TIMED_REGION_MS / 1e3:.0f} s timed",
                        "launches_per_step": launches_per_step,
                        "entry_point": "ac_rope_kv_append + ac_paged_decode_attn_fused_merge"
                        if args.three_launches else "ac_decode_step_fused",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "us_per_call": ms_step * 1e3,
+            "us_x_sm_mhz": ms_step * 1e3 * sm_mhz if sm_mhz else None,
             "frac_of_hbm_peak": value / world / peak,
             "frac_of_nominal_8000": value / world / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": attn_gbs, "peak": peak, "unit": "GB/s",
                          "frac": attn_gbs / peak, "peak_kind": peak_kind,
                          "kernel": "paged_decode_attn_kernel" + ("" if args.three_launches else " (fused step)"),
-                         "traffic": ncu_traffic("paged_decode_attn_kernel", w.name)},
+                         "traffic": ncu_traffic("paged_decode_attn_kernel", w.name),
+                         "read_only_stream": read_stream,
+                         "frac_of_read_only_stream": (attn_gbs / read_stream["best_gbs"]) if read_stream else None},
             "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
-            "gpu_launches": args.steps * launches_per_step,
+            "gpu_launches": args.steps * launches_per_step * timed_blocks,
             "clocks": clocks, "status_flag": flag, "workloads": others,
             "kernels_alone": kernels_alone, "prelude_fusion": prelude, "attention_block": block,
+            "rope_variants": rope_variants,
         }
         print(json.dumps(line))
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
-
-
-def runner_splits(w, ac):
-    return ac.ac_decode_plan(w.B, w.Hq, w.Hkv, w.d, w.page_size, w.max_context_len, ac.ac_sm_count())[0]
 
 
 def main():
@@ -711,6 +845,8 @@ def main():
     ap.add_argument("--prelude-only", action="store_true",
                     help="time only the projection fusions (ac_qkv_rope_kv_append, ac_oproj_residual_rmsnorm) "
                          "at batch 8 and print their rows; used for profiling those kernels")
+    ap.add_argument("--rope-variants-only", action="store_true",
+                    help="time only ac_rope_kv_append_ex with the prelude variants on (profiling that kernel)")
     ap.add_argument("--only-headline", action="store_true",
                     help="skip the other workloads and the CPU baseline")
     args = ap.parse_args()

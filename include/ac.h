@@ -360,6 +360,15 @@ int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* 
                         int B, int Hq, int Hkv, int d, int page_size, int num_pages,
                         int max_context_len, int32_t* status_flag, void* stream);
 
+/* Calibration helper (no paper counterpart): enqueues a plain coalesced read-only pass over
+ * buffer[0, bytes) -- 16-byte streaming loads, nothing written -- on `stream`.  Timed by the caller
+ * (CUDA events around it) it gives the read-only HBM ceiling of the machine, which a benchmark can
+ * print beside the copy-measured peak its roofline fractions use.  buffer: device memory, 16-byte
+ * aligned, bytes >= 16 (a tail shorter than 16 bytes is not read); sink: optional device word that
+ * receives the fold of a thread's loads only if that happens to equal one constant (it keeps the
+ * loads alive; expect it untouched).  ac_init must have succeeded on the current device. */
+int ac_hbm_read_probe(const void* buffer, size_t bytes, void* sink, void* stream);
+
 /* Size of the library's built-in partial-result array (bytes), held by every GPU that loads the
  * library until the process exits. */
 #define AC_STATIC_SCRATCH_BYTES (8u << 20)

@@ -27,7 +27,8 @@ EXPORTS = ("ac_init", "ac_status_string", "ac_last_cuda_error", "ac_sm_count", "
            "ac_splitkv_merge", "ac_decode_step_host", "ac_paged_decode_attn_static_scratch",
            "ac_fused_workspace_bytes", "ac_fused_workspace_reset", "ac_paged_decode_attn_fused_merge",
            "ac_decode_step_fused", "ac_paged_decode_attn_ex", "ac_decode_step_fused_ex",
-           "ac_rope_kv_append_ex", "ac_qkv_rope_kv_append", "ac_oproj_residual_rmsnorm")
+           "ac_rope_kv_append_ex", "ac_qkv_rope_kv_append", "ac_oproj_residual_rmsnorm",
+           "ac_hbm_read_probe")
 AC_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -119,6 +120,8 @@ def lib():
                                                           c_void_p, c_int, c_float, c_int, c_void_p] +
                                                           [c_int] * 7 + [c_void_p, c_void_p])
         L.ac_paged_decode_attn_static_scratch.restype = c_int
+        L.ac_hbm_read_probe.argtypes = [c_void_p, c_size_t, c_void_p, c_void_p]
+        L.ac_hbm_read_probe.restype = c_int
         _lib = L
     return _lib
 
@@ -340,3 +343,8 @@ def ac_paged_decode_attn_static_scratch(q_rot, k_cache, v_cache, stride_page, st
         _ptr(block_table), max_pages_per_seq, _ptr(context_lens), new_tokens, softmax_scale, num_splits,
         _ptr(out), B, Hq, Hkv, d, page_size, num_pages, max_context_len, _ptr(status_flag),
         _stream(stream)), "ac_paged_decode_attn_static_scratch")
+
+
+def ac_hbm_read_probe(buffer, nbytes, sink=None, stream=None):
+    """Enqueues one read-only pass over ``buffer`` (calibration; the caller times it)."""
+    _check(lib().ac_hbm_read_probe(_ptr(buffer), nbytes, _ptr(sink), _stream(stream)), "ac_hbm_read_probe")

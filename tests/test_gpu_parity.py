@@ -861,6 +861,20 @@ def test_random_configurations_match_oracle(rt, seed):
                     check_cache=True)
 
 
+def test_hbm_read_probe_runs_and_validates(rt):
+    import torch
+    from paper_2606_07665_b200 import binding as ac
+    buf = torch.full((1 << 20,), 0x01010101, dtype=torch.int32, device="cuda")
+    sink = torch.zeros(2, dtype=torch.int64, device="cuda")
+    ac.ac_hbm_read_probe(buf, buf.numel() * 4, sink)
+    ac.ac_hbm_read_probe(buf, 16 * 3 + 5, sink)               # ragged tail is ignored
+    torch.cuda.synchronize()
+    assert int(sink[0].item()) == 0 and int(buf.sum().item()) == (1 << 20) * 0x01010101
+    assert ac.lib().ac_hbm_read_probe(None, 1024, None, None) == 1
+    assert ac.lib().ac_hbm_read_probe(buf.data_ptr() + 4, 1024, None, None) == 4
+    assert ac.lib().ac_hbm_read_probe(buf.data_ptr(), 8, None, None) == 2
+
+
 def test_maximum_batch(rt):
     """B = 65535, the largest batch the ABI accepts (grid.y limit): every row gets its own CTA."""
     B = 65535
