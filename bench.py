@@ -274,7 +274,8 @@ def aggregate_throughput(kv_bytes_per_rank, ms_slowest_rank, world):
 TIMED_REGION_MS = 1000.0          # repeat the K-step block until about this much device time is timed
 
 
-def blocks_for(ms_per_block: float, target_ms: float = TIMED_REGION_MS) -> int:
+def blocks_for(ms_per_block: float, target_ms: float | None = None) -> int:
+    target_ms = TIMED_REGION_MS if target_ms is None else target_ms
     return int(max(1, min(2000, -(-target_ms // max(ms_per_block, 1e-3)))))
 
 
@@ -353,7 +354,7 @@ def time_e2e(st, steps, warmup, torch):
         one()
     w1.record(stream)
     torch.cuda.synchronize()
-    n_blocks = blocks_for(w0.elapsed_time(w1) / max(1, warmup) * steps, 300.0)
+    n_blocks = blocks_for(w0.elapsed_time(w1) / max(1, warmup) * steps, 0.3 * TIMED_REGION_MS)
     marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_blocks + 1)]
     marks[0].record(stream)
     for blk in range(n_blocks):
@@ -847,9 +848,14 @@ def main():
                          "at batch 8 and print their rows; used for profiling those kernels")
     ap.add_argument("--rope-variants-only", action="store_true",
                     help="time only ac_rope_kv_append_ex with the prelude variants on (profiling that kernel)")
+    ap.add_argument("--timed-ms", type=float, default=None,
+                    help="device time to fill with repeated K-step blocks (default 1000; profiling runs pass a small value)")
     ap.add_argument("--only-headline", action="store_true",
                     help="skip the other workloads and the CPU baseline")
     args = ap.parse_args()
+    if args.timed_ms is not None:
+        global TIMED_REGION_MS
+        TIMED_REGION_MS = max(0.0, args.timed_ms)
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
