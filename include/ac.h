@@ -301,7 +301,11 @@ typedef struct ac_attn_options {
                         for free) shortens the tail of grids that are several waves deep.  Any
                         permutation gives the same results.  NULL: the kernel ranks the requests
                         itself when B <= 128 and serves them in index order otherwise. */
-    int reserved[4];
+    const struct ac_rope_options* rope; /* ac_decode_step_fused_ex only: prelude variants (per-head Q/K
+                        RMSNorm, partial rotary, interleaved pairing) applied to q_in and k_new inside the
+                        step, with the arithmetic and the table shapes of ac_rope_kv_append_ex; NULL or
+                        all-default options = the plain rotation */
+    int reserved[2];
 } ac_attn_options;
 
 /* ac_paged_decode_attn / ac_paged_decode_attn_fused_merge / ac_decode_step_fused with options

@@ -34,7 +34,8 @@ AC_STATIC_SCRATCH_BYTES = 8 << 20
 
 class AcAttnOptions(ctypes.Structure):
     """Mirror of ac_attn_options."""
-    _fields_ = [("window", c_int), ("fused_merge", c_int), ("row_order", c_void_p), ("reserved", c_int * 4)]
+    _fields_ = [("window", c_int), ("fused_merge", c_int), ("row_order", c_void_p), ("rope", c_void_p),
+                ("reserved", c_int * 2)]
 
 
 class AcRopeOptions(ctypes.Structure):
@@ -200,12 +201,7 @@ def ac_rope_kv_append_ex(q_in, q_out, k_new, v_new, k_cache, v_cache, stride_pag
                          max_position, B, Hq, Hkv, d, page_size, num_pages, status_flag=None, stream=None,
                          rotary_dim=0, interleaved=False, q_norm_weight=None, k_norm_weight=None,
                          norm_eps=0.0):
-    opt = AcRopeOptions()
-    opt.rotary_dim = int(rotary_dim)
-    opt.interleaved = 1 if interleaved else 0
-    opt.q_norm_weight = _ptr(q_norm_weight)
-    opt.k_norm_weight = _ptr(k_norm_weight)
-    opt.norm_eps = float(norm_eps)
+    opt = _rope_options(rotary_dim, interleaved, q_norm_weight, k_norm_weight, norm_eps)
     _check(lib().ac_rope_kv_append_ex(_ptr(q_in), _ptr(q_out), _ptr(k_new), _ptr(v_new), _ptr(k_cache),
                                       _ptr(v_cache), stride_page, stride_token, stride_head,
                                       _ptr(block_table), max_pages_per_seq, _ptr(context_lens),
@@ -277,12 +273,25 @@ def ac_decode_step_fused(q_in, q_rot_out, k_new, v_new, k_cache, v_cache, stride
         _ptr(status_flag), _stream(stream)), "ac_decode_step_fused")
 
 
-def _options(window: int = 0, fused_merge: bool = False, row_order=None):
+def _rope_options(rotary_dim=0, interleaved=False, q_norm_weight=None, k_norm_weight=None, norm_eps=0.0):
+    opt = AcRopeOptions()
+    opt.rotary_dim = int(rotary_dim)
+    opt.interleaved = 1 if interleaved else 0
+    opt.q_norm_weight = _ptr(q_norm_weight)
+    opt.k_norm_weight = _ptr(k_norm_weight)
+    opt.norm_eps = float(norm_eps)
+    return opt
+
+
+def _options(window: int = 0, fused_merge: bool = False, row_order=None, rope=None):
+    """rope: an AcRopeOptions instance (kept alive by the returned structure) or None."""
     opt = AcAttnOptions()
     opt.window = int(window)
     opt.fused_merge = 1 if fused_merge else 0
     opt.row_order = _ptr(row_order)
-    return ctypes.byref(opt)
+    opt.rope = ctypes.addressof(rope) if rope is not None else None
+    opt._keep = rope
+    return opt
 
 
 def ac_paged_decode_attn_ex(q_rot, k_cache, v_cache, stride_page, stride_token, stride_head, block_table,
@@ -294,21 +303,26 @@ def ac_paged_decode_attn_ex(q_rot, k_cache, v_cache, stride_page, stride_token, 
         _ptr(q_rot), _ptr(k_cache), _ptr(v_cache), stride_page, stride_token, stride_head,
         _ptr(block_table), max_pages_per_seq, _ptr(context_lens), new_tokens, softmax_scale, num_splits,
         _ptr(workspace), workspace_bytes, _ptr(out), B, Hq, Hkv, d, page_size, num_pages,
-        max_context_len, _ptr(status_flag), _stream(stream), _options(window, fused_merge, row_order)),
-        "ac_paged_decode_attn_ex")
+        max_context_len, _ptr(status_flag), _stream(stream),
+        ctypes.byref(_options(window, fused_merge, row_order))), "ac_paged_decode_attn_ex")
 
 
 def ac_decode_step_fused_ex(q_in, q_rot_out, k_new, v_new, k_cache, v_cache, stride_page, stride_token,
                             stride_head, block_table, max_pages_per_seq, context_lens, rope_cos, rope_sin,
                             max_position, softmax_scale, num_splits, workspace, workspace_bytes, out, B,
                             Hq, Hkv, d, page_size, num_pages, max_context_len, status_flag=None,
-                            stream=None, window=0, row_order=None):
+                            stream=None, window=0, row_order=None, rotary_dim=0, interleaved=False,
+                            q_norm_weight=None, k_norm_weight=None, norm_eps=0.0):
+    """The rope keywords are those of ac_rope_kv_append_ex (all default = the plain rotation)."""
+    variants = rotary_dim or interleaved or q_norm_weight is not None or k_norm_weight is not None
+    rope = _rope_options(rotary_dim, interleaved, q_norm_weight, k_norm_weight, norm_eps) if variants else None
+    opt = _options(window, False, row_order, rope)
     _check(lib().ac_decode_step_fused_ex(
         _ptr(q_in), _ptr(q_rot_out), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), stride_page,
         stride_token, stride_head, _ptr(block_table), max_pages_per_seq, _ptr(context_lens),
         _ptr(rope_cos), _ptr(rope_sin), max_position, softmax_scale, num_splits, _ptr(workspace),
         workspace_bytes, _ptr(out), B, Hq, Hkv, d, page_size, num_pages, max_context_len,
-        _ptr(status_flag), _stream(stream), _options(window, False, row_order)), "ac_decode_step_fused_ex")
+        _ptr(status_flag), _stream(stream), ctypes.byref(opt)), "ac_decode_step_fused_ex")
 
 
 def ac_splitkv_merge(workspace, num_splits, context_lens, out, B, Hq, d, stream=None):

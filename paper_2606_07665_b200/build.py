@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(PKG_DIR, "libac.so")
 SOURCES = ["ac_api.cu", "rope_kv_append.cu", "paged_decode_attn.cu", "splitkv_merge.cu",
            "attn_static_scratch.cu", "qkv_prelude.cu", "stage_inputs.cu", "proj_tc.cu", "hbm_probe.cu"]
 HEADERS = [os.path.join(CSRC, "ac_device.cuh"), os.path.join(CSRC, "ac_internal.h"),
+           os.path.join(CSRC, "rope_variant.cuh"),
            os.path.join(ROOT, "include", "ac.h")]
 
 

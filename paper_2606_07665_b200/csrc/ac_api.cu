@@ -316,6 +316,28 @@ int ac_decode_plan_for_lengths(const int32_t* token_counts_host, int B, int Hq, 
                        num_splits_out, split_tokens_out, workspace_bytes_out);
 }
 
+// Checks ac_rope_options and translates them; *out stays nullptr when they describe the plain rotation.
+static int parse_rope_options(const ac_rope_options* options, int d, RopeVariant* variant,
+                              const RopeVariant** out) {
+    *out = nullptr;
+    if (options == nullptr) return AC_OK;
+    const int rd = options->rotary_dim == 0 ? d : options->rotary_dim;
+    if (rd < 2 || rd > d || (rd & 1)) return AC_ERR_SHAPE;
+    const bool plain = rd == d && !options->interleaved && !options->q_norm_weight && !options->k_norm_weight;
+    if (plain) return AC_OK;
+    variant->rotary_dim = rd;
+    variant->interleaved = options->interleaved ? 1 : 0;
+    variant->q_norm_weight = options->q_norm_weight;
+    variant->k_norm_weight = options->k_norm_weight;
+    variant->norm_eps = options->norm_eps;
+    if ((variant->q_norm_weight || variant->k_norm_weight) && !(options->norm_eps >= 0.0f)) return AC_ERR_SHAPE;
+    if ((variant->q_norm_weight && !aligned16(variant->q_norm_weight)) ||
+        (variant->k_norm_weight && !aligned16(variant->k_norm_weight)))
+        return AC_ERR_ALIGN;
+    *out = variant;
+    return AC_OK;
+}
+
 int ac_rope_kv_append_ex(const void* q_in, void* q_out, const void* k_new, const void* v_new,
                          void* k_cache, void* v_cache, int64_t stride_page, int64_t stride_token,
                          int64_t stride_head, const int32_t* block_table, int max_pages_per_seq,
@@ -336,22 +358,8 @@ int ac_rope_kv_append_ex(const void* q_in, void* q_out, const void* k_new, const
         return AC_ERR_ALIGN;
     RopeVariant variant;
     const RopeVariant* vp = nullptr;
-    if (options != nullptr) {
-        const int rd = options->rotary_dim == 0 ? d : options->rotary_dim;
-        if (rd < 2 || rd > d || (rd & 1)) return AC_ERR_SHAPE;
-        const bool plain = rd == d && !options->interleaved && !options->q_norm_weight &&
-                           !options->k_norm_weight;
-        if (!plain) {
-            variant.rotary_dim = rd;
-            variant.interleaved = options->interleaved ? 1 : 0;
-            variant.q_norm_weight = options->q_norm_weight;
-            variant.k_norm_weight = options->k_norm_weight;
-            variant.norm_eps = options->norm_eps;
-            if ((variant.q_norm_weight || variant.k_norm_weight) && !(options->norm_eps >= 0.0f))
-                return AC_ERR_SHAPE;
-            vp = &variant;
-        }
-    }
+    st = parse_rope_options(options, d, &variant, &vp);
+    if (st != AC_OK) return st;
     int dev;
     st = current_ready_device(&dev);
     if (st != AC_OK) return st;
@@ -661,7 +669,12 @@ static int decode_step_fused_impl(const void* q_in, void* q_rot_out, const void*
     if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(rope_cos) || !aligned16(rope_sin) ||
         (q_rot_out && !aligned16(q_rot_out)))
         return AC_ERR_ALIGN;
+    RopeVariant variant;
+    const RopeVariant* vp = nullptr;
+    const int pst = parse_rope_options(options != nullptr ? options->rope : nullptr, d, &variant, &vp);
+    if (pst != AC_OK) return pst;
     FusedRopeArgs rope;
+    rope.variant = vp;
     rope.q_rot_out = q_rot_out;
     rope.k_new = k_new;
     rope.v_new = v_new;

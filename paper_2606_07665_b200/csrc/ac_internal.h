@@ -37,6 +37,15 @@ struct CacheView {
     int num_pages, page_size, Hkv, d;
 };
 
+// Prelude variants of the RoPE + append kernel and of the fused step (validated by the ABI layer).
+struct RopeVariant {
+    int rotary_dim;               // even, 2 .. d
+    int interleaved;              // 0: pair (i, i + rotary_dim/2); 1: pair (2i, 2i + 1)
+    const void* q_norm_weight;    // bf16 [d] or nullptr
+    const void* k_norm_weight;    // bf16 [d] or nullptr
+    float norm_eps;
+};
+
 // Extra inputs of the fused step: the attention kernel itself rotates q/k and appends k/v.
 struct FusedRopeArgs {
     void* q_rot_out;          // optional
@@ -49,15 +58,7 @@ struct FusedRopeArgs {
     const float* rope_sin;
     int max_position, num_pages;
     void* out_mirror;         // optional: a second copy of the bf16 result, e.g. in host memory the GPU can write
-};
-
-// Prelude variants of the RoPE + append kernel (validated by the ABI layer).
-struct RopeVariant {
-    int rotary_dim;               // even, 2 .. d
-    int interleaved;              // 0: pair (i, i + rotary_dim/2); 1: pair (2i, 2i + 1)
-    const void* q_norm_weight;    // bf16 [d] or nullptr
-    const void* k_norm_weight;    // bf16 [d] or nullptr
-    float norm_eps;
+    const RopeVariant* variant;   // optional: prelude variants applied to q and k_new (nullptr: plain rotation)
 };
 
 // Per-kernel launchers; each validates nothing (the ABI layer did) and returns a cudaError_t.

@@ -32,6 +32,7 @@
 
 #include "ac_device.cuh"
 #include "ac_internal.h"
+#include "rope_variant.cuh"
 
 namespace ac {
 namespace {
@@ -90,7 +91,17 @@ struct AttnParams {
     int window;                   // > 0: attend over the last `window` tokens of each row only
     int cluster_merge;            // 1: the splits of a (request, KV head) are one thread-block cluster and
                                   //    split 0 merges them out of the others' shared memory
+    // -- only for the fused step with prelude variants (ROPE = 2)
+    int rotary_dim;               // even, 2 .. D: elements [0, rotary_dim) rotate; tables are [max_position, rotary_dim/2]
+    int interleaved;              // 0: pair (i, i + rotary_dim/2); 1: pair (2i, 2i + 1)
+    const uint16_t* q_norm_w;     // bf16 [D] or nullptr: RMSNorm of every q head vector before the rotation
+    const uint16_t* k_norm_w;     // same for k
+    float norm_eps;
 };
+
+// Rotation flavours of the kernel: none (q arrives rotated), the plain rotate-half of the fused step,
+// and the fused step with the prelude variants (per-head RMSNorm, partial rotary, interleaved pairing).
+constexpr int ROPE_NONE = 0, ROPE_PLAIN = 1, ROPE_VARIANT = 2;
 
 // ---- thread-block cluster helpers (fused merge through distributed shared memory) ------------------
 __device__ __forceinline__ uint32_t cluster_map_shared(uint32_t local_addr, uint32_t rank) {
@@ -118,7 +129,7 @@ __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-template <int D, bool WIDE, bool ROPE>
+template <int D, bool WIDE, int ROPE>
 __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
     const AttnParams p) {
@@ -279,7 +290,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
 
     // Fused step: the rotary angles of this CTA's query rows depend only on ctx; fetch them now so
     // that they are in registers when q itself can be read (after the dependency is met).
-    constexpr int QP = ROPE ? (16 * (D / 2) + THREADS - 1) / THREADS : 1;   // rotary pairs per thread
+    constexpr int QP = ROPE == ROPE_PLAIN ? (16 * (D / 2) + THREADS - 1) / THREADS : 1;   // rotary pairs per thread
     // The new token can be appended only if its position has a rope-table row, a block-table entry
     // and a tile in this launch's split grid (max_context_len too small for the row otherwise).
     const bool rope_ok = ROPE && ctx < p.max_position &&
@@ -287,7 +298,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
                          static_cast<long long>(ctx) <
                              window_base + static_cast<long long>(S) * p.split_tokens;
     float q_cos[QP], q_sin[QP];
-    if (ROPE) {
+    if (ROPE == ROPE_PLAIN) {
         const float* cos_row = p.rope_cos + static_cast<size_t>(ctx) * (D / 2);
         const float* sin_row = p.rope_sin + static_cast<size_t>(ctx) * (D / 2);
 #pragma unroll
@@ -318,7 +329,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     int page_next = issued < n_my ? load_page_id(issued) : 0;
     if (!dependency_met) dependency_sync();                    // q was written by the preceding kernel
     uint16_t q_raw_lo[QP], q_raw_hi[QP];
-    if (ROPE) {
+    if (ROPE == ROPE_PLAIN) {
         const uint16_t* qsrc = p.q + (static_cast<size_t>(b) * p.Hq + h * G) * D;
 #pragma unroll
         for (int k = 0; k < QP; ++k) {
@@ -333,7 +344,10 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
 
     // ---- fused step: rotate and append the new k/v early, under the latency of the first tiles ------
     constexpr int APPEND_PAIRS = D / 64;          // rotary pairs per lane (D/2 pairs over 32 lanes)
+    constexpr int EPL = D / 32;                   // variants: lane l holds elements l*EPL .. l*EPL + EPL - 1
     uint16_t k_rot_lo[APPEND_PAIRS], k_rot_hi[APPEND_PAIRS];
+    uint16_t k_var[EPL];
+    __shared__ uint16_t s_kpark[ROPE == ROPE_VARIANT ? D : 8];     // the appending warp's parked k vector
     uint2 v_new4 = make_uint2(0u, 0u);
     int append_j = -1;                            // index of this warp's tile that holds the new slot
     bool append_ok = false;
@@ -353,17 +367,29 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
                                     static_cast<size_t>(h) * p.stride_head;
                 const uint16_t* ksrc = p.k_new + (static_cast<size_t>(b) * p.Hkv + h) * D;
                 const uint16_t* vsrc = p.v_new + (static_cast<size_t>(b) * p.Hkv + h) * D;
-                const float* cos_row = p.rope_cos + static_cast<size_t>(ctx) * (D / 2);
-                const float* sin_row = p.rope_sin + static_cast<size_t>(ctx) * (D / 2);
+                if (ROPE == ROPE_VARIANT) {
+                    const int half_r = p.rotary_dim / 2;
 #pragma unroll
-                for (int u = 0; u < APPEND_PAIRS; ++u) {
-                    const int i = lane + 32 * u;
-                    const uint16_t a = ksrc[i], bb = ksrc[i + D / 2];
-                    const float c = cos_row[i], sn = sin_row[i];
-                    k_rot_lo[u] = rope_first_half(a, bb, c, sn);
-                    k_rot_hi[u] = rope_second_half(a, bb, c, sn);
-                    p.k_cache[goff + i] = k_rot_lo[u];
-                    p.k_cache[goff + i + D / 2] = k_rot_hi[u];
+                    for (int e = 0; e < EPL; ++e) k_var[e] = ksrc[lane * EPL + e];
+                    rope_variant_vector<D>(k_var, p.k_norm_w, p.norm_eps,
+                                           p.rope_cos + static_cast<size_t>(ctx) * half_r,
+                                           p.rope_sin + static_cast<size_t>(ctx) * half_r, p.rotary_dim,
+                                           p.interleaved, s_kpark, lane);
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) p.k_cache[goff + lane * EPL + e] = k_var[e];
+                } else {
+                    const float* cos_row = p.rope_cos + static_cast<size_t>(ctx) * (D / 2);
+                    const float* sin_row = p.rope_sin + static_cast<size_t>(ctx) * (D / 2);
+#pragma unroll
+                    for (int u = 0; u < APPEND_PAIRS; ++u) {
+                        const int i = lane + 32 * u;
+                        const uint16_t a = ksrc[i], bb = ksrc[i + D / 2];
+                        const float c = cos_row[i], sn = sin_row[i];
+                        k_rot_lo[u] = rope_first_half(a, bb, c, sn);
+                        k_rot_hi[u] = rope_second_half(a, bb, c, sn);
+                        p.k_cache[goff + i] = k_rot_lo[u];
+                        p.k_cache[goff + i + D / 2] = k_rot_hi[u];
+                    }
                 }
                 if (lane * 4 < D) {
                     v_new4 = *reinterpret_cast<const uint2*>(vsrc + lane * 4);
@@ -379,7 +405,42 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     uint32_t qa[KSTEPS][2 * ROWS];
     constexpr int QSTRIDE = D + 8;                 // padded row: fragment loads hit 32 distinct banks
     __shared__ __align__(16) uint16_t s_q[ROPE ? 16 * QSTRIDE : 8];
-    if (ROPE) {
+    if (ROPE == ROPE_VARIANT) {
+        // Prelude variants: one warp per query row (rows warp, warp + 6, ...): optional RMSNorm, then the
+        // partial / interleaved rotation, with the row's place in the shared tile as the parking space
+        // for the partner look-ups.  Same arithmetic as the stand-alone variant kernel.
+        uint16_t* qdst = (p.q_rot_out != nullptr && split == 0)
+                             ? p.q_rot_out + (static_cast<size_t>(b) * p.Hq + h * G) * D : nullptr;
+        const uint16_t* qsrc = p.q + (static_cast<size_t>(b) * p.Hq + h * G) * D;
+        const int half_r = p.rotary_dim / 2;
+        for (int row = warp; row < (WIDE ? 16 : 8); row += WARPS) {
+            uint16_t xq[EPL];
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) xq[e] = row < G ? qsrc[row * D + lane * EPL + e] : static_cast<uint16_t>(0);
+            if (row < G && rope_ok) {
+                rope_variant_vector<D>(xq, p.q_norm_w, p.norm_eps, p.rope_cos + static_cast<size_t>(ctx) * half_r,
+                                       p.rope_sin + static_cast<size_t>(ctx) * half_r, p.rotary_dim, p.interleaved,
+                                       s_q + row * QSTRIDE, lane);
+                if (qdst != nullptr) {
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) qdst[row * D + lane * EPL + e] = xq[e];
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) s_q[row * QSTRIDE + lane * EPL + e] = xq[e];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < KSTEPS; ++kk) {
+            const int col = kk * 16 + 2 * t;
+            qa[kk][0] = *reinterpret_cast<const uint32_t*>(s_q + g * QSTRIDE + col);
+            qa[kk][ROWS] = *reinterpret_cast<const uint32_t*>(s_q + g * QSTRIDE + col + 8);
+            if (WIDE) {
+                qa[kk][1] = *reinterpret_cast<const uint32_t*>(s_q + (g + 8) * QSTRIDE + col);
+                qa[kk][ROWS + 1] = *reinterpret_cast<const uint32_t*>(s_q + (g + 8) * QSTRIDE + col + 8);
+            }
+        }
+    } else if (ROPE) {
         // The CTA rotates its G query rows once (pair i with i + D/2, exact then rounded, as the
         // stand-alone kernel does) into shared memory; every warp then reads its fragments from there.
         uint16_t* qdst = (p.q_rot_out != nullptr && split == 0)
@@ -480,11 +541,17 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
                 return (col >> 6) * L::HALF_BYTES + slot_in_tile * 128 +
                        ((((col & 63) >> 3) ^ (slot_in_tile & 7)) << 4) + ((col & 7) << 1);
             };
+            if (ROPE == ROPE_VARIANT) {
 #pragma unroll
-            for (int u = 0; u < APPEND_PAIRS; ++u) {
-                const int i = lane + 32 * u;
-                *reinterpret_cast<uint16_t*>(smem_gen + (kbase - smem_base) + tile_byte(i)) = k_rot_lo[u];
-                *reinterpret_cast<uint16_t*>(smem_gen + (kbase - smem_base) + tile_byte(i + D / 2)) = k_rot_hi[u];
+                for (int e = 0; e < EPL; ++e)
+                    *reinterpret_cast<uint16_t*>(smem_gen + (kbase - smem_base) + tile_byte(lane * EPL + e)) = k_var[e];
+            } else {
+#pragma unroll
+                for (int u = 0; u < APPEND_PAIRS; ++u) {
+                    const int i = lane + 32 * u;
+                    *reinterpret_cast<uint16_t*>(smem_gen + (kbase - smem_base) + tile_byte(i)) = k_rot_lo[u];
+                    *reinterpret_cast<uint16_t*>(smem_gen + (kbase - smem_base) + tile_byte(i + D / 2)) = k_rot_hi[u];
+                }
             }
             if (lane * 4 < D)
                 *reinterpret_cast<uint2*>(smem_gen + (vbase - smem_base) + tile_byte(lane * 4)) = v_new4;
@@ -784,7 +851,7 @@ __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     }
 }
 
-template <int D, bool WIDE, bool ROPE>
+template <int D, bool WIDE, int ROPE>
 cudaError_t launch_one(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnParams& p_in, int B,
                        cudaStream_t stream) {
     AttnParams p = p_in;
@@ -834,23 +901,20 @@ cudaError_t launch_one(const CUtensorMap& k_map, const CUtensorMap& v_map, const
 cudaError_t attn_set_attributes(int smem_optin) {
     if (Smem<128>::TOTAL > smem_optin) return cudaErrorInvalidConfiguration;
     cudaError_t e;
-#define AC_SET(D_, W_)                                                                             \
-    e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, false>,                              \
+#define AC_SET_ONE(D_, W_, R_)                                                                     \
+    e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, R_>,                                 \
                              cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D_>::TOTAL);        \
     if (e != cudaSuccess) return e;                                                                \
-    e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, true>,                               \
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D_>::TOTAL);        \
-    if (e != cudaSuccess) return e;                                                                \
-    e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, false>,                              \
-                             cudaFuncAttributeNonPortableClusterSizeAllowed, 1);                   \
-    if (e != cudaSuccess) return e;                                                                \
-    e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, true>,                               \
+    e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, R_>,                                 \
                              cudaFuncAttributeNonPortableClusterSizeAllowed, 1);                   \
     if (e != cudaSuccess) return e;
+#define AC_SET(D_, W_)                                                                             \
+    AC_SET_ONE(D_, W_, ROPE_NONE) AC_SET_ONE(D_, W_, ROPE_PLAIN) AC_SET_ONE(D_, W_, ROPE_VARIANT)
     AC_SET(128, false)
     AC_SET(128, true)
     AC_SET(64, false)
     AC_SET(64, true)
+#undef AC_SET_ONE
 #undef AC_SET
     return cudaSuccess;
 }
@@ -920,21 +984,38 @@ cudaError_t launch_paged_decode_attn(const CUtensorMap& k_map, const CUtensorMap
     p.Hq = Hq;
     p.Hkv = Hkv;
     p.page_size = page_size;
+    p.rotary_dim = d;
+    p.interleaved = 0;
+    p.q_norm_w = p.k_norm_w = nullptr;
+    p.norm_eps = 0.0f;
     const bool wide = Hq / Hkv > 8;
+    if (rope != nullptr && rope->variant != nullptr) {
+        p.rotary_dim = rope->variant->rotary_dim;
+        p.interleaved = rope->variant->interleaved;
+        p.q_norm_w = static_cast<const uint16_t*>(rope->variant->q_norm_weight);
+        p.k_norm_w = static_cast<const uint16_t*>(rope->variant->k_norm_weight);
+        p.norm_eps = rope->variant->norm_eps;
+        if (d == 128) {
+            return wide ? launch_one<128, true, ROPE_VARIANT>(k_map, v_map, p, B, stream)
+                        : launch_one<128, false, ROPE_VARIANT>(k_map, v_map, p, B, stream);
+        }
+        return wide ? launch_one<64, true, ROPE_VARIANT>(k_map, v_map, p, B, stream)
+                    : launch_one<64, false, ROPE_VARIANT>(k_map, v_map, p, B, stream);
+    }
     if (rope != nullptr) {
         if (d == 128) {
-            return wide ? launch_one<128, true, true>(k_map, v_map, p, B, stream)
-                        : launch_one<128, false, true>(k_map, v_map, p, B, stream);
+            return wide ? launch_one<128, true, ROPE_PLAIN>(k_map, v_map, p, B, stream)
+                        : launch_one<128, false, ROPE_PLAIN>(k_map, v_map, p, B, stream);
         }
-        return wide ? launch_one<64, true, true>(k_map, v_map, p, B, stream)
-                    : launch_one<64, false, true>(k_map, v_map, p, B, stream);
+        return wide ? launch_one<64, true, ROPE_PLAIN>(k_map, v_map, p, B, stream)
+                    : launch_one<64, false, ROPE_PLAIN>(k_map, v_map, p, B, stream);
     }
     if (d == 128) {
-        return wide ? launch_one<128, true, false>(k_map, v_map, p, B, stream)
-                    : launch_one<128, false, false>(k_map, v_map, p, B, stream);
+        return wide ? launch_one<128, true, ROPE_NONE>(k_map, v_map, p, B, stream)
+                    : launch_one<128, false, ROPE_NONE>(k_map, v_map, p, B, stream);
     }
-    return wide ? launch_one<64, true, false>(k_map, v_map, p, B, stream)
-                : launch_one<64, false, false>(k_map, v_map, p, B, stream);
+    return wide ? launch_one<64, true, ROPE_NONE>(k_map, v_map, p, B, stream)
+                : launch_one<64, false, ROPE_NONE>(k_map, v_map, p, B, stream);
 }
 
 }  // namespace ac

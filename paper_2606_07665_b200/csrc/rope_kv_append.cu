@@ -12,6 +12,7 @@
 // round-to-nearest-even identical to a direct rounding of the fp64 value.
 #include "ac_device.cuh"
 #include "ac_internal.h"
+#include "rope_variant.cuh"
 
 namespace ac {
 namespace {
@@ -163,56 +164,11 @@ __global__ void __launch_bounds__(128) rope_kv_append_ex_kernel(
     uint16_t x[EPL];
 #pragma unroll
     for (int e = 0; e < EPL; ++e) x[e] = src[lane * EPL + e];
-    if (norm_w != nullptr) {
-        double ss = 0.0;
+    acdev::rope_variant_vector<D>(x, norm_w, norm_eps, rope_cos + static_cast<size_t>(p) * (rotary_dim / 2),
+                                  rope_sin + static_cast<size_t>(p) * (rotary_dim / 2), rotary_dim, interleaved,
+                                  s_vec[warp], lane);
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) {
-            const double v = static_cast<double>(acdev::bf16_bits_to_float(x[e]));
-            ss = __dadd_rn(ss, __dmul_rn(v, v));
-        }
-#pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) ss = __dadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, off));
-        const double r = __ddiv_rn(1.0, __dsqrt_rn(__dadd_rn(__ddiv_rn(ss, static_cast<double>(D)),
-                                                             static_cast<double>(norm_eps))));
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) {
-            const double v = static_cast<double>(acdev::bf16_bits_to_float(x[e]));
-            const uint16_t y1 = acdev::f64_to_bf16_rne(__dmul_rn(v, r));
-            const double w = static_cast<double>(acdev::bf16_bits_to_float(norm_w[lane * EPL + e]));
-            x[e] = acdev::f64_to_bf16_rne(__dmul_rn(static_cast<double>(acdev::bf16_bits_to_float(y1)), w));
-        }
-    }
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) s_vec[warp][lane * EPL + e] = x[e];
-    __syncwarp();
-
-    const int half = rotary_dim / 2;
-    uint16_t out[EPL];
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-        const int j = lane * EPL + e;
-        if (j >= rotary_dim) {
-            out[e] = x[e];
-            continue;
-        }
-        int i, partner;
-        bool first;
-        if (interleaved) {
-            i = j >> 1;
-            first = (j & 1) == 0;
-            partner = first ? j + 1 : j - 1;
-        } else {
-            first = j < half;
-            i = first ? j : j - half;
-            partner = first ? j + half : j - half;
-        }
-        const float c = rope_cos[static_cast<size_t>(p) * half + i];
-        const float sn = rope_sin[static_cast<size_t>(p) * half + i];
-        const uint16_t other = s_vec[warp][partner];
-        out[e] = first ? acdev::rope_first_half(x[e], other, c, sn) : acdev::rope_second_half(other, x[e], c, sn);
-    }
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) dst[lane * EPL + e] = out[e];
+    for (int e = 0; e < EPL; ++e) dst[lane * EPL + e] = x[e];
     if (!is_q) {
         const uint16_t* src_v = v_new + (static_cast<size_t>(b) * Hkv + (hh - Hq)) * D;
 #pragma unroll

@@ -138,7 +138,9 @@ class DecodeStep:
             ac.ac_splitkv_merge(self.workspace, self.num_splits, self.context_lens, self.out, self.B,
                                 self.Hq, self.d, stream)
 
-    def decode_step_fused(self, stream=None) -> None:
+    def decode_step_fused(self, stream=None, **rope_variants) -> None:
+        """rope_variants: rotary_dim, interleaved, q_norm_weight, k_norm_weight, norm_eps (prelude
+        variants applied inside the step; norm weights are device int16 tensors holding bf16 bits)."""
         ac.ac_decode_step_fused_ex(self.q_in, self.q_rot, self.k_new, self.v_new, self.k_cache,
                                    self.v_cache, self.stride_page, self.stride_token, self.stride_head,
                                    self.block_table, self.w.max_pages_per_seq, self.context_lens,
@@ -146,7 +148,7 @@ class DecodeStep:
                                    self.workspace if self.num_splits > 1 else None, self.workspace_bytes,
                                    self.out, self.B, self.Hq, self.Hkv, self.d, self.ps, self.num_pages,
                                    self.max_context_len, self.status_flag, stream, window=self.window,
-                                   row_order=self.row_order)
+                                   row_order=self.row_order, **rope_variants)
 
     def step(self, stream=None) -> None:
         if self.fused_step:

@@ -123,8 +123,11 @@ def test_rope_constructed_near_tie(rt):
     dict(norm="q_only"),
     dict(),                                                    # options present but plain
 ])
+@pytest.mark.parametrize("path", ["kernel", "step"])
 @pytest.mark.parametrize("d", [128, 64])
-def test_rope_prelude_variants_bit_exact_and_feed_attention(rt, kw, d):
+def test_rope_prelude_variants_bit_exact_and_feed_attention(rt, kw, d, path):
+    # path "kernel": the stand-alone variant kernel followed by attention; "step": the same variants
+    # applied inside the single-launch step (ac_decode_step_fused_ex with rope options)
     import torch
     kw = dict(kw)
     norm = kw.pop("norm", False)
@@ -141,11 +144,18 @@ def test_rope_prelude_variants_bit_exact_and_feed_attention(rt, kw, d):
         w.page_size, rotary_dim=rotary_dim or None, interleaved=interleaved, q_norm_weight=qw,
         k_norm_weight=kw_bits, norm_eps=1e-6)
     out_ref = O.oracle_paged_decode_attn(q_rot, k_after, v_after, w.block_table, w.context_lens, w.page_size)
-    st = rt.DecodeStep(w, num_splits=2)
+    st = rt.DecodeStep(w, num_splits=2, fused_step=(path == "step"))
     dev = lambda a: None if a is None else torch.from_numpy(a.view(np.int16)).cuda()
-    st.rope_kv_append_ex(rotary_dim=rotary_dim, interleaved=interleaved, q_norm_weight=dev(qw),
-                         k_norm_weight=dev(kw_bits), norm_eps=1e-6)
-    st.attention()
+    if path == "step":
+        st.q_rot.fill_(0x7FC0)
+        st.decode_step_fused(rotary_dim=rotary_dim, interleaved=interleaved, q_norm_weight=dev(qw),
+                             k_norm_weight=dev(kw_bits), norm_eps=1e-6)
+        torch.cuda.synchronize()
+        st.q_rot[2] = st.q_in[2]                      # the inactive row's q is not written by the step
+    else:
+        st.rope_kv_append_ex(rotary_dim=rotary_dim, interleaved=interleaved, q_norm_weight=dev(qw),
+                             k_norm_weight=dev(kw_bits), norm_eps=1e-6)
+        st.attention()
     torch.cuda.synchronize()
     assert int(st.status_flag.item()) == 0
     assert np.array_equal(rt.bits_of(st.q_rot), q_rot), "q after norm/rotation differs"
