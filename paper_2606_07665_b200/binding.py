@@ -28,7 +28,7 @@ EXPORTS = ("ac_init", "ac_status_string", "ac_last_cuda_error", "ac_sm_count", "
            "ac_fused_workspace_bytes", "ac_fused_workspace_reset", "ac_paged_decode_attn_fused_merge",
            "ac_decode_step_fused", "ac_paged_decode_attn_ex", "ac_decode_step_fused_ex",
            "ac_rope_kv_append_ex", "ac_qkv_rope_kv_append", "ac_oproj_residual_rmsnorm",
-           "ac_hbm_read_probe")
+           "ac_hbm_read_probe", "ac_qkv_rope_kv_append_ex")
 AC_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -90,6 +90,8 @@ def lib():
                                             [c_int64] * 3 + [c_void_p, c_int, c_void_p, c_void_p, c_void_p,
                                             c_int] + [c_int] * 6 + [c_void_p, c_void_p])
         L.ac_qkv_rope_kv_append.restype = c_int
+        L.ac_qkv_rope_kv_append_ex.argtypes = L.ac_qkv_rope_kv_append.argtypes + [POINTER(AcRopeOptions)]
+        L.ac_qkv_rope_kv_append_ex.restype = c_int
         L.ac_oproj_residual_rmsnorm.argtypes = [c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p,
                                                 c_float, c_void_p, c_int, c_void_p]
         L.ac_oproj_residual_rmsnorm.restype = c_int
@@ -218,6 +220,20 @@ def ac_qkv_rope_kv_append(x, w_qkv, H, q_out, k_cache, v_cache, stride_page, str
                                        max_pages_per_seq, _ptr(context_lens), _ptr(rope_cos),
                                        _ptr(rope_sin), max_position, B, Hq, Hkv, d, page_size, num_pages,
                                        _ptr(status_flag), _stream(stream)), "ac_qkv_rope_kv_append")
+
+
+def ac_qkv_rope_kv_append_ex(x, w_qkv, H, q_out, k_cache, v_cache, stride_page, stride_token, stride_head,
+                             block_table, max_pages_per_seq, context_lens, rope_cos, rope_sin, max_position,
+                             B, Hq, Hkv, d, page_size, num_pages, status_flag=None, stream=None,
+                             rotary_dim=0, interleaved=False, q_norm_weight=None, k_norm_weight=None,
+                             norm_eps=0.0):
+    opt = _rope_options(rotary_dim, interleaved, q_norm_weight, k_norm_weight, norm_eps)
+    _check(lib().ac_qkv_rope_kv_append_ex(_ptr(x), _ptr(w_qkv), H, _ptr(q_out), _ptr(k_cache), _ptr(v_cache),
+                                          stride_page, stride_token, stride_head, _ptr(block_table),
+                                          max_pages_per_seq, _ptr(context_lens), _ptr(rope_cos),
+                                          _ptr(rope_sin), max_position, B, Hq, Hkv, d, page_size, num_pages,
+                                          _ptr(status_flag), _stream(stream), ctypes.byref(opt)),
+           "ac_qkv_rope_kv_append_ex")
 
 
 def ac_oproj_residual_rmsnorm(attn_out, w_o, K, N, residual_in, residual_out, norm_weight, norm_eps,

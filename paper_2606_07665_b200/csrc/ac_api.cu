@@ -389,6 +389,18 @@ int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out, 
                           const int32_t* context_lens, const float* rope_cos, const float* rope_sin,
                           int max_position, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
                           int32_t* status_flag, void* stream) {
+    return ac_qkv_rope_kv_append_ex(x, w_qkv, H, q_out, k_cache, v_cache, stride_page, stride_token,
+                                    stride_head, block_table, max_pages_per_seq, context_lens, rope_cos,
+                                    rope_sin, max_position, B, Hq, Hkv, d, page_size, num_pages, status_flag,
+                                    stream, nullptr);
+}
+
+int ac_qkv_rope_kv_append_ex(const void* x, const void* w_qkv, int H, void* q_out, void* k_cache,
+                             void* v_cache, int64_t stride_page, int64_t stride_token, int64_t stride_head,
+                             const int32_t* block_table, int max_pages_per_seq,
+                             const int32_t* context_lens, const float* rope_cos, const float* rope_sin,
+                             int max_position, int B, int Hq, int Hkv, int d, int page_size, int num_pages,
+                             int32_t* status_flag, void* stream, const ac_rope_options* options) {
     if (!x || !w_qkv || !q_out || !k_cache || !v_cache || !block_table || !context_lens || !rope_cos ||
         !rope_sin)
         return AC_ERR_NULL;
@@ -402,6 +414,10 @@ int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out, 
     if (!aligned16(x) || !aligned16(w_qkv) || !aligned16(q_out) || !aligned16(k_cache) ||
         !aligned16(v_cache))
         return AC_ERR_ALIGN;
+    RopeVariant variant;
+    const RopeVariant* vp = nullptr;
+    st = parse_rope_options(options, d, &variant, &vp);
+    if (st != AC_OK) return st;
     int dev;
     st = current_ready_device(&dev);
     if (st != AC_OK) return st;
@@ -410,7 +426,8 @@ int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out, 
     // x [B, H] as (64 elements, batch row, 64-element K block).
     const cuuint64_t row_bytes = static_cast<cuuint64_t>(H) * 2;
     CUtensorMap w_map, x_map;
-    if (B > kWarpMmaMaxBatch) {
+    // The prelude variants run on the warp-MMA kernel at every batch size (16 rows per grid slice).
+    if (B > kWarpMmaMaxBatch && vp == nullptr) {
         // Batched decode: batch tiles of up to 128 rows on the tcgen05 path (boxes of 24 pairs x 2 K blocks).
         cuuint64_t wdims[5] = {64, static_cast<cuuint64_t>(d / 2), 2, static_cast<cuuint64_t>(Hq + 2 * Hkv),
                                static_cast<cuuint64_t>(H / 64)};
@@ -463,7 +480,7 @@ int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out, 
     cudaError_t e = launch_qkv_rope_kv_append(w_map, x_map, q_out, k_cache, v_cache, stride_page,
                                               stride_token, stride_head, block_table, max_pages_per_seq,
                                               context_lens, rope_cos, rope_sin, max_position, B, H, Hq,
-                                              Hkv, d, page_size, num_pages, status_flag,
+                                              Hkv, d, page_size, num_pages, status_flag, vp,
                                               static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
 }

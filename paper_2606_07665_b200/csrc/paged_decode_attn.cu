@@ -103,32 +103,6 @@ struct AttnParams {
 // and the fused step with the prelude variants (per-head RMSNorm, partial rotary, interleaved pairing).
 constexpr int ROPE_NONE = 0, ROPE_PLAIN = 1, ROPE_VARIANT = 2;
 
-// ---- thread-block cluster helpers (fused merge through distributed shared memory) ------------------
-__device__ __forceinline__ uint32_t cluster_map_shared(uint32_t local_addr, uint32_t rank) {
-    uint32_t r;                   // address of the same shared-memory location in CTA `rank` of the cluster
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ float4 cluster_load_f32x4(uint32_t cluster_addr) {
-    float4 v;
-    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                 : "r"(cluster_addr)
-                 : "memory");
-    return v;
-}
-__device__ __forceinline__ float cluster_load_f32(uint32_t cluster_addr) {
-    float v;
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
-    return v;
-}
-// Hardware barrier over the threads of the cluster (not a spin).  Every CTA of a cluster-merge launch
-// executes exactly two of them, on every path.
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-
 template <int D, bool WIDE, int ROPE>
 __global__ void __launch_bounds__(THREADS, 2) paged_decode_attn_kernel(
     const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,

@@ -30,7 +30,7 @@ namespace {
 
 using namespace acdev;
 
-enum { EPI_QKV_ROPE_APPEND = 0, EPI_RESIDUAL_ADD = 1 };
+enum { EPI_QKV_ROPE_APPEND = 0, EPI_RESIDUAL_ADD = 1, EPI_QKV_ROPE_VARIANT = 2 };
 
 constexpr int QKV_WARPS = 8;                          // consumer warps; warp QKV_WARPS produces
 constexpr int QKV_THREADS = (QKV_WARPS + 1) * 32;
@@ -41,7 +41,7 @@ constexpr int W_BLOCK_BYTES = 16 * 128;               // one swizzled [16 rows x
 // rotary pairs), 1 for the output projection (16 consecutive features; 256 CTAs for N = 4096, so that
 // most SMs stream for two CTAs -- 128 CTAs of 32 features left 20 SMs idle and the rest at the rate
 // of a single CTA).
-__host__ __device__ constexpr int row_blocks(int epi) { return epi == 1 ? 1 : 2; }
+__host__ __device__ constexpr int row_blocks(int epi) { return epi == EPI_RESIDUAL_ADD ? 1 : 2; }
 
 template <int BT, int RB>
 struct QkvSmem {
@@ -53,6 +53,11 @@ struct QkvSmem {
     static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
     static constexpr int TOTAL = BAR_OFFSET + 2 * STAGES * 8 + 1024;
     static_assert(QKV_WARPS * 16 * RB * BT * 4 <= STAGES * STAGE_BYTES, "reduction buffer must fit");
+    // prelude variants: behind the reduction buffer, the CTA's rounded features [32][BT] (bf16 bits), the
+    // same after the norm, and one fp64 sum of squares per batch row
+    static constexpr int VAR_OFFSET = QKV_WARPS * 16 * RB * BT * 4;
+    static constexpr int VAR_BYTES = 2 * 32 * BT * 2 + BT * 8;
+    static_assert(RB != 2 || VAR_OFFSET + VAR_BYTES <= STAGES * STAGE_BYTES, "variant buffers must fit");
 };
 
 struct QkvParams {
@@ -71,6 +76,11 @@ struct QkvParams {
     const uint16_t* residual_in;  // [B, N] bf16
     uint16_t* residual_out;       // [B, N] bf16 (may alias residual_in)
     int N;                        // output features
+    // prelude variants only (EPI_QKV_ROPE_VARIANT)
+    int rotary_dim, interleaved;
+    const uint16_t* q_norm_w;
+    const uint16_t* k_norm_w;
+    float norm_eps;
 };
 
 template <int BT, int EPI>
@@ -246,6 +256,110 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
         return;
     }
 
+    if (EPI == EPI_QKV_ROPE_VARIANT) {
+        // ---- epilogue with the prelude variants ------------------------------------------------------
+        // The d/32 CTAs that share a head (blockIdx.x) are one thread-block cluster.  A CTA holds 32 of
+        // the head's features; the per-head RMSNorm needs the sum of squares of all d, and partial or
+        // interleaved rotary pairs a feature with one that may live in a sister CTA.  So: every CTA
+        // parks its rounded features and their partial sum of squares in shared memory, a cluster
+        // barrier publishes them, the norm reads the sister CTAs' sums (fp64, exact, fixed order) and
+        // parks the normalised features, a second barrier publishes those, and the rotation fetches each
+        // partner from whichever CTA owns it.  A third barrier keeps every CTA's shared memory alive
+        // until its sisters are done reading.  Every CTA executes all three on every path.
+        const int d = p.d, half_d = d / 2;
+        uint16_t* vals = reinterpret_cast<uint16_t*>(smem_gen + L::VAR_OFFSET);      // [32][BT]
+        uint16_t* valsn = vals + 32 * BT;                                            // [32][BT] after the norm
+        double* sums = reinterpret_cast<double*>(valsn + 32 * BT);                   // [BT]
+        const bool is_q = hh < p.Hq, is_k = !is_q && hh < p.Hq + p.Hkv;
+        const uint16_t* norm_w = is_q ? p.q_norm_w : (is_k ? p.k_norm_w : nullptr);
+        const int n_cta = d / 32;                       // CTAs in the cluster
+        for (int item = threadIdx.x; item < 32 * BT; item += QKV_THREADS) {
+            const int r = item / BT, n = item - r * BT;
+            float y = 0.0f;
+#pragma unroll
+            for (int w = 0; w < QKV_WARPS; ++w) y += red[(w * TROWS + r) * BT + n];
+            vals[item] = static_cast<uint16_t>(pack_bf16x2(y, 0.0f) & 0xFFFFu);
+        }
+        __syncthreads();
+        if (threadIdx.x < BT) {
+            double ss = 0.0;
+            for (int r = 0; r < 32; ++r) {
+                const double v = static_cast<double>(bf16_bits_to_float(vals[r * BT + threadIdx.x]));
+                ss = __dadd_rn(ss, __dmul_rn(v, v));
+            }
+            sums[threadIdx.x] = ss;
+        }
+        cluster_sync_all();
+        for (int item = threadIdx.x; item < 32 * BT; item += QKV_THREADS) {
+            const int r = item / BT, n = item - r * BT;
+            uint16_t v16 = vals[item];
+            if (norm_w != nullptr) {
+                double total = 0.0;
+                for (int c = 0; c < n_cta; ++c)
+                    total = __dadd_rn(total, cluster_load_f64(cluster_map_shared(smem_addr(sums + n), c)));
+                const double rr = __ddiv_rn(1.0, __dsqrt_rn(__dadd_rn(__ddiv_rn(total, static_cast<double>(d)),
+                                                                      static_cast<double>(p.norm_eps))));
+                const int f = (r >> 4) * half_d + 16 * blk + (r & 15);               // feature inside the head
+                const uint16_t y1 = f64_to_bf16_rne(__dmul_rn(static_cast<double>(bf16_bits_to_float(v16)), rr));
+                v16 = f64_to_bf16_rne(__dmul_rn(static_cast<double>(bf16_bits_to_float(y1)),
+                                                static_cast<double>(bf16_bits_to_float(norm_w[f]))));
+            }
+            valsn[item] = v16;
+        }
+        cluster_sync_all();
+        const int R = p.rotary_dim, half_r = R / 2;
+        for (int item = threadIdx.x; item < 32 * BT; item += QKV_THREADS) {
+            const int r = item / BT, n = item - r * BT;
+            const int b = b0 + n;
+            if (b >= p.B) continue;
+            const int ctx = p.context_lens[b];
+            if (ctx < 0) continue;                         // inactive row
+            const int page_idx = ctx / p.page_size;
+            if (ctx >= p.max_position || page_idx >= p.max_pages_per_seq) {
+                if (p.status_flag != nullptr && r == 0 && blk == 0) atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
+                continue;
+            }
+            const int f = (r >> 4) * half_d + 16 * blk + (r & 15);
+            uint16_t v16 = valsn[item];
+            if ((is_q || is_k) && f < R) {
+                int i, partner;
+                bool first;
+                if (p.interleaved) {
+                    i = f >> 1;
+                    first = (f & 1) == 0;
+                    partner = first ? f + 1 : f - 1;
+                } else {
+                    first = f < half_r;
+                    i = first ? f : f - half_r;
+                    partner = first ? f + half_r : f - half_r;
+                }
+                // the partner feature lives in CTA (partner mod d/2) / 16 of the cluster, local row below
+                const int owner = (partner % half_d) >> 4;
+                const int prow = (partner / half_d) * 16 + (partner & 15);
+                const uint16_t other = cluster_load_u16(cluster_map_shared(smem_addr(valsn + prow * BT + n), owner));
+                const float c = p.rope_cos[static_cast<size_t>(ctx) * half_r + i];
+                const float sn = p.rope_sin[static_cast<size_t>(ctx) * half_r + i];
+                v16 = first ? rope_first_half(v16, other, c, sn) : rope_second_half(other, v16, c, sn);
+            }
+            if (is_q) {
+                p.q_out[(static_cast<size_t>(b) * p.Hq + hh) * d + f] = v16;
+            } else {
+                const int page = p.block_table[static_cast<size_t>(b) * p.max_pages_per_seq + page_idx];
+                if (page < 0 || page >= p.num_pages) {
+                    if (p.status_flag != nullptr && r == 0 && blk == 0) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
+                    continue;
+                }
+                const int h = is_k ? hh - p.Hq : hh - p.Hq - p.Hkv;
+                uint16_t* dst = (is_k ? p.k_cache : p.v_cache) + static_cast<size_t>(page) * p.stride_page +
+                                static_cast<size_t>(ctx - page_idx * p.page_size) * p.stride_token +
+                                static_cast<size_t>(h) * p.stride_head;
+                dst[f] = v16;
+            }
+        }
+        cluster_sync_all();
+        return;
+    }
+
     // ---- epilogue: round, rotate, scatter --------------------------------------------------------
     const int d = p.d, half = d / 2;
     for (int item = threadIdx.x; item < 16 * BT; item += QKV_THREADS) {
@@ -307,11 +421,15 @@ cudaError_t launch_qkv(const CUtensorMap& w_map, const CUtensorMap& x_map, const
     cfg.blockDim = dim3(QKV_THREADS);
     cfg.dynamicSmemBytes = QkvSmem<BT, row_blocks(EPI)>::TOTAL;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;     // prelude variants: the CTAs of a head
+    attr[1].val.clusterDim.x = static_cast<unsigned>(p.d / 32);
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = EPI == EPI_QKV_ROPE_VARIANT ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, qkv_rope_append_kernel<BT, EPI>, w_map, x_map, p);
 }
 
@@ -330,6 +448,8 @@ cudaError_t qkv_set_attributes(int smem_optin) {
     AC_SET(16, EPI_QKV_ROPE_APPEND)
     AC_SET(8, EPI_RESIDUAL_ADD)
     AC_SET(16, EPI_RESIDUAL_ADD)
+    AC_SET(8, EPI_QKV_ROPE_VARIANT)
+    AC_SET(16, EPI_QKV_ROPE_VARIANT)
 #undef AC_SET
     return cudaSuccess;
 }
@@ -345,7 +465,7 @@ cudaError_t launch_qkv_rope_kv_append(const CUtensorMap& w_map, const CUtensorMa
                                       const int32_t* context_lens, const float* rope_cos,
                                       const float* rope_sin, int max_position, int B, int H, int Hq,
                                       int Hkv, int d, int page_size, int num_pages, int32_t* status_flag,
-                                      cudaStream_t stream) {
+                                      const RopeVariant* variant, cudaStream_t stream) {
     QkvParams p;
     p.q_out = static_cast<uint16_t*>(q_out);
     p.k_cache = static_cast<uint16_t*>(k_cache);
@@ -371,6 +491,19 @@ cudaError_t launch_qkv_rope_kv_append(const CUtensorMap& w_map, const CUtensorMa
     p.residual_out = nullptr;
     p.N = 0;
     const int bt = qkv_batch_tile(B);
+    p.rotary_dim = d;
+    p.interleaved = 0;
+    p.q_norm_w = p.k_norm_w = nullptr;
+    p.norm_eps = 0.0f;
+    if (variant != nullptr) {
+        p.rotary_dim = variant->rotary_dim;
+        p.interleaved = variant->interleaved;
+        p.q_norm_w = static_cast<const uint16_t*>(variant->q_norm_weight);
+        p.k_norm_w = static_cast<const uint16_t*>(variant->k_norm_weight);
+        p.norm_eps = variant->norm_eps;
+        if (bt == 8) return launch_qkv<8, EPI_QKV_ROPE_VARIANT>(w_map, x_map, p, stream);
+        return launch_qkv<16, EPI_QKV_ROPE_VARIANT>(w_map, x_map, p, stream);
+    }
     if (bt == 8) return launch_qkv<8, EPI_QKV_ROPE_APPEND>(w_map, x_map, p, stream);
     return launch_qkv<16, EPI_QKV_ROPE_APPEND>(w_map, x_map, p, stream);
 }

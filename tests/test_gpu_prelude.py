@@ -92,6 +92,124 @@ def test_qkv_prelude_matches_oracle(B, H, Hq, Hkv, d, ps):
     print(f"[prelude] B={B} H={H}: exact fraction of v = {ev:.4f}")
 
 
+@pytest.mark.parametrize("kw", [
+    dict(rotary_dim=64),                                       # partial rotary, half-split: partners in sister CTAs
+    dict(interleaved=True),
+    dict(rotary_dim=32, interleaved=True),
+    dict(norm=True),                                           # per-head Q/K RMSNorm, then full rotary
+    dict(norm=True, rotary_dim=64, interleaved=True),          # Qwen3- and GLM-4-style options together
+    dict(norm="q_only", rotary_dim=64),
+])
+@pytest.mark.parametrize("B,d", [(5, 128), (16, 64), (40, 128)])
+def test_qkv_prelude_variants_bit_exact_when_the_projection_is_exact(kw, B, d):
+    """ac_qkv_rope_kv_append_ex: small-integer x and W make the projection exact, so q and both pools must
+    equal the oracle's chain (projection -> RMSNorm -> partial / interleaved rotation -> append) bit for
+    bit; 40 rows run as three 16-row grid slices."""
+    import torch
+    from paper_2606_07665_b200 import binding as ac
+    from paper_2606_07665_b200 import build, runner
+    build.build()
+    torch.cuda.set_device(0)
+    ac.ac_init(0)
+    kw = dict(kw)
+    norm = kw.pop("norm", False)
+    rotary_dim = min(kw.get("rotary_dim", 0), d)
+    interleaved = kw.get("interleaved", False)
+    H, Hq, Hkv, ps = 320, 6, 2, 16
+    rng = np.random.default_rng(777 + B + d)
+    lens = rng.integers(0, 400, size=B).tolist()
+    w = W.make_workload("prelude_var", 400 + B, B=B, Hq=Hq, Hkv=Hkv, d=d, page_size=ps,
+                        num_pages=B * (400 // ps + 2) + 4, context_lens=lens, rope_base=10000.0,
+                        inactive_rows=(1,))
+    R = rotary_dim or d
+    w.rope_cos, w.rope_sin = W.rope_table(w.max_position, R, w.rope_base)
+    x = W.f32_to_bf16_bits(rng.integers(-2, 3, size=(B, H)).astype(np.float32))
+    wq = W.f32_to_bf16_bits(rng.integers(-2, 3, size=((Hq + 2 * Hkv) * d, H)).astype(np.float32))
+    qw = W.f32_to_bf16_bits((1 + 0.2 * rng.standard_normal(d)).astype(np.float32)) if norm else None
+    kw_bits = W.f32_to_bf16_bits((1 + 0.2 * rng.standard_normal(d)).astype(np.float32)) if norm is True else None
+    q0, k0, v0 = O.oracle_qkv_projection(x, wq, Hq, Hkv, d)
+    q_ref, k_ref, v_ref = O.oracle_rope_kv_append_ex(q0, k0, v0, w.k_cache, w.v_cache, w.block_table,
+                                                     w.context_lens, w.rope_cos, w.rope_sin, ps,
+                                                     rotary_dim=rotary_dim or None, interleaved=interleaved,
+                                                     q_norm_weight=qw, k_norm_weight=kw_bits, norm_eps=1e-6)
+    st = runner.DecodeStep(w, num_splits=1)
+    dev = lambda a: None if a is None else torch.from_numpy(a.view(np.int16)).cuda()
+    st.q_rot.fill_(0x7FC0)
+    ac.ac_qkv_rope_kv_append_ex(dev(x), dev(wq), H, st.q_rot, st.k_cache, st.v_cache, st.stride_page,
+                                st.stride_token, st.stride_head, st.block_table, w.max_pages_per_seq,
+                                st.context_lens, st.rope_cos, st.rope_sin, w.max_position, B, Hq, Hkv, d, ps,
+                                w.num_pages, st.status_flag, rotary_dim=rotary_dim, interleaved=interleaved,
+                                q_norm_weight=dev(qw), k_norm_weight=dev(kw_bits), norm_eps=1e-6)
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) == 0
+    active = w.context_lens >= 0
+    q_gpu = runner.bits_of(st.q_rot)
+    assert np.array_equal(q_gpu[active], q_ref[active]), "q differs"
+    assert (q_gpu[~active] == 0x7FC0).all()
+    k_gpu, v_gpu = st.cache_bits()
+    assert np.array_equal(k_gpu, k_ref), "K pool differs"
+    assert np.array_equal(v_gpu, v_ref), "V pool differs"
+    out_ref = O.oracle_paged_decode_attn(q_ref, k_ref, v_ref, w.block_table, w.context_lens, ps)
+    st.attention()
+    torch.cuda.synchronize()
+    err = np.abs(st.out_f64() - out_ref)
+    scale = max(1.0, float(np.abs(out_ref).max()))         # integer projections make outputs of size ~50
+    assert err.max() <= 2e-2 * scale and err.mean() <= 2e-3 * scale
+
+
+def test_qkv_prelude_variants_on_random_inputs():
+    """N(0,1) inputs, Qwen3-like options (Q/K RMSNorm) on an 8-row batch of a 2048-hidden layer: the
+    fp32 projection may be one bf16 step off now and then, and the norm spreads such a step over the
+    head vector, so q and the appended k are held to the oracle within two bf16 steps of the pair's
+    magnitude; v is not touched by the options."""
+    import torch
+    from paper_2606_07665_b200 import binding as ac
+    from paper_2606_07665_b200 import build, runner
+    build.build()
+    torch.cuda.set_device(0)
+    ac.ac_init(0)
+    B, H, Hq, Hkv, d, ps = 8, 2048, 16, 4, 128, 16
+    rng = np.random.default_rng(991)
+    lens = rng.integers(0, 300, size=B).tolist()
+    w = W.make_workload("prelude_var_n", 500, B=B, Hq=Hq, Hkv=Hkv, d=d, page_size=ps, num_pages=B * 21 + 4,
+                        context_lens=lens, rope_base=1000000.0)
+    x, wq = W.make_projection_inputs(501, B, H, Hq, Hkv, d)
+    qw = W.f32_to_bf16_bits((1 + 0.2 * rng.standard_normal(d)).astype(np.float32))
+    kw_bits = W.f32_to_bf16_bits((1 + 0.2 * rng.standard_normal(d)).astype(np.float32))
+    q0, k0, v0 = O.oracle_qkv_projection(x, wq, Hq, Hkv, d)
+    q_ref, k_ref, v_ref = O.oracle_rope_kv_append_ex(q0, k0, v0, w.k_cache, w.v_cache, w.block_table,
+                                                     w.context_lens, w.rope_cos, w.rope_sin, ps,
+                                                     q_norm_weight=qw, k_norm_weight=kw_bits, norm_eps=1e-6)
+    st = runner.DecodeStep(w, num_splits=1)
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda()
+    ac.ac_qkv_rope_kv_append_ex(dev(x), dev(wq), H, st.q_rot, st.k_cache, st.v_cache, st.stride_page,
+                                st.stride_token, st.stride_head, st.block_table, w.max_pages_per_seq,
+                                st.context_lens, st.rope_cos, st.rope_sin, w.max_position, B, Hq, Hkv, d, ps,
+                                w.num_pages, st.status_flag, q_norm_weight=dev(qw), k_norm_weight=dev(kw_bits),
+                                norm_eps=1e-6)
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) == 0
+    q_gpu = runner.bits_of(st.q_rot)
+    k_gpu, v_gpu = st.cache_bits()
+    target = np.zeros(k_ref.shape[:2], dtype=bool)
+    for b in range(B):
+        L = int(w.context_lens[b])
+        target[w.block_table[b, L // ps], L % ps] = True
+
+    def close(got_bits, ref_bits, what):
+        got = W.bf16_bits_to_f32(got_bits).astype(np.float64)
+        ref = W.bf16_bits_to_f32(ref_bits).astype(np.float64)
+        mag = np.sqrt(ref[..., :d // 2] ** 2 + ref[..., d // 2:] ** 2)
+        mag = np.concatenate([mag, mag], axis=-1)
+        assert (np.abs(got - ref) <= 2.0 ** -5 * mag + 2.0 ** -7).all(), (what, float(np.abs(got - ref).max()))
+        assert float(np.mean(got_bits == ref_bits)) >= 0.9, what
+
+    close(q_gpu, q_ref, "q")
+    close(k_gpu[target], k_ref[target], "k")
+    assert np.array_equal(k_gpu[~target], w.k_cache[~target]) and np.array_equal(v_gpu[~target], w.v_cache[~target])
+    _close_bf16(v_gpu[target], v_ref[target], "v")
+
+
 @pytest.mark.parametrize("B", [8, 100])
 def test_qkv_prelude_bit_exact_when_the_projection_is_exact(B):
     """Small-integer x and W make every dot product an integer that fp32 and fp64 both hold exactly, so
