@@ -464,7 +464,43 @@ def time_prelude_fusion(torch, device, batches=(1, 8, 32, 128, 256), replicas=12
         rows.append({"kernel": "ac_qkv_rope_kv_append", "B": B, "weight_mb": round(wbytes / 1e6, 1),
                      "us_per_call": round(us, 2), "weight_gbs": round(wbytes / us / 1e3, 1),
                      "status_flag": int(st.status_flag.item())})
-        del graph, xs, ws
+        del graph
+        if B <= 16:
+            # the same launch with per-head Q/K RMSNorm folded into its epilogue (cluster of four CTAs per head)
+            nw = torch.from_numpy(W.f32_to_bf16_bits(np.ones(d, dtype=np.float32)).view(np.int16)).to(device)
+
+            def call_ex(i, stream):
+                ac.ac_qkv_rope_kv_append_ex(xs[i], ws[i], H, st.q_rot, st.k_cache, st.v_cache, st.stride_page,
+                                            st.stride_token, st.stride_head, st.block_table, w.max_pages_per_seq,
+                                            st.context_lens, st.rope_cos, st.rope_sin, w.max_position, B, Hq,
+                                            Hkv, d, ps, w.num_pages, st.status_flag, stream,
+                                            q_norm_weight=nw, k_norm_weight=nw, norm_eps=1e-6)
+
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                for i in range(replicas):
+                    call_ex(i, side)
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for i in range(replicas):
+                    call_ex(i, side)
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            t0.record()
+            for _ in range(replays):
+                graph.replay()
+            t1.record()
+            torch.cuda.synchronize()
+            us = t0.elapsed_time(t1) * 1e3 / (replays * replicas)
+            rows.append({"kernel": "ac_qkv_rope_kv_append_ex (Q/K RMSNorm)", "B": B,
+                         "weight_mb": round(wbytes / 1e6, 1), "us_per_call": round(us, 2),
+                         "weight_gbs": round(wbytes / us / 1e3, 1), "status_flag": int(st.status_flag.item())})
+            del graph
+        del xs, ws
 
         # output projection + residual + RMSNorm on the same layer: W_o [4096, 4096] (33.6 MB)
         K, N = Hq * d, H
@@ -612,6 +648,27 @@ def time_rope_variants(torch, device, batch=256, reps=50):
         rows.append({"kernel": "rope_kv_append_ex_kernel", "variant": label, "B": batch,
                      "us_per_call_own_launch": round(statistics.median(times), 2),
                      "status_flag": int(st.status_flag.item())})
+    return rows
+
+
+def time_model_variants(torch, device, peak):
+    """The single-launch step with the prelude variants two of the paper's model families need, in-graph
+    and K/V cold like the other workloads: a Qwen3-like layer (32 query / 8 KV heads, per-head Q/K
+    RMSNorm) and a GLM-4-like one (32 query / 2 KV heads, rotary on 64 of 128 elements, interleaved
+    pairs), batch 32, contexts uniform in [512, 2048]."""
+    from paper_2606_07665_b200 import runner
+    rows = []
+    for name in ("qwen3_like_b32", "glm4_like_b32"):
+        w = W.NAMED[name]()
+        us, info = time_in_graph(lambda: runner.DecodeStep(w, device=device, fused_step=True, rope_variants="workload"),
+                                 w.kv_bytes, torch)
+        rows.append({"workload": name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "kv_mb": round(w.kv_bytes / 1e6, 1),
+                     "variants": sorted(w.extra["rope_variants"]),
+                     "num_splits": info["num_splits"], "us_per_call": round(us, 2),
+                     "kv_gbs": round(w.kv_bytes / us / 1e3, 1),
+                     "frac_of_hbm_peak": round(w.kv_bytes / us / 1e3 / peak, 4),
+                     "entry_point": "ac_decode_step_fused_ex + ac_attn_options.rope",
+                     "status_flag": info["status_flag"]})
     return rows
 
 
@@ -771,6 +828,7 @@ def run_ours(args):
             kernels_alone = time_kernels_alone(w, device, runner, torch)
             read_stream = time_read_stream(torch, device)
             rope_variants = time_rope_variants(torch, device)
+            model_variants = time_model_variants(torch, device, peak)
             prelude = time_prelude_fusion(torch, device)
             for r in prelude:
                 r["frac_of_hbm_peak"] = round(r["weight_gbs"] / peak, 4)
@@ -789,6 +847,7 @@ def run_ours(args):
             kernels_alone = None
             read_stream = None
             rope_variants = []
+            model_variants = []
         sm_mhz = clocks.get("sm_mhz") if clocks else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -820,7 +879,7 @@ def run_ours(args):
             "gpu_launches": args.steps * launches_per_step * timed_blocks,
             "clocks": clocks, "status_flag": flag, "workloads": others,
             "kernels_alone": kernels_alone, "prelude_fusion": prelude, "attention_block": block,
-            "rope_variants": rope_variants,
+            "rope_variants": rope_variants, "model_variants": model_variants,
         }
         print(json.dumps(line))
     if world > 1:

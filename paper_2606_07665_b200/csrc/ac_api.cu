@@ -212,6 +212,11 @@ static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_con
     const double hbm = 6.5e12 * sm_count / 148.0;      // bytes/s the whole GPU streams
     const double cta_rate = 33e9;                       // bytes/s one CTA streams on its own
     const double wave_cost = 3e-6;
+    // A grid that could have fitted the GPU at once but spills into a further wave pays much more than
+    // a ramp for it: the CTAs of that wave start only when first-wave CTAs retire and then need their
+    // whole own duration (measured on batches of 32 requests: 295 CTAs 19 us, 350 CTAs 30 us; 256 CTAs
+    // 34 us, 415 CTAs 43 us).
+    const double spill_wave_cost = 8e-6;
     long long active_rows = B;
     double total_tokens = static_cast<double>(B) * max_context_len;
     if (token_counts != nullptr) {
@@ -269,11 +274,11 @@ static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_con
                 const double last = n - (waves - 1.0) * slots;
                 t = (waves - 1.0) * slots * c / hbm;
                 const double t_last_bw = last * c / hbm, t_last_cta = c / cta_rate;
-                t += (t_last_bw > t_last_cta ? t_last_bw : t_last_cta) + waves * wave_cost;
+                t += (t_last_bw > t_last_cta ? t_last_bw : t_last_cta) + wave_cost + (waves - 1.0) * spill_wave_cost;
             } else {
                 const double t_bw = total_tokens * Hkv * bytes_per_token / hbm;
                 const double t_cta = longest * bytes_per_token / cta_rate;
-                t = (t_bw > t_cta ? t_bw : t_cta) + waves * wave_cost;
+                t = (t_bw > t_cta ? t_bw : t_cta) + wave_cost + (waves - 1.0) * spill_wave_cost;
             }
             if (cand > 1)            // partials out and back in plus the ticket round trip, or two cluster barriers
                 t += in_cluster ? 0.3e-6 : 2.0 * active_rows * Hq * cand * (d + 1.0) * 4.0 / hbm + 1.6e-6;

@@ -30,8 +30,17 @@ class DecodeStep:
 
     def __init__(self, w, device="cuda:0", num_splits: int | None = None, layout: str = "token_major",
                  max_context_len: int | None = None, fused_merge: bool = True,
-                 fused_step: bool = False, window: int = 0, row_order="auto"):
+                 fused_step: bool = False, window: int = 0, row_order="auto", rope_variants=None):
         self.w = w
+        # prelude variants the single-launch step applies (rotary_dim, interleaved, q_norm_weight,
+        # k_norm_weight, norm_eps); None = the plain rotation
+        if isinstance(rope_variants, str) and rope_variants == "workload":
+            # the options the workload itself names, norm weights moved to the device
+            self.rope_variants = {
+                k: (torch.from_numpy(np.ascontiguousarray(v).view(np.int16)).to(device) if isinstance(v, np.ndarray) else v)
+                for k, v in w.extra.get("rope_variants", {}).items()}
+        else:
+            self.rope_variants = dict(rope_variants) if rope_variants else {}
         self.window = int(window) if window else int(getattr(w, "window", 0))   # > 0: sliding window
         self.fused_step = bool(fused_step)             # one launch: RoPE + append + attention + merge
         self.fused_merge = bool(fused_merge) or self.fused_step
@@ -148,7 +157,7 @@ class DecodeStep:
                                    self.workspace if self.num_splits > 1 else None, self.workspace_bytes,
                                    self.out, self.B, self.Hq, self.Hkv, self.d, self.ps, self.num_pages,
                                    self.max_context_len, self.status_flag, stream, window=self.window,
-                                   row_order=self.row_order, **rope_variants)
+                                   row_order=self.row_order, **{**self.rope_variants, **rope_variants})
 
     def step(self, stream=None) -> None:
         if self.fused_step:

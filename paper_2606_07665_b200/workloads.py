@@ -266,6 +266,30 @@ def sliding_window_4k() -> DecodeWorkload:
     return w
 
 
+def qwen3_like_b32() -> DecodeWorkload:
+    """A layer shaped like the paper's Qwen3 family: 32 query / 8 KV heads, head_dim 128, per-head Q/K
+    RMSNorm before the rotation; batch 32, lengths uniform in [512, 2048].  ``extra['rope_variants']``
+    names the prelude options (norm weights 1 + 0.1 N(0,1), seeded)."""
+    w = make_workload("qwen3_like_b32", 76, B=32, Hq=32, Hkv=8, d=128, page_size=16, num_pages=32 * 132 + 8,
+                      len_range=(512, 2048), rope_base=1000000.0)
+    g = np.random.default_rng([76, 20])
+    w.extra["rope_variants"] = dict(
+        q_norm_weight=f32_to_bf16_bits((1 + 0.1 * g.standard_normal(128)).astype(np.float32)),
+        k_norm_weight=f32_to_bf16_bits((1 + 0.1 * g.standard_normal(128)).astype(np.float32)), norm_eps=1e-6)
+    return w
+
+
+def glm4_like_b32() -> DecodeWorkload:
+    """A layer shaped like the paper's GLM-4 family: 32 query / 2 KV heads (the 32:2 ratio), head_dim
+    128, rotary embedding on the first 64 elements only, interleaved pairs; batch 32, lengths uniform
+    in [512, 2048].  The rope tables are [max_position, 32]."""
+    w = make_workload("glm4_like_b32", 77, B=32, Hq=32, Hkv=2, d=128, page_size=16, num_pages=32 * 132 + 8,
+                      len_range=(512, 2048), rope_base=1000000.0)
+    w.rope_cos, w.rope_sin = rope_table(w.max_position, 64, w.rope_base)
+    w.extra["rope_variants"] = dict(rotary_dim=64, interleaved=True)
+    return w
+
+
 NAMED = {
     "tiny": tiny,
     "single_request": single_request,
@@ -274,4 +298,6 @@ NAMED = {
     **{f"graph_sweep_b{b}": (lambda b=b: graph_sweep(b)) for b in GRAPH_SWEEP_BATCHES},
     "gqa_group16": gqa_group16,
     "sliding_window_4k": sliding_window_4k,
+    "qwen3_like_b32": qwen3_like_b32,
+    "glm4_like_b32": glm4_like_b32,
 }

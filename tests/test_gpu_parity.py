@@ -771,6 +771,29 @@ def test_workload_sliding_window_4k(rt, fused):
     run_and_compare(rt, w, fused=fused, window=w.window)
 
 
+@pytest.mark.parametrize("name", ["qwen3_like_b32", "glm4_like_b32"])
+def test_workload_model_variants(rt, name):
+    # the two model-shaped workloads of the benchmark: the single-launch step with the options the
+    # workload names (Q/K RMSNorm; 32:2 GQA with partial, interleaved rotary) against the oracle's chain
+    import torch
+    w = W.NAMED[name]()
+    opts = w.extra["rope_variants"]
+    q_rot, k_after, v_after = O.oracle_rope_kv_append_ex(
+        w.q, w.k_new, w.v_new, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.rope_cos, w.rope_sin,
+        w.page_size, rotary_dim=opts.get("rotary_dim"), interleaved=opts.get("interleaved", False),
+        q_norm_weight=opts.get("q_norm_weight"), k_norm_weight=opts.get("k_norm_weight"),
+        norm_eps=opts.get("norm_eps", 0.0))
+    out_ref = O.oracle_paged_decode_attn(q_rot, k_after, v_after, w.block_table, w.context_lens, w.page_size)
+    st = rt.DecodeStep(w, fused_step=True, rope_variants="workload")
+    st.step()
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) == 0
+    assert np.array_equal(rt.bits_of(st.q_rot), q_rot), "q after norm/rotation differs"
+    k_gpu, v_gpu = st.cache_bits()
+    assert np.array_equal(k_gpu, k_after) and np.array_equal(v_gpu, v_after)
+    check_out(st.out_f64(), out_ref, name)
+
+
 _LONG_CONTEXT_ORACLE = {}
 
 
