@@ -465,8 +465,8 @@ def time_prelude_fusion(torch, device, batches=(1, 8, 32, 128, 256), replicas=12
                      "us_per_call": round(us, 2), "weight_gbs": round(wbytes / us / 1e3, 1),
                      "status_flag": int(st.status_flag.item())})
         del graph
-        if B <= 16:
-            # the same launch with per-head Q/K RMSNorm folded into its epilogue (cluster of four CTAs per head)
+        if B <= 128:
+            # the same launch with per-head Q/K RMSNorm folded into its epilogue (the CTAs of a head as a cluster)
             nw = torch.from_numpy(W.f32_to_bf16_bits(np.ones(d, dtype=np.float32)).view(np.int16)).to(device)
 
             def call_ex(i, stream):

@@ -200,12 +200,11 @@ int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out,
 /* ac_qkv_rope_kv_append with the prelude variants of ac_rope_kv_append_ex (family (i) names the per-head
  * Q/K RMSNorm as an option of the fused prelude; the per-model adaptations mention partial rotary):
  * the projected, bf16-rounded q and k head vectors are normalised, rotated over their first
- * rotary_dim elements with the chosen pairing and stored, still in one launch.  The d/32 CTAs that
- * share a head form a thread-block cluster and exchange the sums of squares and the rotation partners
- * through distributed shared memory.  options == NULL (or all defaults) is ac_qkv_rope_kv_append.  With
- * options the call runs on the warp-MMA kernel at every batch size, 16 rows per grid slice (the
- * weights are then streamed once per 16 rows; the tcgen05 kernel has no variant epilogue).  The rope
- * tables are [max_position, rotary_dim/2].  Everything else as ac_qkv_rope_kv_append. */
+ * rotary_dim elements with the chosen pairing and stored, still in one launch.  The CTAs that share a
+ * head (d/32 of the warp-MMA kernel, two or three overlapping tiles of the tcgen05 kernel) form a
+ * thread-block cluster and exchange the sums of squares and the rotation partners through distributed
+ * shared memory.  options == NULL (or all defaults) is ac_qkv_rope_kv_append.  The rope tables are
+ * [max_position, rotary_dim/2].  Everything else as ac_qkv_rope_kv_append. */
 int ac_qkv_rope_kv_append_ex(const void* x, const void* w_qkv, int H, void* q_out,
                              void* k_cache, void* v_cache,
                              int64_t stride_page, int64_t stride_token, int64_t stride_head,

@@ -431,8 +431,7 @@ int ac_qkv_rope_kv_append_ex(const void* x, const void* w_qkv, int H, void* q_ou
     // x [B, H] as (64 elements, batch row, 64-element K block).
     const cuuint64_t row_bytes = static_cast<cuuint64_t>(H) * 2;
     CUtensorMap w_map, x_map;
-    // The prelude variants run on the warp-MMA kernel at every batch size (16 rows per grid slice).
-    if (B > kWarpMmaMaxBatch && vp == nullptr) {
+    if (B > kWarpMmaMaxBatch) {
         // Batched decode: batch tiles of up to 128 rows on the tcgen05 path (boxes of 24 pairs x 2 K blocks).
         cuuint64_t wdims[5] = {64, static_cast<cuuint64_t>(d / 2), 2, static_cast<cuuint64_t>(Hq + 2 * Hkv),
                                static_cast<cuuint64_t>(H / 64)};
@@ -456,7 +455,7 @@ int ac_qkv_rope_kv_append_ex(const void* x, const void* w_qkv, int H, void* q_ou
                                                      stride_token, stride_head, block_table,
                                                      max_pages_per_seq, context_lens, rope_cos, rope_sin,
                                                      max_position, B, H, Hq, Hkv, d, page_size, num_pages,
-                                                     status_flag, static_cast<cudaStream_t>(stream));
+                                                     status_flag, vp, static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? AC_OK : fail_cuda(static_cast<int>(e));
     }
     {

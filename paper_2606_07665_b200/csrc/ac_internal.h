@@ -105,7 +105,7 @@ cudaError_t launch_qkv_rope_kv_append_tc(const CUtensorMap& w_map, const CUtenso
                                          const int32_t* context_lens, const float* rope_cos,
                                          const float* rope_sin, int max_position, int B, int K, int Hq,
                                          int Hkv, int d, int page_size, int num_pages,
-                                         int32_t* status_flag, cudaStream_t stream);
+                                         int32_t* status_flag, const RopeVariant* variant, cudaStream_t stream);
 cudaError_t launch_oproj_residual_tc(const CUtensorMap& w_map, const CUtensorMap& x_map,
                                      const void* residual_in, void* residual_out, int B, int K, int N,
                                      cudaStream_t stream);

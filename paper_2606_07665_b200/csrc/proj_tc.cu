@@ -37,7 +37,7 @@ namespace {
 
 using namespace acdev;
 
-enum { TC_EPI_QKV_ROPE_APPEND = 0, TC_EPI_RESIDUAL_ADD = 1 };
+enum { TC_EPI_QKV_ROPE_APPEND = 0, TC_EPI_RESIDUAL_ADD = 1, TC_EPI_QKV_ROPE_VARIANT = 2 };
 
 constexpr int TC_M = 128;                       // rows of the MMA tile: batch rows per CTA, at most
 constexpr int TC_MAX_STAGES = 12;
@@ -47,12 +47,12 @@ constexpr int TC_SMEM_TOTAL = TC_BAR_OFFSET + (2 * TC_MAX_STAGES + 1) * 8 + 16 +
 
 template <int EPI>
 struct TcTile {
-    static constexpr int N = EPI == TC_EPI_QKV_ROPE_APPEND ? 48 : 32;        // features per CTA
-    static constexpr int GROUPS = EPI == TC_EPI_QKV_ROPE_APPEND ? 3 : 2;     // epilogue warps per 32 rows
+    static constexpr int N = EPI == TC_EPI_RESIDUAL_ADD ? 32 : 48;           // features per CTA
+    static constexpr int GROUPS = EPI == TC_EPI_RESIDUAL_ADD ? 2 : 3;        // epilogue warps per 32 rows
     static constexpr int THREADS = 64 + 128 * GROUPS + 32;       // the last warp holds the second MMA issuer
     static constexpr int MMA2_WARP = 2 + 4 * GROUPS;
     static constexpr int B_BLOCK = N * 128;          // one swizzled [N rows x 128 B] block of W
-    static constexpr uint32_t ACC_COLS = EPI == TC_EPI_QKV_ROPE_APPEND ? 64 : 32;    // a power of two >= N
+    static constexpr uint32_t ACC_COLS = EPI == TC_EPI_RESIDUAL_ADD ? 32 : 64;       // a power of two >= N
     static constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;                              // two accumulators
 };
 
@@ -78,7 +78,23 @@ struct TcParams {
     const uint16_t* residual_in;
     uint16_t* residual_out;
     int N;
+    // prelude variants only (TC_EPI_QKV_ROPE_VARIANT)
+    int rotary_dim, interleaved;
+    const uint16_t* q_norm_w;
+    const uint16_t* k_norm_w;
+    float norm_eps;
 };
+
+// Pairs of a head that QKV tile `blk` OWNS (tiles overlap; every pair has one owner): with 64 pairs
+// per head tile 0 owns [0, 16), tile 1 [16, 40), tile 2 [40, 64); with 32 pairs tile 0 owns [0, 8) and
+// tile 1 [8, 32).
+__host__ __device__ inline int qkv_tile_own_begin(int half_d, int blk) { return qkv_tile_first_pair(half_d, blk); }
+__host__ __device__ inline int qkv_tile_own_end(int half_d, int blk) {
+    return half_d == 64 ? (blk == 0 ? 16 : blk == 1 ? 40 : 64) : (blk == 0 ? 8 : 32);
+}
+__host__ __device__ inline int qkv_tile_owner(int half_d, int pair) {
+    return half_d == 64 ? (pair < 16 ? 0 : pair < 40 ? 1 : 2) : (pair < 8 ? 0 : 1);
+}
 
 // ---- tcgen05 wrappers ---------------------------------------------------------------------------
 
@@ -166,7 +182,7 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
 
     const int blk = blockIdx.x;          // pair tile inside the head (QKV) / unused (o_proj)
     const int hh = blockIdx.y;           // head slot (QKV) / block of 32 output features (o_proj)
-    const int pair0 = EPI == TC_EPI_QKV_ROPE_APPEND ? qkv_tile_first_pair(p.d / 2, blk) : 0;
+    const int pair0 = EPI == TC_EPI_RESIDUAL_ADD ? 0 : qkv_tile_first_pair(p.d / 2, blk);
     // The x box holds x_rows rows per 64-element block; the MMA always reads 128.  Rows past x_rows are
     // whatever the ring holds: every accumulator row depends on its own x row only, and the epilogue
     // skips them.  A stage is the x tile followed by the W tile.
@@ -308,6 +324,31 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
                     *reinterpret_cast<uint4*>(dst + v * 8) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
                 }
             }
+        } else if (EPI == TC_EPI_QKV_ROPE_VARIANT) {
+            // prelude variants: this warp only rounds its 8 pairs and parks them in shared memory (the
+            // ring is free once the accumulators are complete); the norm and the rotation follow below,
+            // by all threads of the CTA, because they reach across columns and across sister CTAs.
+            uint16_t* vals = reinterpret_cast<uint16_t*>(smem_gen);          // [128 rows][48]
+            const bool ready = mbar_wait_bounded(done_bar, 0);
+            if (!ready && lane == 0 && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_WAIT_TIMEOUT);
+            tc_fence_after_sync();
+            uint32_t lo[8], hi[8], lo_odd[8], hi_odd[8];
+            tmem_ld_32x8(lane_base + 8 * group, lo);
+            tmem_ld_32x8(lane_base + T::N / 2 + 8 * group, hi);
+            tmem_ld_32x8(lane_base + T::ACC_COLS + 8 * group, lo_odd);
+            tmem_ld_32x8(lane_base + T::ACC_COLS + T::N / 2 + 8 * group, hi_odd);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                float a = __uint_as_float(lo[e]), bq = __uint_as_float(hi[e]);
+                if (n_chunks > 1) {
+                    a += __uint_as_float(lo_odd[e]);
+                    bq += __uint_as_float(hi_odd[e]);
+                }
+                const uint32_t pk = (ready && ok) ? pack_bf16x2(a, bq) : 0u;
+                vals[row * T::N + 8 * group + e] = static_cast<uint16_t>(pk & 0xFFFFu);
+                vals[row * T::N + T::N / 2 + 8 * group + e] = static_cast<uint16_t>(pk >> 16);
+            }
         } else {
             // 8 rotary pairs: first halves in columns 8 group .., second halves in columns 24 + 8 group ..
             const int d = p.d, half_d = d / 2;
@@ -420,6 +461,114 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
             }
         }
     }
+    if (EPI == TC_EPI_QKV_ROPE_VARIANT) {
+        // ---- prelude variants: norm and rotation across the tiles of a head ----------------------------
+        // The two or three tiles of a head slot (blockIdx.x) are one thread-block cluster.  Tiles overlap,
+        // so every pair has one OWNER tile: sums of squares count owned pairs only, and a rotation
+        // partner is fetched from its owner.  Three cluster barriers, executed by every thread of every
+        // CTA on every path: parked features and partial sums visible; normalised features visible;
+        // nobody's shared memory released while a sister still reads it.
+        const int d = p.d, half_d = d / 2;
+        uint16_t* vals = reinterpret_cast<uint16_t*>(smem_gen);                        // [128][48] rounded
+        uint16_t* valsn = vals + TC_M * T::N;                                           // [128][48] after the norm
+        double* sums = reinterpret_cast<double*>(valsn + TC_M * T::N);                  // [128]
+        int* row_ctx = reinterpret_cast<int*>(sums + TC_M);                             // [128]; -1: row not stored
+        unsigned long long* row_dst = reinterpret_cast<unsigned long long*>(row_ctx + TC_M);   // [128] destination rows
+        const bool is_q = hh < p.Hq, is_k = !is_q && hh < p.Hq + p.Hkv;
+        const uint16_t* norm_w = is_q ? p.q_norm_w : (is_k ? p.k_norm_w : nullptr);
+        const int n_tiles = gridDim.x;
+        __syncthreads();                                      // the epilogue warps have parked the features
+        if (threadIdx.x < TC_M) {
+            const int row = threadIdx.x;
+            const int b = b0 + row;
+            double ss = 0.0;
+            for (int i = qkv_tile_own_begin(half_d, blk); i < qkv_tile_own_end(half_d, blk); ++i) {
+                const double a = static_cast<double>(bf16_bits_to_float(vals[row * T::N + (i - pair0)]));
+                const double bq = static_cast<double>(bf16_bits_to_float(vals[row * T::N + T::N / 2 + (i - pair0)]));
+                ss = __dadd_rn(ss, __dadd_rn(__dmul_rn(a, a), __dmul_rn(bq, bq)));
+            }
+            sums[row] = ss;
+            // where the row goes (as in the plain epilogue)
+            int ctx = -1;
+            unsigned long long dst = 0;
+            if (row < p.x_rows && b < p.B) {
+                ctx = p.context_lens[b];
+                if (ctx >= 0) {
+                    const int page_idx = ctx / p.page_size;
+                    if (ctx >= p.max_position || page_idx >= p.max_pages_per_seq) {
+                        if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
+                        ctx = -1;
+                    } else if (is_q) {
+                        dst = reinterpret_cast<unsigned long long>(p.q_out + (static_cast<size_t>(b) * p.Hq + hh) * d);
+                    } else {
+                        const int page = p.block_table[static_cast<size_t>(b) * p.max_pages_per_seq + page_idx];
+                        if (page < 0 || page >= p.num_pages) {
+                            if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
+                            ctx = -1;
+                        } else {
+                            const int h = is_k ? hh - p.Hq : hh - p.Hq - p.Hkv;
+                            dst = reinterpret_cast<unsigned long long>(
+                                (is_k ? p.k_cache : p.v_cache) + static_cast<size_t>(page) * p.stride_page +
+                                static_cast<size_t>(ctx - page_idx * p.page_size) * p.stride_token +
+                                static_cast<size_t>(h) * p.stride_head);
+                        }
+                    }
+                }
+            }
+            row_ctx[row] = ctx;
+            row_dst[row] = dst;
+        }
+        cluster_sync_all();
+        for (int item = threadIdx.x; item < TC_M * T::N; item += T::THREADS) {
+            const int row = item / T::N, col = item - row * T::N;
+            uint16_t v16 = vals[item];
+            if (norm_w != nullptr) {
+                double total = 0.0;
+                for (int c = 0; c < n_tiles; ++c)
+                    total = __dadd_rn(total, cluster_load_f64(cluster_map_shared(smem_addr(sums + row), c)));
+                const double rr = __ddiv_rn(1.0, __dsqrt_rn(__dadd_rn(__ddiv_rn(total, static_cast<double>(d)),
+                                                                      static_cast<double>(p.norm_eps))));
+                const int f = (col >= T::N / 2 ? half_d : 0) + pair0 + (col % (T::N / 2));     // feature inside the head
+                const uint16_t y1 = f64_to_bf16_rne(__dmul_rn(static_cast<double>(bf16_bits_to_float(v16)), rr));
+                v16 = f64_to_bf16_rne(__dmul_rn(static_cast<double>(bf16_bits_to_float(y1)),
+                                                static_cast<double>(bf16_bits_to_float(norm_w[f]))));
+            }
+            valsn[item] = v16;
+        }
+        cluster_sync_all();
+        const int R = p.rotary_dim, half_r = R / 2;
+        for (int item = threadIdx.x; item < TC_M * T::N; item += T::THREADS) {
+            const int row = item / T::N, col = item - row * T::N;
+            const int ctx = row_ctx[row];
+            if (ctx < 0) continue;
+            const int pair = pair0 + (col % (T::N / 2));
+            const int f = (col >= T::N / 2 ? half_d : 0) + pair;
+            uint16_t v16 = valsn[item];
+            if ((is_q || is_k) && f < R) {
+                int i, partner;
+                bool first;
+                if (p.interleaved) {
+                    i = f >> 1;
+                    first = (f & 1) == 0;
+                    partner = first ? f + 1 : f - 1;
+                } else {
+                    first = f < half_r;
+                    i = first ? f : f - half_r;
+                    partner = first ? f + half_r : f - half_r;
+                }
+                const int ppair = partner % half_d;
+                const int owner = qkv_tile_owner(half_d, ppair);
+                const int pcol = (partner >= half_d ? T::N / 2 : 0) + (ppair - qkv_tile_first_pair(half_d, owner));
+                const uint16_t other = cluster_load_u16(cluster_map_shared(smem_addr(valsn + row * T::N + pcol), owner));
+                const float c = p.rope_cos[static_cast<size_t>(ctx) * half_r + i];
+                const float sn = p.rope_sin[static_cast<size_t>(ctx) * half_r + i];
+                v16 = first ? rope_first_half(v16, other, c, sn) : rope_second_half(other, v16, c, sn);
+            }
+            reinterpret_cast<uint16_t*>(row_dst[row])[f] = v16;
+        }
+        cluster_sync_all();
+    }
+
     // ---- release TMEM (every path reaches this point) ----------------------------------------------
     tc_fence_before_sync();
     __syncthreads();
@@ -437,11 +586,15 @@ cudaError_t launch_tc_k(const CUtensorMap& w_map, const CUtensorMap& x_map, cons
     cfg.blockDim = dim3(TcTile<EPI>::THREADS);
     cfg.dynamicSmemBytes = TC_SMEM_TOTAL;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;     // prelude variants: the tiles of a head slot
+    attr[1].val.clusterDim.x = grid.x;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = EPI == TC_EPI_QKV_ROPE_VARIANT ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, proj_tc_kernel<EPI, KBLK>, w_map, x_map, p);
 }
 
@@ -480,6 +633,12 @@ cudaError_t proj_tc_set_attributes(int smem_optin) {
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(proj_tc_kernel<TC_EPI_RESIDUAL_ADD, 4>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(proj_tc_kernel<TC_EPI_QKV_ROPE_VARIANT, 2>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(proj_tc_kernel<TC_EPI_QKV_ROPE_VARIANT, 4>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_TOTAL);
     return e;
 }
 
@@ -490,7 +649,7 @@ cudaError_t launch_qkv_rope_kv_append_tc(const CUtensorMap& w_map, const CUtenso
                                          const int32_t* context_lens, const float* rope_cos,
                                          const float* rope_sin, int max_position, int B, int K, int Hq,
                                          int Hkv, int d, int page_size, int num_pages,
-                                         int32_t* status_flag, cudaStream_t stream) {
+                                         int32_t* status_flag, const RopeVariant* variant, cudaStream_t stream) {
     TcParams p = {};
     p.q_out = static_cast<uint16_t*>(q_out);
     p.k_cache = static_cast<uint16_t*>(k_cache);
@@ -513,9 +672,16 @@ cudaError_t launch_qkv_rope_kv_append_tc(const CUtensorMap& w_map, const CUtenso
     p.Hkv = Hkv;
     p.d = d;
     p.x_rows = proj_tc_batch_rows(B);
-    return launch_tc<TC_EPI_QKV_ROPE_APPEND>(w_map, x_map, p, proj_tc_k_blocks(B),
-                                             dim3(d == 128 ? 3 : 2, Hq + 2 * Hkv, (B + p.x_rows - 1) / p.x_rows),
-                                             stream);
+    const dim3 grid(d == 128 ? 3 : 2, Hq + 2 * Hkv, (B + p.x_rows - 1) / p.x_rows);
+    if (variant != nullptr) {
+        p.rotary_dim = variant->rotary_dim;
+        p.interleaved = variant->interleaved;
+        p.q_norm_w = static_cast<const uint16_t*>(variant->q_norm_weight);
+        p.k_norm_w = static_cast<const uint16_t*>(variant->k_norm_weight);
+        p.norm_eps = variant->norm_eps;
+        return launch_tc<TC_EPI_QKV_ROPE_VARIANT>(w_map, x_map, p, proj_tc_k_blocks(B), grid, stream);
+    }
+    return launch_tc<TC_EPI_QKV_ROPE_APPEND>(w_map, x_map, p, proj_tc_k_blocks(B), grid, stream);
 }
 
 cudaError_t launch_oproj_residual_tc(const CUtensorMap& w_map, const CUtensorMap& x_map,

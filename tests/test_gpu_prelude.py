@@ -100,11 +100,12 @@ def test_qkv_prelude_matches_oracle(B, H, Hq, Hkv, d, ps):
     dict(norm=True, rotary_dim=64, interleaved=True),          # Qwen3- and GLM-4-style options together
     dict(norm="q_only", rotary_dim=64),
 ])
-@pytest.mark.parametrize("B,d", [(5, 128), (16, 64), (40, 128)])
+@pytest.mark.parametrize("B,d", [(5, 128), (16, 64), (40, 128), (100, 64), (200, 128)])
 def test_qkv_prelude_variants_bit_exact_when_the_projection_is_exact(kw, B, d):
     """ac_qkv_rope_kv_append_ex: small-integer x and W make the projection exact, so q and both pools must
     equal the oracle's chain (projection -> RMSNorm -> partial / interleaved rotation -> append) bit for
-    bit; 40 rows run as three 16-row grid slices."""
+    bit, on the warp-MMA kernel (up to 16 rows) and on the tcgen05 kernel (one ragged tile of 40 or 104
+    rows, two tiles of 104)."""
     import torch
     from paper_2606_07665_b200 import binding as ac
     from paper_2606_07665_b200 import build, runner
