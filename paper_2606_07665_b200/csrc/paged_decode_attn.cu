@@ -8,9 +8,11 @@
 // issuing thread on the order of 100 ns, so the number of loads per tile matters: splitting head_dim
 // into the innermost 64 elements and an outer block index keeps the swizzle span at 128 bytes while
 // still fetching the whole 256-byte rows with one instruction.)  Every warp runs its own ring of
-// STAGES tiles with one mbarrier per stage and takes tiles warp, warp+WARPS, ... of the CTA's token
-// range; there is no CTA-wide synchronisation in the main loop.  The physical page id of a tile is fetched from the block table one tile ahead of the
-// TMA issue that needs it.  KV bytes are read once, so the loads carry an evict-first L2 policy.
+// STAGES tiles (two; four when the grid is at most one CTA per SM and the splits are long) with one
+// mbarrier per stage and takes tiles warp, warp+WARPS, ... of the CTA's token range; there is no
+// CTA-wide synchronisation in the main loop.  The physical page id of a tile is fetched from the block
+// table one tile ahead of the TMA issue that needs it.  KV bytes are read once, so the loads carry an
+// evict-first L2 policy.
 //
 // Arithmetic.  The Hq/Hkv query heads of the group are the rows of a 16-row MMA tile (rows >= group
 // size are zero).  S = Q K^T and O += P V use the bf16 m16n8k16 warp MMA with fp32 accumulators; the
@@ -23,6 +25,10 @@
 // that arrives last (ticket on a global counter, partials through global memory), or, for grids of
 // at most one CTA per SM, by the CTA of split 0 of a thread-block cluster that reads the other splits'
 // results out of their shared memory.
+//
+// In the fused step (ROPE_PLAIN, ROPE_VARIANT) the kernel also rotates the new q and k -- with the plain
+// rotate-half pairing, or with the prelude variants: per-head RMSNorm, partial rotary, interleaved
+// pairing -- and appends k and v to the cache page before attending over them.
 //
 // With a group of 4-8 query rows the path needs G flop per KV byte; at HBM speed that exceeds what
 // the fp32 pipes deliver for G >= 7, which is why the products run on the tensor pipe even though
@@ -60,7 +66,7 @@ struct Smem {
 };
 
 struct AttnParams {
-    // -- only for the fused step (ROPE = true): the kernel rotates q/k and appends k/v itself
+    // -- only for the fused step (ROPE != ROPE_NONE): the kernel rotates q/k and appends k/v itself
     uint16_t* q_rot_out;          // [B, Hq, D] rotated q, optional (must not alias q)
     const uint16_t* k_new;        // [B, Hkv, D] un-rotated
     const uint16_t* v_new;        // [B, Hkv, D]
@@ -71,7 +77,7 @@ struct AttnParams {
     const float* rope_sin;
     int max_position, num_pages;
     // -- always
-    const uint16_t* q;            // [B, Hq, D] bf16: already rotated (ROPE = false) or raw (ROPE = true)
+    const uint16_t* q;            // [B, Hq, D] bf16: already rotated (ROPE_NONE) or raw (fused step)
     const int32_t* block_table;   // [B, max_pages_per_seq]
     const int32_t* context_lens;  // [B]
     float* partial_o;             // [B, Hq, S, D]   (S > 1)
