@@ -164,6 +164,30 @@ def test_rope_prelude_variants_bit_exact_and_feed_attention(rt, kw, d, path):
     check_out(st.out_f64(), out_ref, f"prelude variant {kw} norm={norm} d={d}")
 
 
+@pytest.mark.parametrize("window,splits", [(100, 1), (333, 3)])
+def test_fused_step_variants_with_a_sliding_window(rt, window, splits):
+    # the prelude variants and the sliding window together in the single-launch step
+    import torch
+    w = small(58, B=3, Hq=12, Hkv=3, d=128, context_lens=[700, 45, 333], num_pages=96)
+    w.rope_cos, w.rope_sin = W.rope_table(w.max_position, 64, w.rope_base)
+    rng = np.random.default_rng(4)
+    qw = W.f32_to_bf16_bits((1 + 0.2 * rng.standard_normal(w.d)).astype(np.float32))
+    q_rot, k_after, v_after = O.oracle_rope_kv_append_ex(
+        w.q, w.k_new, w.v_new, w.k_cache, w.v_cache, w.block_table, w.context_lens, w.rope_cos, w.rope_sin,
+        w.page_size, rotary_dim=64, interleaved=True, q_norm_weight=qw, k_norm_weight=qw, norm_eps=1e-6)
+    out_ref = O.oracle_paged_decode_attn(q_rot, k_after, v_after, w.block_table, w.context_lens, w.page_size,
+                                         window=window)
+    st = rt.DecodeStep(w, num_splits=splits, fused_step=True, window=window)
+    nw = torch.from_numpy(qw.view(np.int16)).cuda()
+    st.decode_step_fused(rotary_dim=64, interleaved=True, q_norm_weight=nw, k_norm_weight=nw, norm_eps=1e-6)
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) == 0
+    assert np.array_equal(rt.bits_of(st.q_rot), q_rot)
+    k_gpu, v_gpu = st.cache_bits()
+    assert np.array_equal(k_gpu, k_after) and np.array_equal(v_gpu, v_after)
+    check_out(st.out_f64(), out_ref, f"variants + window {window}")
+
+
 def test_append_flags_out_of_range_and_writes_nothing(rt):
     import torch
     w = small(34, B=2, context_lens=[40, 50], num_pages=32)

@@ -211,6 +211,59 @@ def test_qkv_prelude_variants_on_random_inputs():
     _close_bf16(v_gpu[target], v_ref[target], "v")
 
 
+@pytest.mark.parametrize("variant", [False, True])
+@pytest.mark.parametrize("B", [6, 40])
+def test_qkv_prelude_flags_rows_it_cannot_store(B, variant):
+    """A row whose page id lies outside the pool, and one whose position lies outside the rope table: the
+    projection launch sets both status bits, writes neither q nor the cache for them, and serves the
+    other rows exactly -- plain and with the prelude variants, on the warp-MMA kernel (6 rows) and on
+    the tcgen05 kernel (40 rows)."""
+    import torch
+    from paper_2606_07665_b200 import binding as ac
+    from paper_2606_07665_b200 import build, runner
+    build.build()
+    torch.cuda.set_device(0)
+    ac.ac_init(0)
+    H, Hq, Hkv, d, ps = 256, 4, 2, 128, 16
+    rng = np.random.default_rng(31 + B)
+    lens = rng.integers(20, 300, size=B).tolist()
+    w = W.make_workload("prelude_flags", 600 + B, B=B, Hq=Hq, Hkv=Hkv, d=d, page_size=ps,
+                        num_pages=B * 21 + 4, context_lens=lens, rope_base=10000.0)
+    x = W.f32_to_bf16_bits(rng.integers(-2, 3, size=(B, H)).astype(np.float32))
+    wq = W.f32_to_bf16_bits(rng.integers(-2, 3, size=((Hq + 2 * Hkv) * d, H)).astype(np.float32))
+    opts = dict(rotary_dim=64, interleaved=True) if variant else {}
+    if variant:
+        w.rope_cos, w.rope_sin = W.rope_table(w.max_position, 64, w.rope_base)
+    q0, k0, v0 = O.oracle_qkv_projection(x, wq, Hq, Hkv, d)
+    bad_page, bad_pos = 1, 3
+    ok_rows = [b for b in range(B) if b not in (bad_page, bad_pos)]
+    lens_ok = w.context_lens.copy()
+    lens_ok[[bad_page, bad_pos]] = -1                      # the oracle skips the two rows
+    q_ref, k_ref, v_ref = O.oracle_rope_kv_append_ex(q0, k0, v0, w.k_cache, w.v_cache, w.block_table, lens_ok,
+                                                     w.rope_cos, w.rope_sin, ps, rotary_dim=opts.get("rotary_dim"),
+                                                     interleaved=opts.get("interleaved", False))
+    st = runner.DecodeStep(w, num_splits=1)
+    bt = w.block_table.copy()
+    bt[bad_page, lens[bad_page] // ps] = 1_000_000
+    st.block_table.copy_(torch.from_numpy(bt))
+    lens_dev = w.context_lens.copy()
+    lens_dev[bad_pos] = w.max_position + 3
+    st.context_lens.copy_(torch.from_numpy(lens_dev))
+    st.q_rot.fill_(0x7FC0)
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda()
+    ac.ac_qkv_rope_kv_append_ex(dev(x), dev(wq), H, st.q_rot, st.k_cache, st.v_cache, st.stride_page,
+                                st.stride_token, st.stride_head, st.block_table, w.max_pages_per_seq,
+                                st.context_lens, st.rope_cos, st.rope_sin, w.max_position, B, Hq, Hkv, d, ps,
+                                w.num_pages, st.status_flag, **opts)
+    torch.cuda.synchronize()
+    assert int(st.status_flag.item()) == 3
+    q_gpu = runner.bits_of(st.q_rot)
+    assert np.array_equal(q_gpu[ok_rows], q_ref[ok_rows])
+    assert (q_gpu[bad_pos] == 0x7FC0).all()                # q of the row with the bad page id is still valid
+    k_gpu, v_gpu = st.cache_bits()
+    assert np.array_equal(k_gpu, k_ref) and np.array_equal(v_gpu, v_ref)
+
+
 @pytest.mark.parametrize("B", [8, 100])
 def test_qkv_prelude_bit_exact_when_the_projection_is_exact(B):
     """Small-integer x and W make every dot product an integer that fp32 and fp64 both hold exactly, so
