@@ -436,7 +436,9 @@ int ac_qkv_rope_kv_append_ex(const void* x, const void* w_qkv, int H, void* q_ou
         cuuint64_t wdims[5] = {64, static_cast<cuuint64_t>(d / 2), 2, static_cast<cuuint64_t>(Hq + 2 * Hkv),
                                static_cast<cuuint64_t>(H / 64)};
         cuuint64_t wstrides[4] = {row_bytes, row_bytes * (d / 2), row_bytes * d, 128};
-        cuuint32_t wbox[5] = {64, 24, 2, 1, static_cast<cuuint32_t>(proj_tc_k_blocks(B))};
+        // 24 pairs per tile (plain epilogue: overlapping tiles), 32 with the prelude variants (disjoint tiles)
+        cuuint32_t wbox[5] = {64, static_cast<cuuint32_t>(vp != nullptr ? 32 : 24), 2, 1,
+                              static_cast<cuuint32_t>(proj_tc_k_blocks(B))};
         cuuint32_t es5[5] = {1, 1, 1, 1, 1};
         CUresult r = g_encode_tiled(&w_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(w_qkv),
                                     wdims, wstrides, wbox, es5, CU_TENSOR_MAP_INTERLEAVE_NONE,

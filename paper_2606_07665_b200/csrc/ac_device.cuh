@@ -142,6 +142,15 @@ __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// The two halves of that barrier, for a CTA that only has to outlive its sisters' reads of its shared
+// memory: arrive when done reading theirs, wait before exiting.  No other cluster barrier in between.
+__device__ __forceinline__ void cluster_arrive_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait_all() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // ---- ldmatrix / mma ---------------------------------------------------------------------------
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3,

@@ -12,6 +12,13 @@
 //            has 64 pairs (d = 128), so three tiles start at pairs 0, 16 and 40: 144 CTAs for 48 head
 //            slots; the pairs that two tiles share are computed twice and stored twice with the same
 //            bits (12.5 % more weight traffic for 50 % more SMs).
+//   QKV with prelude variants (per-head norm, partial or interleaved rotary)
+//            64 features per CTA = 32 pairs, disjoint tiles (two per head for d = 128, one for d = 64)
+//            that form a thread-block cluster: the norm needs the sum of squares over the whole head,
+//            and a partial half-split rotation needs partners from the sister tile, both through
+//            distributed shared memory.  Clusters of three 1-CTA-per-SM tiles left SMs idle; clusters
+//            of two pack.  The epilogue parks the rounded accumulators in the idle ring and runs the
+//            norm and the rotation with one warp per batch row and one lane per pair.
 //   o_proj   32 consecutive output features per CTA (128 CTAs for N = 4096).
 // Per CTA:
 //   warp 0   producer: per 128-wide K chunk one 3-D TMA load of the x tile [x_rows x 2 x 64] and one
@@ -47,8 +54,11 @@ constexpr int TC_SMEM_TOTAL = TC_BAR_OFFSET + (2 * TC_MAX_STAGES + 1) * 8 + 16 +
 
 template <int EPI>
 struct TcTile {
-    static constexpr int N = EPI == TC_EPI_RESIDUAL_ADD ? 32 : 48;           // features per CTA
-    static constexpr int GROUPS = EPI == TC_EPI_RESIDUAL_ADD ? 2 : 3;        // epilogue warps per 32 rows
+    // features per CTA: 48 (QKV; three overlapping tiles per head put a CTA on nearly every SM), 32
+    // (o_proj), 64 (QKV with prelude variants: two disjoint tiles per head, which pair up as clusters
+    // of two without leaving SMs idle the way clusters of three 1-CTA-per-SM tiles did)
+    static constexpr int N = EPI == TC_EPI_RESIDUAL_ADD ? 32 : (EPI == TC_EPI_QKV_ROPE_VARIANT ? 64 : 48);
+    static constexpr int GROUPS = N / 16;                                     // epilogue warps per 32 rows
     static constexpr int THREADS = 64 + 128 * GROUPS + 32;       // the last warp holds the second MMA issuer
     static constexpr int MMA2_WARP = 2 + 4 * GROUPS;
     static constexpr int B_BLOCK = N * 128;          // one swizzled [N rows x 128 B] block of W
@@ -85,16 +95,51 @@ struct TcParams {
     float norm_eps;
 };
 
-// Pairs of a head that QKV tile `blk` OWNS (tiles overlap; every pair has one owner): with 64 pairs
-// per head tile 0 owns [0, 16), tile 1 [16, 40), tile 2 [40, 64); with 32 pairs tile 0 owns [0, 8) and
-// tile 1 [8, 32).
-__host__ __device__ inline int qkv_tile_own_begin(int half_d, int blk) { return qkv_tile_first_pair(half_d, blk); }
-__host__ __device__ inline int qkv_tile_own_end(int half_d, int blk) {
-    return half_d == 64 ? (blk == 0 ? 16 : blk == 1 ? 40 : 64) : (blk == 0 ? 8 : 32);
+// Where the variant epilogue keeps its working set, in the shared memory of the (by then idle) ring.
+// A feature row is 66 values long so that 32 threads, one batch row each, hit 32 different banks.
+struct VariantSmem {
+    static constexpr int ROW = 66;                                    // bf16 values per parked row
+    static constexpr int VALS = 0;                                    // [128][ROW] rounded features
+    static constexpr int VALSN = VALS + TC_M * ROW * 2;               // [128][ROW] after the norm
+    static constexpr int PSUM = VALSN + TC_M * ROW * 2;               // [4 column groups][128] sums of squares
+    static constexpr int RSCALE = PSUM + 4 * TC_M * 8;                // [128] 1 / rms of the row
+    static constexpr int ROW_DST = RSCALE + TC_M * 8;                 // [128] destination rows
+    static constexpr int ROW_CTX = ROW_DST + TC_M * 8;                // [128] position; -1: row not stored
+    static constexpr int END = ROW_CTX + TC_M * 4;
+    static_assert(PSUM % 8 == 0 && END <= TC_RING_BYTES, "variant epilogue working set");
+};
+
+// y = bf16(bf16(v * rr) * w) with both roundings to nearest even of the fp64 products (the per-head
+// RMSNorm of one feature; rr = 1 / rms as fp64, w a bf16 weight).  The first product is evaluated in
+// fp32 with its residual (rr split in two floats), which provably rounds like the fp64 product when the
+// result is three fp32 ulps clear of every midpoint between bf16 values; otherwise fp64 decides.  The
+// second product of two bf16 values is exact in fp32.
+// The rare fp64 ways out of rmsnorm_feature, kept out of line so that the common path holds no fp64.
+__device__ __noinline__ uint16_t bf16_of_product_f64(float a, double b) {
+    return f64_to_bf16_rne(__dmul_rn(static_cast<double>(a), b));
 }
-__host__ __device__ inline int qkv_tile_owner(int half_d, int pair) {
-    return half_d == 64 ? (pair < 16 ? 0 : pair < 40 ? 1 : 2) : (pair < 8 ? 0 : 1);
+
+__device__ __forceinline__ uint16_t rmsnorm_feature(uint16_t v16, double rr, float rr_hi, float rr_lo, float wf) {
+    const float v = bf16_bits_to_float(v16);
+    const float pr = __fmul_rn(v, rr_hi);
+    const float pl = __fmaf_rn(v, rr_hi, -pr);                        // exact residual of the product
+    const float r = __fadd_rn(pr, __fmaf_rn(v, rr_lo, pl));
+    const uint32_t u = __float_as_uint(r);
+    const float mag = fabsf(pr);
+    uint16_t y1 = static_cast<uint16_t>((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
+    if (!((((u & 0xFFFFu) - 0x7FFEu) > 4u) && mag >= 0x1p-60f && mag <= 0x1p100f))
+        y1 = bf16_of_product_f64(v, rr);
+    const float y1f = bf16_bits_to_float(y1);
+    const float q = __fmul_rn(y1f, wf);
+    const float qmag = fabsf(q);
+    if (!(qmag >= 0x1p-100f && qmag <= 0x1p100f))                     // zero, tiny, huge or NaN: the plain way
+        return bf16_of_product_f64(y1f, static_cast<double>(wf));
+    const uint32_t uq = __float_as_uint(q);
+    return static_cast<uint16_t>((uq + 0x7FFFu + ((uq >> 16) & 1u)) >> 16);
 }
+
+// The variant epilogue's tiles are disjoint blocks of 32 pairs: tile blk holds pairs [32 blk, 32 blk + 32).
+constexpr int kVariantTilePairs = 32;
 
 // ---- tcgen05 wrappers ---------------------------------------------------------------------------
 
@@ -182,7 +227,8 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
 
     const int blk = blockIdx.x;          // pair tile inside the head (QKV) / unused (o_proj)
     const int hh = blockIdx.y;           // head slot (QKV) / block of 32 output features (o_proj)
-    const int pair0 = EPI == TC_EPI_RESIDUAL_ADD ? 0 : qkv_tile_first_pair(p.d / 2, blk);
+    const int pair0 = EPI == TC_EPI_RESIDUAL_ADD ? 0
+                      : EPI == TC_EPI_QKV_ROPE_VARIANT ? kVariantTilePairs * blk : qkv_tile_first_pair(p.d / 2, blk);
     // The x box holds x_rows rows per 64-element block; the MMA always reads 128.  Rows past x_rows are
     // whatever the ring holds: every accumulator row depends on its own x row only, and the epilogue
     // skips them.  A stage is the x tile followed by the W tile.
@@ -210,6 +256,54 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_d = *tmem_slot_gen;
+    // Prelude variants.  After the accumulators are parked in shared memory, the norm and the rotation
+    // run with one epilogue warp per batch row and one lane per rotary pair of the tile (both halves).
+    // What does not depend on the accumulators is fetched under the main loop: this lane's two norm
+    // weights here, the rotation geometry of its two features -- partner, table entry, which half; the
+    // same for every row -- and, in the epilogue warps, the table entries of the warp's rows.
+    constexpr int VWARPS = 4 * T::GROUPS;                    // epilogue warps
+    constexpr int VROWS = (TC_M + VWARPS - 1) / VWARPS;      // rows per epilogue warp in those passes
+    const int n_rows = max(0, min(p.x_rows, p.B - b0));      // batch rows this CTA holds
+    uint16_t norm_w_lo = 0, norm_w_hi = 0;
+    int v_feat[2] = {0, 0}, v_ri[2] = {0, 0}, v_pcol[2] = {0, 0}, v_owner[2] = {0, 0};
+    bool v_rot[2] = {false, false}, v_first[2] = {false, false};
+    float v_cs[VROWS][2], v_sn[VROWS][2];
+    if (EPI == TC_EPI_QKV_ROPE_VARIANT) {
+        const bool rotated_head = hh < p.Hq + p.Hkv;
+        const uint16_t* nw = hh < p.Hq ? p.q_norm_w : (rotated_head ? p.k_norm_w : nullptr);
+        const int half_d = p.d / 2, R = p.rotary_dim, half_r = R / 2;
+        if (nw != nullptr) {
+            norm_w_lo = nw[pair0 + lane];
+            norm_w_hi = nw[half_d + pair0 + lane];
+        }
+#pragma unroll
+        for (int hsel = 0; hsel < 2; ++hsel) {
+            const int f = (hsel == 0 ? 0 : half_d) + pair0 + lane;           // feature inside the head
+            v_feat[hsel] = f;
+            v_rot[hsel] = rotated_head && f < R;
+            int partner;
+            if (p.interleaved) {
+                v_ri[hsel] = f >> 1;
+                v_first[hsel] = (f & 1) == 0;
+                partner = v_first[hsel] ? f + 1 : f - 1;
+            } else {
+                v_first[hsel] = f < half_r;
+                v_ri[hsel] = v_first[hsel] ? f : f - half_r;
+                partner = v_first[hsel] ? f + half_r : f - half_r;
+            }
+            if (!v_rot[hsel]) partner = f;
+            const int ppair = partner & (half_d - 1);                        // head_dim / 2 is 32 or 64
+            v_owner[hsel] = ppair / kVariantTilePairs;
+            v_pcol[hsel] = (partner >= half_d ? T::N / 2 : 0) + (ppair - kVariantTilePairs * v_owner[hsel]);
+        }
+#pragma unroll
+        for (int it = 0; it < VROWS; ++it)
+#pragma unroll
+            for (int hsel = 0; hsel < 2; ++hsel) {
+                v_cs[it][hsel] = 1.0f;
+                v_sn[it][hsel] = 0.0f;
+            }
+    }
     cudaGridDependencySynchronize();      // x (and the residual) come from the preceding kernel
 
     bool timed_out = false;
@@ -328,7 +422,59 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
             // prelude variants: this warp only rounds its 8 pairs and parks them in shared memory (the
             // ring is free once the accumulators are complete); the norm and the rotation follow below,
             // by all threads of the CTA, because they reach across columns and across sister CTAs.
-            uint16_t* vals = reinterpret_cast<uint16_t*>(smem_gen);          // [128 rows][48]
+            // where the row goes (as in the plain epilogue), looked up under the main loop
+            int ctx = -1;
+            unsigned long long dst = 0;
+            {
+                // table entries of the rows this warp rotates later (rows warp - 2, + 16, ...); a full
+                // half-split rotation turns both halves of a pair by the same entry
+                const int half_r = p.rotary_dim / 2;
+                const bool one_entry = v_rot[0] == v_rot[1] && v_ri[0] == v_ri[1];
+#pragma unroll
+                for (int it = 0; it < VROWS; ++it) {
+                    const int prow = (warp - 2) + it * VWARPS;
+                    if (prow >= n_rows) continue;            // the same for the whole warp
+                    const int c = p.context_lens[b0 + prow];
+                    const bool valid = c >= 0 && c < p.max_position;
+                    // loads without a condition (entry 0 when there is nothing to rotate)
+                    const size_t e0 = (valid && v_rot[0]) ? static_cast<size_t>(c) * half_r + v_ri[0] : 0;
+                    v_cs[it][0] = __ldg(p.rope_cos + e0);
+                    v_sn[it][0] = __ldg(p.rope_sin + e0);
+                    if (one_entry) {
+                        v_cs[it][1] = v_cs[it][0];
+                        v_sn[it][1] = v_sn[it][0];
+                    } else {
+                        const size_t e1 = (valid && v_rot[1]) ? static_cast<size_t>(c) * half_r + v_ri[1] : 0;
+                        v_cs[it][1] = __ldg(p.rope_cos + e1);
+                        v_sn[it][1] = __ldg(p.rope_sin + e1);
+                    }
+                }
+            }
+            if (group == 0 && ok) {
+                const bool is_q = hh < p.Hq, is_k = !is_q && hh < p.Hq + p.Hkv;
+                ctx = p.context_lens[b];
+                if (ctx >= 0) {
+                    const int page_idx = ctx / p.page_size;
+                    if (ctx >= p.max_position || page_idx >= p.max_pages_per_seq) {
+                        if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
+                        ctx = -1;
+                    } else if (is_q) {
+                        dst = reinterpret_cast<unsigned long long>(p.q_out + (static_cast<size_t>(b) * p.Hq + hh) * p.d);
+                    } else {
+                        const int page = p.block_table[static_cast<size_t>(b) * p.max_pages_per_seq + page_idx];
+                        if (page < 0 || page >= p.num_pages) {
+                            if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
+                            ctx = -1;
+                        } else {
+                            const int h = is_k ? hh - p.Hq : hh - p.Hq - p.Hkv;
+                            dst = reinterpret_cast<unsigned long long>(
+                                (is_k ? p.k_cache : p.v_cache) + static_cast<size_t>(page) * p.stride_page +
+                                static_cast<size_t>(ctx - page_idx * p.page_size) * p.stride_token +
+                                static_cast<size_t>(h) * p.stride_head);
+                        }
+                    }
+                }
+            }
             const bool ready = mbar_wait_bounded(done_bar, 0);
             if (!ready && lane == 0 && p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_WAIT_TIMEOUT);
             tc_fence_after_sync();
@@ -338,16 +484,30 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
             tmem_ld_32x8(lane_base + T::ACC_COLS + 8 * group, lo_odd);
             tmem_ld_32x8(lane_base + T::ACC_COLS + T::N / 2 + 8 * group, hi_odd);
             tmem_ld_wait();
+            uint32_t* vrow = reinterpret_cast<uint32_t*>(smem_gen + VariantSmem::VALS) + row * (VariantSmem::ROW / 2);
+            double ss = 0.0;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                float a = __uint_as_float(lo[e]), bq = __uint_as_float(hi[e]);
-                if (n_chunks > 1) {
-                    a += __uint_as_float(lo_odd[e]);
-                    bq += __uint_as_float(hi_odd[e]);
+            for (int e = 0; e < 8; e += 2) {
+                uint32_t pk[2];
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    float a = __uint_as_float(lo[e + t]), bq = __uint_as_float(hi[e + t]);
+                    if (n_chunks > 1) {
+                        a += __uint_as_float(lo_odd[e + t]);
+                        bq += __uint_as_float(hi_odd[e + t]);
+                    }
+                    pk[t] = (ready && ok) ? pack_bf16x2(a, bq) : 0u;
+                    const double ar = static_cast<double>(__uint_as_float(pk[t] << 16));
+                    const double br = static_cast<double>(__uint_as_float(pk[t] & 0xFFFF0000u));
+                    ss = __dadd_rn(ss, __dadd_rn(__dmul_rn(ar, ar), __dmul_rn(br, br)));
                 }
-                const uint32_t pk = (ready && ok) ? pack_bf16x2(a, bq) : 0u;
-                vals[row * T::N + 8 * group + e] = static_cast<uint16_t>(pk & 0xFFFFu);
-                vals[row * T::N + T::N / 2 + 8 * group + e] = static_cast<uint16_t>(pk >> 16);
+                vrow[(8 * group + e) >> 1] = (pk[0] & 0xFFFFu) | (pk[1] << 16);
+                vrow[(T::N / 2 + 8 * group + e) >> 1] = (pk[0] >> 16) | (pk[1] & 0xFFFF0000u);
+            }
+            reinterpret_cast<double*>(smem_gen + VariantSmem::PSUM)[group * TC_M + row] = ss;
+            if (group == 0) {                                // the ring is free: these arrays live in it too
+                reinterpret_cast<int*>(smem_gen + VariantSmem::ROW_CTX)[row] = ready ? ctx : -1;
+                reinterpret_cast<unsigned long long*>(smem_gen + VariantSmem::ROW_DST)[row] = dst;
             }
         } else {
             // 8 rotary pairs: first halves in columns 8 group .., second halves in columns 24 + 8 group ..
@@ -463,110 +623,94 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
     }
     if (EPI == TC_EPI_QKV_ROPE_VARIANT) {
         // ---- prelude variants: norm and rotation across the tiles of a head ----------------------------
-        // The two or three tiles of a head slot (blockIdx.x) are one thread-block cluster.  Tiles overlap,
-        // so every pair has one OWNER tile: sums of squares count owned pairs only, and a rotation
-        // partner is fetched from its owner.  Three cluster barriers, executed by every thread of every
-        // CTA on every path: parked features and partial sums visible; normalised features visible;
-        // nobody's shared memory released while a sister still reads it.
-        const int d = p.d, half_d = d / 2;
-        uint16_t* vals = reinterpret_cast<uint16_t*>(smem_gen);                        // [128][48] rounded
-        uint16_t* valsn = vals + TC_M * T::N;                                           // [128][48] after the norm
-        double* sums = reinterpret_cast<double*>(valsn + TC_M * T::N);                  // [128]
-        int* row_ctx = reinterpret_cast<int*>(sums + TC_M);                             // [128]; -1: row not stored
-        unsigned long long* row_dst = reinterpret_cast<unsigned long long*>(row_ctx + TC_M);   // [128] destination rows
+        // The tiles of a head slot (blockIdx.x: two blocks of 32 pairs for head_dim 128, one for 64) are
+        // one thread-block cluster.  With remote rotation partners three cluster barriers: parked features
+        // and partial sums visible; normalised features visible; nobody's shared memory released while a
+        // sister still reads it.  With local partners the sums are the only remote reads: one barrier
+        // before them, and one whose arrival follows them and whose wait is the last thing the CTA does.
+        // Every thread of every CTA of a cluster takes the same path through them.
+        const int d = p.d;
+        constexpr int VS = VariantSmem::ROW;
+        uint16_t* vals = reinterpret_cast<uint16_t*>(smem_gen + VariantSmem::VALS);
+        uint16_t* valsn = reinterpret_cast<uint16_t*>(smem_gen + VariantSmem::VALSN);
+        double* psum = reinterpret_cast<double*>(smem_gen + VariantSmem::PSUM);
+        double* rscale = reinterpret_cast<double*>(smem_gen + VariantSmem::RSCALE);
+        int* row_ctx = reinterpret_cast<int*>(smem_gen + VariantSmem::ROW_CTX);
+        unsigned long long* row_dst = reinterpret_cast<unsigned long long*>(smem_gen + VariantSmem::ROW_DST);
         const bool is_q = hh < p.Hq, is_k = !is_q && hh < p.Hq + p.Hkv;
         const uint16_t* norm_w = is_q ? p.q_norm_w : (is_k ? p.k_norm_w : nullptr);
         const int n_tiles = gridDim.x;
-        __syncthreads();                                      // the epilogue warps have parked the features
-        if (threadIdx.x < TC_M) {
-            const int row = threadIdx.x;
-            const int b = b0 + row;
-            double ss = 0.0;
-            for (int i = qkv_tile_own_begin(half_d, blk); i < qkv_tile_own_end(half_d, blk); ++i) {
-                const double a = static_cast<double>(bf16_bits_to_float(vals[row * T::N + (i - pair0)]));
-                const double bq = static_cast<double>(bf16_bits_to_float(vals[row * T::N + T::N / 2 + (i - pair0)]));
-                ss = __dadd_rn(ss, __dadd_rn(__dmul_rn(a, a), __dmul_rn(bq, bq)));
+        const bool pass_warp = warp >= 2 && warp < T::MMA2_WARP;     // the epilogue warps run the passes
+        static_assert(EPI != TC_EPI_QKV_ROPE_VARIANT || T::N / 2 == 32, "one lane per rotary pair of the tile");
+        // A rotation partner sits in a sister's tile only for a half-split rotation over part of the head.
+        // Both conditions are the same in every CTA of the cluster (same head slot, same parameters).
+        const bool remote_partner = (is_q || is_k) && !p.interleaved && p.rotary_dim != d;
+        const bool has_norm = norm_w != nullptr;
+        if (has_norm || remote_partner) cluster_sync_all();   // everybody's parked features and partial sums
+        else __syncthreads();
+        if (norm_w != nullptr && threadIdx.x < n_rows) {
+            double total = 0.0;
+            for (int c = 0; c < n_tiles; ++c)
+#pragma unroll
+                for (int g = 0; g < T::GROUPS; ++g)
+                    total = __dadd_rn(total, cluster_load_f64(cluster_map_shared(smem_addr(psum + g * TC_M + threadIdx.x), c)));
+            // head_dim is a power of two: the mean is an exact scaling; 1 / x by the correctly rounded reciprocal
+            rscale[threadIdx.x] = __drcp_rn(__dsqrt_rn(__dadd_rn(__dmul_rn(total, 1.0 / static_cast<double>(d)),
+                                                                 static_cast<double>(p.norm_eps))));
+        }
+        __syncthreads();
+        // Sisters read this CTA's partial sums above: it must not exit before they have.  With local
+        // partners that is the last remote access, so arrive now and wait at the very end.
+        const bool split_barrier = has_norm && !remote_partner;
+        if (split_barrier) cluster_arrive_all();
+        // Every sister of the cluster has the same head slot, hence the same answer to "is there a norm":
+        // without one the rotation reads the parked features where they are.
+        const uint16_t* rot_src = norm_w != nullptr ? valsn : vals;
+        if (norm_w != nullptr && pass_warp) {
+            const float w_lo = bf16_bits_to_float(norm_w_lo), w_hi = bf16_bits_to_float(norm_w_hi);
+#pragma unroll
+            for (int it = 0; it < VROWS; ++it) {
+                const int row = (warp - 2) + it * VWARPS;
+                if (row >= n_rows) continue;
+                const double rr = rscale[row];
+                const float rr_hi = __double2float_rn(rr);
+                const float rr_lo = __double2float_rn(__dsub_rn(rr, static_cast<double>(rr_hi)));
+#pragma unroll
+                for (int hsel = 0; hsel < 2; ++hsel) {
+                    const int item = row * VS + hsel * (T::N / 2) + lane;
+                    valsn[item] = rmsnorm_feature(vals[item], rr, rr_hi, rr_lo, hsel == 0 ? w_lo : w_hi);
+                }
             }
-            sums[row] = ss;
-            // where the row goes (as in the plain epilogue)
-            int ctx = -1;
-            unsigned long long dst = 0;
-            if (row < p.x_rows && b < p.B) {
-                ctx = p.context_lens[b];
-                if (ctx >= 0) {
-                    const int page_idx = ctx / p.page_size;
-                    if (ctx >= p.max_position || page_idx >= p.max_pages_per_seq) {
-                        if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
-                        ctx = -1;
-                    } else if (is_q) {
-                        dst = reinterpret_cast<unsigned long long>(p.q_out + (static_cast<size_t>(b) * p.Hq + hh) * d);
-                    } else {
-                        const int page = p.block_table[static_cast<size_t>(b) * p.max_pages_per_seq + page_idx];
-                        if (page < 0 || page >= p.num_pages) {
-                            if (p.status_flag != nullptr) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
-                            ctx = -1;
-                        } else {
-                            const int h = is_k ? hh - p.Hq : hh - p.Hq - p.Hkv;
-                            dst = reinterpret_cast<unsigned long long>(
-                                (is_k ? p.k_cache : p.v_cache) + static_cast<size_t>(page) * p.stride_page +
-                                static_cast<size_t>(ctx - page_idx * p.page_size) * p.stride_token +
-                                static_cast<size_t>(h) * p.stride_head);
-                        }
+        }
+        if (remote_partner) cluster_sync_all();               // the sisters' normalised features
+        else __syncthreads();
+        if (pass_warp) {
+#pragma unroll
+            for (int it = 0; it < VROWS; ++it) {
+                const int row = (warp - 2) + it * VWARPS;
+                if (row >= n_rows || row_ctx[row] < 0) continue;     // the same for the whole warp
+                uint16_t* dst_row = reinterpret_cast<uint16_t*>(row_dst[row]);
+#pragma unroll
+                for (int hsel = 0; hsel < 2; ++hsel) {
+                    uint16_t v16 = rot_src[row * VS + hsel * (T::N / 2) + lane];
+                    if (v_rot[hsel]) {
+                        const uint16_t* psrc = rot_src + row * VS + v_pcol[hsel];
+                        const uint16_t other = v_owner[hsel] == blk
+                                                   ? *psrc
+                                                   : cluster_load_u16(cluster_map_shared(smem_addr(psrc), v_owner[hsel]));
+                        // first half: x c - partner s; second half: x c + partner s
+                        const float mine = bf16_bits_to_float(v16), theirs = bf16_bits_to_float(other);
+                        const float s_signed = v_first[hsel] ? v_sn[it][hsel] : -v_sn[it][hsel];
+                        bool proven;
+                        v16 = rope_diff_of_products_f32(mine, v_cs[it][hsel], theirs, s_signed, proven);
+                        if (!proven) v16 = rope_diff_of_products_f64(mine, v_cs[it][hsel], theirs, s_signed);
                     }
+                    dst_row[v_feat[hsel]] = v16;
                 }
             }
-            row_ctx[row] = ctx;
-            row_dst[row] = dst;
         }
-        cluster_sync_all();
-        for (int item = threadIdx.x; item < TC_M * T::N; item += T::THREADS) {
-            const int row = item / T::N, col = item - row * T::N;
-            uint16_t v16 = vals[item];
-            if (norm_w != nullptr) {
-                double total = 0.0;
-                for (int c = 0; c < n_tiles; ++c)
-                    total = __dadd_rn(total, cluster_load_f64(cluster_map_shared(smem_addr(sums + row), c)));
-                const double rr = __ddiv_rn(1.0, __dsqrt_rn(__dadd_rn(__ddiv_rn(total, static_cast<double>(d)),
-                                                                      static_cast<double>(p.norm_eps))));
-                const int f = (col >= T::N / 2 ? half_d : 0) + pair0 + (col % (T::N / 2));     // feature inside the head
-                const uint16_t y1 = f64_to_bf16_rne(__dmul_rn(static_cast<double>(bf16_bits_to_float(v16)), rr));
-                v16 = f64_to_bf16_rne(__dmul_rn(static_cast<double>(bf16_bits_to_float(y1)),
-                                                static_cast<double>(bf16_bits_to_float(norm_w[f]))));
-            }
-            valsn[item] = v16;
-        }
-        cluster_sync_all();
-        const int R = p.rotary_dim, half_r = R / 2;
-        for (int item = threadIdx.x; item < TC_M * T::N; item += T::THREADS) {
-            const int row = item / T::N, col = item - row * T::N;
-            const int ctx = row_ctx[row];
-            if (ctx < 0) continue;
-            const int pair = pair0 + (col % (T::N / 2));
-            const int f = (col >= T::N / 2 ? half_d : 0) + pair;
-            uint16_t v16 = valsn[item];
-            if ((is_q || is_k) && f < R) {
-                int i, partner;
-                bool first;
-                if (p.interleaved) {
-                    i = f >> 1;
-                    first = (f & 1) == 0;
-                    partner = first ? f + 1 : f - 1;
-                } else {
-                    first = f < half_r;
-                    i = first ? f : f - half_r;
-                    partner = first ? f + half_r : f - half_r;
-                }
-                const int ppair = partner % half_d;
-                const int owner = qkv_tile_owner(half_d, ppair);
-                const int pcol = (partner >= half_d ? T::N / 2 : 0) + (ppair - qkv_tile_first_pair(half_d, owner));
-                const uint16_t other = cluster_load_u16(cluster_map_shared(smem_addr(valsn + row * T::N + pcol), owner));
-                const float c = p.rope_cos[static_cast<size_t>(ctx) * half_r + i];
-                const float sn = p.rope_sin[static_cast<size_t>(ctx) * half_r + i];
-                v16 = first ? rope_first_half(v16, other, c, sn) : rope_second_half(other, v16, c, sn);
-            }
-            reinterpret_cast<uint16_t*>(row_dst[row])[f] = v16;
-        }
-        cluster_sync_all();
+        if (remote_partner) cluster_sync_all();               // nobody's shared memory goes while a sister reads it
+        else if (split_barrier) cluster_wait_all();
     }
 
     // ---- release TMEM (every path reaches this point) ----------------------------------------------
@@ -674,12 +818,13 @@ cudaError_t launch_qkv_rope_kv_append_tc(const CUtensorMap& w_map, const CUtenso
     p.x_rows = proj_tc_batch_rows(B);
     const dim3 grid(d == 128 ? 3 : 2, Hq + 2 * Hkv, (B + p.x_rows - 1) / p.x_rows);
     if (variant != nullptr) {
+        const dim3 vgrid(d / 2 / kVariantTilePairs, Hq + 2 * Hkv, (B + p.x_rows - 1) / p.x_rows);
         p.rotary_dim = variant->rotary_dim;
         p.interleaved = variant->interleaved;
         p.q_norm_w = static_cast<const uint16_t*>(variant->q_norm_weight);
         p.k_norm_w = static_cast<const uint16_t*>(variant->k_norm_weight);
         p.norm_eps = variant->norm_eps;
-        return launch_tc<TC_EPI_QKV_ROPE_VARIANT>(w_map, x_map, p, proj_tc_k_blocks(B), grid, stream);
+        return launch_tc<TC_EPI_QKV_ROPE_VARIANT>(w_map, x_map, p, proj_tc_k_blocks(B), vgrid, stream);
     }
     return launch_tc<TC_EPI_QKV_ROPE_APPEND>(w_map, x_map, p, proj_tc_k_blocks(B), grid, stream);
 }

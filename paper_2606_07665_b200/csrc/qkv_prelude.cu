@@ -290,15 +290,20 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
             sums[threadIdx.x] = ss;
         }
         cluster_sync_all();
+        __shared__ double s_rscale[16];                 // 1 / rms of each batch row of the tile
+        if (norm_w != nullptr && threadIdx.x < BT) {
+            double total = 0.0;
+            for (int c = 0; c < n_cta; ++c)
+                total = __dadd_rn(total, cluster_load_f64(cluster_map_shared(smem_addr(sums + threadIdx.x), c)));
+            s_rscale[threadIdx.x] = __ddiv_rn(1.0, __dsqrt_rn(__dadd_rn(__ddiv_rn(total, static_cast<double>(d)),
+                                                                        static_cast<double>(p.norm_eps))));
+        }
+        __syncthreads();
         for (int item = threadIdx.x; item < 32 * BT; item += QKV_THREADS) {
             const int r = item / BT, n = item - r * BT;
             uint16_t v16 = vals[item];
             if (norm_w != nullptr) {
-                double total = 0.0;
-                for (int c = 0; c < n_cta; ++c)
-                    total = __dadd_rn(total, cluster_load_f64(cluster_map_shared(smem_addr(sums + n), c)));
-                const double rr = __ddiv_rn(1.0, __dsqrt_rn(__dadd_rn(__ddiv_rn(total, static_cast<double>(d)),
-                                                                      static_cast<double>(p.norm_eps))));
+                const double rr = s_rscale[n];
                 const int f = (r >> 4) * half_d + 16 * blk + (r & 15);               // feature inside the head
                 const uint16_t y1 = f64_to_bf16_rne(__dmul_rn(static_cast<double>(bf16_bits_to_float(v16)), rr));
                 v16 = f64_to_bf16_rne(__dmul_rn(static_cast<double>(bf16_bits_to_float(y1)),
