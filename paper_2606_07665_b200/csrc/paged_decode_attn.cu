@@ -683,9 +683,13 @@ __global__ void __launch_bounds__(THREADS, STAGES == kStages ? 2 : 1) paged_deco
     }
     __syncthreads();
 
-    for (int e = threadIdx.x; e < G * D; e += THREADS) {
-        const int row = e / D;
-        const int col = e - row * D;
+    // One item = four consecutive output elements of one query row: a warp covers one row per pass, so
+    // the weights of the row's four partial results are computed once per item and reused for its four
+    // columns, and every load and store is 16 bytes (8 for the bf16 result) wide.
+    constexpr int C4 = D / 4;
+    for (int e = threadIdx.x; e < G * C4; e += THREADS) {
+        const int row = e / C4;
+        const int col = (e - row * C4) * 4;
         float mw[WARPS];
         float M = -INFINITY;
 #pragma unroll
@@ -693,25 +697,30 @@ __global__ void __launch_bounds__(THREADS, STAGES == kStages ? 2 : 1) paged_deco
             mw[w] = reinterpret_cast<const float*>(smem_gen + w * L::RING_BYTES)[WROWS * WSTRIDE + row];
             M = fmaxf(M, mw[w]);
         }
-        float num = 0.0f, den = 0.0f;
+        float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+        float den = 0.0f;
 #pragma unroll
         for (int w = 0; w < WARPS; ++w) {
             const float* base = reinterpret_cast<const float*>(smem_gen + w * L::RING_BYTES);
             const float wgt = exp2f(mw[w] - M);                 // 0 for a warp that saw no tile
-            num = fmaf(wgt, base[row * WSTRIDE + col], num);
+            const float4 o4 = *reinterpret_cast<const float4*>(base + row * WSTRIDE + col);
+            num.x = fmaf(wgt, o4.x, num.x);
+            num.y = fmaf(wgt, o4.y, num.y);
+            num.z = fmaf(wgt, o4.z, num.z);
+            num.w = fmaf(wgt, o4.w, num.w);
             den = fmaf(wgt, base[WROWS * WSTRIDE + WROWS + row], den);
         }
-        const float val = num / den;
+        const float4 val = make_float4(num.x / den, num.y / den, num.z / den, num.w / den);
         const size_t hq = static_cast<size_t>(b) * p.Hq + h * G + row;
         if (S == 1) {
-            const uint16_t bits = static_cast<uint16_t>(pack_bf16x2(val, 0.0f) & 0xFFFFu);
-            p.out[hq * D + col] = bits;
-            if (p.out_mirror != nullptr) p.out_mirror[hq * D + col] = bits;
+            const uint2 bits = make_uint2(pack_bf16x2(val.x, val.y), pack_bf16x2(val.z, val.w));
+            *reinterpret_cast<uint2*>(p.out + hq * D + col) = bits;
+            if (p.out_mirror != nullptr) *reinterpret_cast<uint2*>(p.out_mirror + hq * D + col) = bits;
         } else if (cluster_merge) {
-            *reinterpret_cast<float*>(smem_gen + staged_o(row, col)) = val;
+            *reinterpret_cast<float4*>(smem_gen + staged_o(row, col)) = val;
             if (col == 0) *reinterpret_cast<float*>(smem_gen + staged_lse(row)) = (M + log2f(den)) * LN2;
         } else {
-            p.partial_o[(hq * S + split) * D + col] = val;
+            *reinterpret_cast<float4*>(p.partial_o + (hq * S + split) * D + col) = val;
             if (col == 0) p.partial_lse[hq * S + split] = (M + log2f(den)) * LN2;
         }
     }
