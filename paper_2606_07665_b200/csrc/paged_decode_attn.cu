@@ -110,6 +110,82 @@ struct AttnParams {
 // and the fused step with the prelude variants (per-head RMSNorm, partial rotary, interleaved pairing).
 constexpr int ROPE_NONE = 0, ROPE_PLAIN = 1, ROPE_VARIANT = 2;
 
+// The merge of the ticket path: the CTA that arrived last combines the splits' partial results of its
+// (request, KV head) out of the workspace.  An item is four consecutive output elements of one query
+// row; a thread owns ITEMS of them (item = thread + k * THREADS) and walks the splits in groups of GS
+// for all its items at once: the ITEMS * GS 16-byte partial loads and their log-sum-exps are issued
+// before any is used, so a group costs one L2 round trip whatever the number of items, and groups are
+// combined with the same running-maximum rescaling as the main loop.  ITEMS * GS <= 16 keeps the
+// loads in registers.
+template <int D, int ITEMS, int GS>
+__device__ __forceinline__ void merge_splits_from_workspace(const AttnParams& p, size_t hq0, int items, int S,
+                                                            int n_active) {
+    constexpr int D4 = D / 4;
+    static_assert(ITEMS * GS <= 16, "loads of a group stay in registers");
+    const float* lse_g[ITEMS];
+    const float4* po[ITEMS];
+    bool live[ITEMS];
+    float M[ITEMS], den[ITEMS];
+    float4 acc[ITEMS];
+    size_t out_at[ITEMS];
+#pragma unroll
+    for (int k = 0; k < ITEMS; ++k) {
+        const int e = threadIdx.x + k * THREADS;
+        live[k] = e < items;
+        const int row = live[k] ? e / D4 : 0;
+        const int c4 = live[k] ? e - row * D4 : 0;
+        lse_g[k] = p.partial_lse + (hq0 + row) * S;
+        po[k] = reinterpret_cast<const float4*>(p.partial_o + (hq0 + row) * S * D) + c4;
+        out_at[k] = (hq0 + row) * D + c4 * 4;
+        M[k] = -INFINITY;
+        den[k] = 0.0f;
+        acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    for (int s0 = 0; s0 < n_active; s0 += GS) {
+        float4 v[ITEMS][GS];
+        float l[ITEMS][GS];
+#pragma unroll
+        for (int k = 0; k < ITEMS; ++k)
+#pragma unroll
+            for (int u = 0; u < GS; ++u) {
+                const bool on = live[k] && s0 + u < n_active;
+                l[k][u] = on ? __ldcg(lse_g[k] + s0 + u) : -INFINITY;
+                v[k][u] = on ? __ldcg(po[k] + static_cast<size_t>(s0 + u) * D4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+        for (int k = 0; k < ITEMS; ++k) {
+            float gm = M[k];
+#pragma unroll
+            for (int u = 0; u < GS; ++u) gm = fmaxf(gm, l[k][u]);
+            const float rescale = __expf(M[k] - gm);           // 0 on the first group (M = -inf)
+            acc[k].x *= rescale;
+            acc[k].y *= rescale;
+            acc[k].z *= rescale;
+            acc[k].w *= rescale;
+            den[k] *= rescale;
+            M[k] = gm;
+#pragma unroll
+            for (int u = 0; u < GS; ++u) {
+                const float wgt = __expf(l[k][u] - gm);        // 0 for the padding entries
+                acc[k].x = fmaf(wgt, v[k][u].x, acc[k].x);
+                acc[k].y = fmaf(wgt, v[k][u].y, acc[k].y);
+                acc[k].z = fmaf(wgt, v[k][u].z, acc[k].z);
+                acc[k].w = fmaf(wgt, v[k][u].w, acc[k].w);
+                den[k] += wgt;
+            }
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < ITEMS; ++k) {
+        if (!live[k]) continue;
+        const float inv = 1.0f / den[k];
+        const uint2 bits = make_uint2(pack_bf16x2(acc[k].x * inv, acc[k].y * inv),
+                                      pack_bf16x2(acc[k].z * inv, acc[k].w * inv));
+        *reinterpret_cast<uint2*>(p.out + out_at[k]) = bits;
+        if (p.out_mirror != nullptr) *reinterpret_cast<uint2*>(p.out_mirror + out_at[k]) = bits;
+    }
+}
+
 template <int D, bool WIDE, int ROPE, int STAGES>
 __global__ void __launch_bounds__(THREADS, STAGES == kStages ? 2 : 1) paged_decode_attn_kernel(
     const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
@@ -687,7 +763,11 @@ __global__ void __launch_bounds__(THREADS, STAGES == kStages ? 2 : 1) paged_deco
     // the weights of the row's four partial results are computed once per item and reused for its four
     // columns, and every load and store is 16 bytes (8 for the bf16 result) wide.
     constexpr int C4 = D / 4;
-    for (int e = threadIdx.x; e < G * C4; e += THREADS) {
+    constexpr int PASSES = (WROWS * C4 + THREADS - 1) / THREADS;   // two or three: unrolled, their loads overlap
+#pragma unroll
+    for (int pass = 0; pass < PASSES; ++pass) {
+        const int e = threadIdx.x + pass * THREADS;
+        if (e >= G * C4) break;
         const int row = e / C4;
         const int col = (e - row * C4) * 4;
         float mw[WARPS];
@@ -791,54 +871,11 @@ __global__ void __launch_bounds__(THREADS, STAGES == kStages ? 2 : 1) paged_deco
     __syncthreads();
     if (!s_is_last) return;
     __threadfence();
-    // Each thread owns four consecutive output elements of one query row and walks the splits in
-    // groups of sixteen: all loads of a group (sixteen 16-byte partial loads and their log-sum-exps)
-    // are issued before any is used, so a group costs one L2 round trip, and groups are combined with
-    // the same running-maximum rescaling as the main loop.
-    constexpr int D4 = D / 4;
-    constexpr int GROUP = 16;
     const size_t hq0 = static_cast<size_t>(b) * p.Hq + h * G;
-    for (int e = threadIdx.x; e < G * D4; e += THREADS) {
-        const int row = e / D4;
-        const int c4 = e - row * D4;
-        const float* lse_g = p.partial_lse + (hq0 + row) * S;
-        const float4* po = reinterpret_cast<const float4*>(p.partial_o + (hq0 + row) * S * D) + c4;
-        float M = -INFINITY, den = 0.0f;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s0 = 0; s0 < n_active; s0 += GROUP) {
-            float4 v[GROUP];
-            float l[GROUP];
-#pragma unroll
-            for (int u = 0; u < GROUP; ++u) {
-                const bool on = s0 + u < n_active;
-                l[u] = on ? __ldcg(lse_g + s0 + u) : -INFINITY;
-                v[u] = on ? __ldcg(po + static_cast<size_t>(s0 + u) * D4) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-            float gm = M;
-#pragma unroll
-            for (int u = 0; u < GROUP; ++u) gm = fmaxf(gm, l[u]);
-            const float rescale = __expf(M - gm);              // 0 on the first group (M = -inf)
-            acc.x *= rescale;
-            acc.y *= rescale;
-            acc.z *= rescale;
-            acc.w *= rescale;
-            den *= rescale;
-            M = gm;
-#pragma unroll
-            for (int u = 0; u < GROUP; ++u) {
-                const float wgt = __expf(l[u] - M);            // 0 for the padding entries
-                acc.x = fmaf(wgt, v[u].x, acc.x);
-                acc.y = fmaf(wgt, v[u].y, acc.y);
-                acc.z = fmaf(wgt, v[u].z, acc.z);
-                acc.w = fmaf(wgt, v[u].w, acc.w);
-                den += wgt;
-            }
-        }
-        const float inv = 1.0f / den;
-        const uint2 bits = make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
-        *reinterpret_cast<uint2*>(p.out + (hq0 + row) * D + c4 * 4) = bits;
-        if (p.out_mirror != nullptr) *reinterpret_cast<uint2*>(p.out_mirror + (hq0 + row) * D + c4 * 4) = bits;
-    }
+    const int items = G * (D / 4);                   // a thread owns up to three of them
+    if (items <= THREADS) merge_splits_from_workspace<D, 1, 16>(p, hq0, items, S, n_active);
+    else if (items <= 2 * THREADS) merge_splits_from_workspace<D, 2, 8>(p, hq0, items, S, n_active);
+    else merge_splits_from_workspace<D, 3, 5>(p, hq0, items, S, n_active);
 }
 
 template <int D, bool WIDE, int ROPE, int STAGES>
