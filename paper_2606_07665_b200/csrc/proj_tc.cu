@@ -109,35 +109,6 @@ struct VariantSmem {
     static_assert(PSUM % 8 == 0 && END <= TC_RING_BYTES, "variant epilogue working set");
 };
 
-// y = bf16(bf16(v * rr) * w) with both roundings to nearest even of the fp64 products (the per-head
-// RMSNorm of one feature; rr = 1 / rms as fp64, w a bf16 weight).  The first product is evaluated in
-// fp32 with its residual (rr split in two floats), which provably rounds like the fp64 product when the
-// result is three fp32 ulps clear of every midpoint between bf16 values; otherwise fp64 decides.  The
-// second product of two bf16 values is exact in fp32.
-// The rare fp64 ways out of rmsnorm_feature, kept out of line so that the common path holds no fp64.
-__device__ __noinline__ uint16_t bf16_of_product_f64(float a, double b) {
-    return f64_to_bf16_rne(__dmul_rn(static_cast<double>(a), b));
-}
-
-__device__ __forceinline__ uint16_t rmsnorm_feature(uint16_t v16, double rr, float rr_hi, float rr_lo, float wf) {
-    const float v = bf16_bits_to_float(v16);
-    const float pr = __fmul_rn(v, rr_hi);
-    const float pl = __fmaf_rn(v, rr_hi, -pr);                        // exact residual of the product
-    const float r = __fadd_rn(pr, __fmaf_rn(v, rr_lo, pl));
-    const uint32_t u = __float_as_uint(r);
-    const float mag = fabsf(pr);
-    uint16_t y1 = static_cast<uint16_t>((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
-    if (!((((u & 0xFFFFu) - 0x7FFEu) > 4u) && mag >= 0x1p-60f && mag <= 0x1p100f))
-        y1 = bf16_of_product_f64(v, rr);
-    const float y1f = bf16_bits_to_float(y1);
-    const float q = __fmul_rn(y1f, wf);
-    const float qmag = fabsf(q);
-    if (!(qmag >= 0x1p-100f && qmag <= 0x1p100f))                     // zero, tiny, huge or NaN: the plain way
-        return bf16_of_product_f64(y1f, static_cast<double>(wf));
-    const uint32_t uq = __float_as_uint(q);
-    return static_cast<uint16_t>((uq + 0x7FFFu + ((uq >> 16) & 1u)) >> 16);
-}
-
 // The variant epilogue's tiles are disjoint blocks of 32 pairs: tile blk holds pairs [32 blk, 32 blk + 32).
 constexpr int kVariantTilePairs = 32;
 

@@ -124,6 +124,73 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
     // and everybody else waits here.
     if (warp != QKV_WARPS) cudaGridDependencySynchronize();
 
+    // Prelude variants: in the epilogue consumer thread t owns items t and t + 256 of the CTA's
+    // [32 features][BT rows] tile.  Where an item goes, which table entry turns it and where its partner
+    // sits do not depend on the accumulators: looked up here, the loads complete under the main loop.
+    constexpr int VTHREADS = QKV_WARPS * 32;
+    constexpr int VITEMS = (32 * BT + VTHREADS - 1) / VTHREADS;
+    uint16_t* v_dst[VITEMS];                          // where the item is stored; nullptr: not stored
+    float v_cos[VITEMS], v_sin[VITEMS], v_w[VITEMS];   // table entry; norm weight of the feature
+    int v_prow[VITEMS], v_owner[VITEMS], v_feat[VITEMS];
+    bool v_rot[VITEMS], v_first[VITEMS];
+    if (EPI == EPI_QKV_ROPE_VARIANT && warp != QKV_WARPS) {
+        const int d = p.d, half_d = d / 2, R = p.rotary_dim, half_r = R / 2;
+        const bool is_q = hh < p.Hq, is_k = !is_q && hh < p.Hq + p.Hkv;
+        const uint16_t* nw = is_q ? p.q_norm_w : (is_k ? p.k_norm_w : nullptr);
+#pragma unroll
+        for (int k = 0; k < VITEMS; ++k) {
+            const int item = threadIdx.x + k * VTHREADS;
+            const int r = (item / BT) & 31, n = item % BT;
+            const int b = b0 + n;
+            const int f = (r >> 4) * half_d + 16 * blk + (r & 15);               // feature inside the head
+            v_feat[k] = f;
+            v_w[k] = nw != nullptr ? bf16_bits_to_float(nw[f]) : 1.0f;
+            v_dst[k] = nullptr;
+            v_cos[k] = 1.0f;
+            v_sin[k] = 0.0f;
+            v_rot[k] = (is_q || is_k) && f < R;
+            int i, partner;
+            if (p.interleaved) {
+                i = f >> 1;
+                v_first[k] = (f & 1) == 0;
+                partner = v_first[k] ? f + 1 : f - 1;
+            } else {
+                v_first[k] = f < half_r;
+                i = v_first[k] ? f : f - half_r;
+                partner = v_first[k] ? f + half_r : f - half_r;
+            }
+            if (!v_rot[k]) partner = f;
+            // the partner feature lives in CTA (partner mod d/2) / 16 of the cluster, local row below
+            v_owner[k] = (partner & (half_d - 1)) >> 4;                          // d/2 is 32 or 64
+            v_prow[k] = (partner >= half_d ? 16 : 0) + (partner & 15);
+            if (item >= 32 * BT || b >= p.B) continue;
+            const int ctx = p.context_lens[b];
+            if (ctx < 0) continue;                         // inactive row
+            const int page_idx = ctx / p.page_size;
+            if (ctx >= p.max_position || page_idx >= p.max_pages_per_seq) {
+                if (p.status_flag != nullptr && r == 0 && blk == 0) atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
+                continue;
+            }
+            if (is_q) {
+                v_dst[k] = p.q_out + (static_cast<size_t>(b) * p.Hq + hh) * d + f;
+            } else {
+                const int page = p.block_table[static_cast<size_t>(b) * p.max_pages_per_seq + page_idx];
+                if (page < 0 || page >= p.num_pages) {
+                    if (p.status_flag != nullptr && r == 0 && blk == 0) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
+                    continue;
+                }
+                const int h = is_k ? hh - p.Hq : hh - p.Hq - p.Hkv;
+                v_dst[k] = (is_k ? p.k_cache : p.v_cache) + static_cast<size_t>(page) * p.stride_page +
+                           static_cast<size_t>(ctx - page_idx * p.page_size) * p.stride_token +
+                           static_cast<size_t>(h) * p.stride_head + f;
+            }
+            if (v_rot[k]) {
+                v_cos[k] = __ldg(p.rope_cos + static_cast<size_t>(ctx) * half_r + i);
+                v_sin[k] = __ldg(p.rope_sin + static_cast<size_t>(ctx) * half_r + i);
+            }
+        }
+    }
+
     bool timed_out = false;
     float acc[RB][NT][4];
 #pragma unroll
@@ -259,29 +326,39 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
     if (EPI == EPI_QKV_ROPE_VARIANT) {
         // ---- epilogue with the prelude variants ------------------------------------------------------
         // The d/32 CTAs that share a head (blockIdx.x) are one thread-block cluster.  A CTA holds 32 of
-        // the head's features; the per-head RMSNorm needs the sum of squares of all d, and partial or
-        // interleaved rotary pairs a feature with one that may live in a sister CTA.  So: every CTA
-        // parks its rounded features and their partial sum of squares in shared memory, a cluster
+        // the head's features; the per-head RMSNorm needs the sum of squares of all d, and a half-split
+        // rotation over part of the head pairs a feature with one that lives in a sister CTA.  So: every
+        // CTA parks its rounded features and their partial sums of squares in shared memory, a cluster
         // barrier publishes them, the norm reads the sister CTAs' sums (fp64, exact, fixed order) and
-        // parks the normalised features, a second barrier publishes those, and the rotation fetches each
-        // partner from whichever CTA owns it.  A third barrier keeps every CTA's shared memory alive
-        // until its sisters are done reading.  Every CTA executes all three on every path.
-        const int d = p.d, half_d = d / 2;
+        // parks the normalised features, and the rotation fetches each partner from whichever CTA owns
+        // it.  With remote partners two more cluster barriers follow (normalised features visible;
+        // nobody's shared memory released while a sister reads it); with local partners the sums are the
+        // only remote reads: the CTA arrives at a second barrier once it has read them and waits for it
+        // as the last thing it does.  All CTAs of a cluster take the same path (same head, same parameters).
+        const int d = p.d;
         uint16_t* vals = reinterpret_cast<uint16_t*>(smem_gen + L::VAR_OFFSET);      // [32][BT]
         uint16_t* valsn = vals + 32 * BT;                                            // [32][BT] after the norm
         double* sums = reinterpret_cast<double*>(valsn + 32 * BT);                   // [BT]
         const bool is_q = hh < p.Hq, is_k = !is_q && hh < p.Hq + p.Hkv;
         const uint16_t* norm_w = is_q ? p.q_norm_w : (is_k ? p.k_norm_w : nullptr);
+        const bool has_norm = norm_w != nullptr;
+        const bool remote_partner = (is_q || is_k) && !p.interleaved && p.rotary_dim != d;
         const int n_cta = d / 32;                       // CTAs in the cluster
-        for (int item = threadIdx.x; item < 32 * BT; item += QKV_THREADS) {
-            const int r = item / BT, n = item - r * BT;
-            float y = 0.0f;
+        const bool pass_thread = warp != QKV_WARPS;     // the consumer threads own the items
+        if (pass_thread) {
 #pragma unroll
-            for (int w = 0; w < QKV_WARPS; ++w) y += red[(w * TROWS + r) * BT + n];
-            vals[item] = static_cast<uint16_t>(pack_bf16x2(y, 0.0f) & 0xFFFFu);
+            for (int k = 0; k < VITEMS; ++k) {
+                const int item = threadIdx.x + k * VTHREADS;
+                if (item >= 32 * BT) continue;
+                const int r = item / BT, n = item - r * BT;
+                float y = 0.0f;
+#pragma unroll
+                for (int w = 0; w < QKV_WARPS; ++w) y += red[(w * TROWS + r) * BT + n];
+                vals[item] = static_cast<uint16_t>(pack_bf16x2(y, 0.0f) & 0xFFFFu);
+            }
         }
         __syncthreads();
-        if (threadIdx.x < BT) {
+        if (has_norm && threadIdx.x < BT) {
             double ss = 0.0;
             for (int r = 0; r < 32; ++r) {
                 const double v = static_cast<double>(bf16_bits_to_float(vals[r * BT + threadIdx.x]));
@@ -289,79 +366,57 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
             }
             sums[threadIdx.x] = ss;
         }
-        cluster_sync_all();
+        if (has_norm || remote_partner) cluster_sync_all();
+        else __syncthreads();
         __shared__ double s_rscale[16];                 // 1 / rms of each batch row of the tile
-        if (norm_w != nullptr && threadIdx.x < BT) {
+        if (has_norm && threadIdx.x < BT) {
             double total = 0.0;
             for (int c = 0; c < n_cta; ++c)
                 total = __dadd_rn(total, cluster_load_f64(cluster_map_shared(smem_addr(sums + threadIdx.x), c)));
-            s_rscale[threadIdx.x] = __ddiv_rn(1.0, __dsqrt_rn(__dadd_rn(__ddiv_rn(total, static_cast<double>(d)),
-                                                                        static_cast<double>(p.norm_eps))));
+            // head_dim is a power of two: the mean is an exact scaling; 1 / x by the correctly rounded reciprocal
+            s_rscale[threadIdx.x] = __drcp_rn(__dsqrt_rn(__dadd_rn(__dmul_rn(total, 1.0 / static_cast<double>(d)),
+                                                                   static_cast<double>(p.norm_eps))));
         }
         __syncthreads();
-        for (int item = threadIdx.x; item < 32 * BT; item += QKV_THREADS) {
-            const int r = item / BT, n = item - r * BT;
-            uint16_t v16 = vals[item];
-            if (norm_w != nullptr) {
-                const double rr = s_rscale[n];
-                const int f = (r >> 4) * half_d + 16 * blk + (r & 15);               // feature inside the head
-                const uint16_t y1 = f64_to_bf16_rne(__dmul_rn(static_cast<double>(bf16_bits_to_float(v16)), rr));
-                v16 = f64_to_bf16_rne(__dmul_rn(static_cast<double>(bf16_bits_to_float(y1)),
-                                                static_cast<double>(bf16_bits_to_float(norm_w[f]))));
-            }
-            valsn[item] = v16;
-        }
-        cluster_sync_all();
-        const int R = p.rotary_dim, half_r = R / 2;
-        for (int item = threadIdx.x; item < 32 * BT; item += QKV_THREADS) {
-            const int r = item / BT, n = item - r * BT;
-            const int b = b0 + n;
-            if (b >= p.B) continue;
-            const int ctx = p.context_lens[b];
-            if (ctx < 0) continue;                         // inactive row
-            const int page_idx = ctx / p.page_size;
-            if (ctx >= p.max_position || page_idx >= p.max_pages_per_seq) {
-                if (p.status_flag != nullptr && r == 0 && blk == 0) atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
-                continue;
-            }
-            const int f = (r >> 4) * half_d + 16 * blk + (r & 15);
-            uint16_t v16 = valsn[item];
-            if ((is_q || is_k) && f < R) {
-                int i, partner;
-                bool first;
-                if (p.interleaved) {
-                    i = f >> 1;
-                    first = (f & 1) == 0;
-                    partner = first ? f + 1 : f - 1;
-                } else {
-                    first = f < half_r;
-                    i = first ? f : f - half_r;
-                    partner = first ? f + half_r : f - half_r;
-                }
-                // the partner feature lives in CTA (partner mod d/2) / 16 of the cluster, local row below
-                const int owner = (partner % half_d) >> 4;
-                const int prow = (partner / half_d) * 16 + (partner & 15);
-                const uint16_t other = cluster_load_u16(cluster_map_shared(smem_addr(valsn + prow * BT + n), owner));
-                const float c = p.rope_cos[static_cast<size_t>(ctx) * half_r + i];
-                const float sn = p.rope_sin[static_cast<size_t>(ctx) * half_r + i];
-                v16 = first ? rope_first_half(v16, other, c, sn) : rope_second_half(other, v16, c, sn);
-            }
-            if (is_q) {
-                p.q_out[(static_cast<size_t>(b) * p.Hq + hh) * d + f] = v16;
-            } else {
-                const int page = p.block_table[static_cast<size_t>(b) * p.max_pages_per_seq + page_idx];
-                if (page < 0 || page >= p.num_pages) {
-                    if (p.status_flag != nullptr && r == 0 && blk == 0) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
-                    continue;
-                }
-                const int h = is_k ? hh - p.Hq : hh - p.Hq - p.Hkv;
-                uint16_t* dst = (is_k ? p.k_cache : p.v_cache) + static_cast<size_t>(page) * p.stride_page +
-                                static_cast<size_t>(ctx - page_idx * p.page_size) * p.stride_token +
-                                static_cast<size_t>(h) * p.stride_head;
-                dst[f] = v16;
+        const bool split_barrier = has_norm && !remote_partner;
+        if (split_barrier) cluster_arrive_all();
+        const uint16_t* rot_src = has_norm ? valsn : vals;
+        if (has_norm && pass_thread) {
+#pragma unroll
+            for (int k = 0; k < VITEMS; ++k) {
+                const int item = threadIdx.x + k * VTHREADS;
+                if (item >= 32 * BT) continue;
+                const double rr = s_rscale[item % BT];
+                const float rr_hi = __double2float_rn(rr);
+                const float rr_lo = __double2float_rn(__dsub_rn(rr, static_cast<double>(rr_hi)));
+                valsn[item] = rmsnorm_feature(vals[item], rr, rr_hi, rr_lo, v_w[k]);
             }
         }
-        cluster_sync_all();
+        if (remote_partner) cluster_sync_all();
+        else __syncthreads();
+        if (pass_thread) {
+#pragma unroll
+            for (int k = 0; k < VITEMS; ++k) {
+                const int item = threadIdx.x + k * VTHREADS;
+                if (item >= 32 * BT || v_dst[k] == nullptr) continue;
+                const int n = item % BT;
+                uint16_t v16 = rot_src[item];
+                if (v_rot[k]) {
+                    const uint16_t* psrc = rot_src + v_prow[k] * BT + n;
+                    const uint16_t other =
+                        v_owner[k] == blk ? *psrc : cluster_load_u16(cluster_map_shared(smem_addr(psrc), v_owner[k]));
+                    // first half: x c - partner s; second half: x c + partner s
+                    const float mine = bf16_bits_to_float(v16), theirs = bf16_bits_to_float(other);
+                    const float s_signed = v_first[k] ? v_sin[k] : -v_sin[k];
+                    bool proven;
+                    v16 = rope_diff_of_products_f32(mine, v_cos[k], theirs, s_signed, proven);
+                    if (!proven) v16 = rope_diff_of_products_f64(mine, v_cos[k], theirs, s_signed);
+                }
+                *v_dst[k] = v16;
+            }
+        }
+        if (remote_partner) cluster_sync_all();
+        else if (split_barrier) cluster_wait_all();
         return;
     }
 
