@@ -9,9 +9,9 @@
 // What sets the pace is how fast one SM pulls its share of W out of DRAM through TMA (about 40 GB/s
 // per SM, whatever the ring depth), so the feature tiles are chosen to put a CTA on nearly every SM:
 //   QKV      48 features per CTA = 24 rotary pairs (W rows i..i+23 and i+d/2.. of one head).  A head
-//            has 64 pairs (d = 128), so three tiles start at pairs 0, 16 and 40: 144 CTAs for 48 head
-//            slots; the pairs that two tiles share are computed twice and stored twice with the same
-//            bits (12.5 % more weight traffic for 50 % more SMs).
+//            has 64 pairs (d = 128), so three tiles start at pairs 0, 24 and 48: 144 CTAs for 48 head
+//            slots.  The third tile holds 16 pairs; the 8 pairs' worth of W rows past the head are
+//            zero-filled by TMA and cost no traffic.
 //   QKV with prelude variants (per-head norm, partial or interleaved rotary)
 //            64 features per CTA = 32 pairs, disjoint tiles (two per head for d = 128, one for d = 64)
 //            that form a thread-block cluster: the norm needs the sum of squares over the whole head,
@@ -66,11 +66,10 @@ struct TcTile {
     static constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;                              // two accumulators
 };
 
-// First rotary pair of QKV tile `blk` inside its head: 24-pair tiles at 0, 16, 40 (64 pairs per head)
-// or at 0, 8 (32 pairs per head); multiples of 8 so that every store is 16-byte aligned.
-__host__ __device__ inline int qkv_tile_first_pair(int half_d, int blk) {
-    return half_d == 64 ? (blk == 0 ? 0 : blk == 1 ? 16 : 40) : 8 * blk;
-}
+// First rotary pair of QKV tile `blk` inside its head: 24-pair tiles at 0, 24 and 48 (64 pairs per
+// head) or at 0 and 24 (32 pairs per head).  The last tile reaches past the head: TMA fills those W
+// rows with zeros without reading anything, and the epilogue skips the column groups that hold them.
+__host__ __device__ inline int qkv_tile_first_pair(int /*half_d*/, int blk) { return 24 * blk; }
 
 struct TcParams {
     uint16_t* q_out;
@@ -275,6 +274,18 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
                 v_sn[it][hsel] = 0.0f;
             }
     }
+    // W does not come from the kernel before this one, x does: the producer sends the weight loads of
+    // the first ring fill on their way before anybody waits for that kernel (with programmatic stream
+    // serialization this CTA may be resident while the predecessor still runs).
+    const int first_fill = n_chunks < stages ? n_chunks : stages;
+    if (threadIdx.x == 0) {
+        const uint64_t stream_once = l2_policy_evict_first();
+        for (int c = 0; c < first_fill; ++c) {
+            mbar_arrive_expect_tx(full_bar + c * 8, stage_bytes);
+            tma_load_5d(smem_base + c * stage_bytes + a_bytes, &w_map, full_bar + c * 8, 0, pair0, 0, hh, c * KBLK,
+                        stream_once);
+        }
+    }
     cudaGridDependencySynchronize();      // x (and the residual) come from the preceding kernel
 
     bool timed_out = false;
@@ -282,9 +293,11 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
         if (lane == 0) {
             const uint64_t stream_once = l2_policy_evict_first();
             const uint64_t keep = l2_policy_evict_last();
-            int stage = 0;
-            uint32_t round = 0;                              // how often the ring has wrapped
-            for (int c = 0; c < n_chunks; ++c) {
+            for (int c = 0; c < first_fill; ++c)             // the x tiles of the first ring fill
+                tma_load_3d(smem_base + c * stage_bytes, &x_map, full_bar + c * 8, 0, b0, c * KBLK, keep);
+            int stage = first_fill == stages ? 0 : first_fill;
+            uint32_t round = first_fill == stages ? 1 : 0;   // how often the ring has wrapped
+            for (int c = first_fill; c < n_chunks; ++c) {
                 if (round > 0 && !mbar_wait_bounded(empty_bar + stage * 8, (round - 1) & 1)) {
                     timed_out = true;
                     break;
@@ -484,6 +497,7 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
             // 8 rotary pairs: first halves in columns 8 group .., second halves in columns 24 + 8 group ..
             const int d = p.d, half_d = d / 2;
             const int i0 = pair0 + 8 * group;                // first pair of this warp inside the head
+            ok = ok && i0 < half_d;                          // the last tile's columns past the head
             uint16_t* dst = nullptr;
             const bool rotate = hh < p.Hq + p.Hkv;           // v heads are stored as they are
             float cs[8], sn[8];
