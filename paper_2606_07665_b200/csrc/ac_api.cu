@@ -211,6 +211,9 @@ static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_con
     const double slots = 2.0 * sm_count;
     const double hbm = 6.5e12 * sm_count / 148.0;      // bytes/s the whole GPU streams
     const double cta_rate = 33e9;                       // bytes/s one CTA streams on its own
+    // Grids of at most one CTA per SM with splits longer than 192 tokens run twelve warps per CTA
+    // (launch_one in paged_decode_attn.cu); fitted to sweeps of the split count like the figure above.
+    const double fat_cta_rate = 75e9;
     const double wave_cost = 3e-6;
     // A grid that could have fitted the GPU at once but spills into a further wave pays much more than
     // a ramp for it: the CTAs of that wave start only when first-wave CTAs retire and then need their
@@ -250,6 +253,8 @@ static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_con
             const bool in_cluster = cand <= kClusterMergeMaxSplits &&
                                     static_cast<long long>(B) * Hkv * cand <= sm_count;
             if (cand > 1 && chunk < (in_cluster ? 128 : 256)) continue;
+            const bool fat = static_cast<long long>(B) * Hkv * cand <= sm_count && chunk > 192;
+            const double rate = fat ? fat_cta_rate : cta_rate;
             double n = static_cast<double>(pairs) * cand;                // CTAs that have tokens
             double longest = chunk;                                       // tokens of the longest CTA
             if (token_counts != nullptr) {
@@ -273,11 +278,11 @@ static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_con
                 const double c = longest * bytes_per_token;
                 const double last = n - (waves - 1.0) * slots;
                 t = (waves - 1.0) * slots * c / hbm;
-                const double t_last_bw = last * c / hbm, t_last_cta = c / cta_rate;
+                const double t_last_bw = last * c / hbm, t_last_cta = c / rate;
                 t += (t_last_bw > t_last_cta ? t_last_bw : t_last_cta) + wave_cost + (waves - 1.0) * spill_wave_cost;
             } else {
                 const double t_bw = total_tokens * Hkv * bytes_per_token / hbm;
-                const double t_cta = longest * bytes_per_token / cta_rate;
+                const double t_cta = longest * bytes_per_token / rate;
                 t = (t_bw > t_cta ? t_bw : t_cta) + wave_cost + (waves - 1.0) * spill_wave_cost;
             }
             if (cand > 1)            // partials out and back in plus the ticket round trip, or two cluster barriers

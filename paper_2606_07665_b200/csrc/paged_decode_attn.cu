@@ -8,8 +8,9 @@
 // issuing thread on the order of 100 ns, so the number of loads per tile matters: splitting head_dim
 // into the innermost 64 elements and an outer block index keeps the swizzle span at 128 bytes while
 // still fetching the whole 256-byte rows with one instruction.)  Every warp runs its own ring of
-// STAGES tiles (two; four when the grid is at most one CTA per SM and the splits are long) with one
-// mbarrier per stage and takes tiles warp, warp+WARPS, ... of the CTA's token range; there is no
+// two tiles with one mbarrier per stage and takes tiles warp, warp+WARPS, ... of the CTA's token range
+// (six warps per CTA and two CTAs per SM; twelve warps when the grid is at most one CTA per SM and
+// the splits are long); there is no
 // CTA-wide synchronisation in the main loop.  The physical page id of a tile is fetched from the block
 // table one tile ahead of the TMA issue that needs it.  KV bytes are read once, so the loads carry an
 // evict-first L2 policy.
@@ -45,24 +46,24 @@ namespace {
 
 using namespace acdev;
 
-constexpr int WARPS = 6;
-constexpr int THREADS = WARPS * 32;
-constexpr int kStages = 2;                    // tiles in flight per warp; kDeepStages when the SM holds one CTA
-constexpr int kDeepStages = 4;
+constexpr int kWarps = 6;                     // warps per CTA, two CTAs per SM
+constexpr int kFatWarps = 12;                 // warps per CTA when the SM holds one CTA (grids of at most one CTA per SM)
+constexpr int kStages = 2;                    // tiles in flight per warp
 constexpr int TILE = 16;                      // tokens per stage
 constexpr int kLongestFirstMaxBatch = 128;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 
-template <int D, int STAGES>
+template <int D, int NW>
 struct Smem {
+    static constexpr int STAGES = kStages;
     static constexpr int HALVES = D / 64;                 // 64-element (128-byte) column blocks
     static constexpr int HALF_BYTES = TILE * 128;         // one swizzled [16 x 128 B] block
     static constexpr int K_BYTES = HALVES * HALF_BYTES;   // K tile; V tile has the same size
     static constexpr int STAGE_BYTES = 2 * K_BYTES;
     static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
-    static constexpr int BAR_OFFSET = WARPS * RING_BYTES;
-    static constexpr int TOTAL = BAR_OFFSET + WARPS * STAGES * 8 + 1024;   // + alignment slack
+    static constexpr int BAR_OFFSET = NW * RING_BYTES;
+    static constexpr int TOTAL = BAR_OFFSET + NW * STAGES * 8 + 1024;      // + alignment slack
 };
 
 struct AttnParams {
@@ -117,7 +118,7 @@ constexpr int ROPE_NONE = 0, ROPE_PLAIN = 1, ROPE_VARIANT = 2;
 // before any is used, so a group costs one L2 round trip whatever the number of items, and groups are
 // combined with the same running-maximum rescaling as the main loop.  ITEMS * GS <= 16 keeps the
 // loads in registers.
-template <int D, int ITEMS, int GS>
+template <int D, int THREADS, int ITEMS, int GS>
 __device__ __forceinline__ void merge_splits_from_workspace(const AttnParams& p, size_t hq0, int items, int S,
                                                             int n_active) {
     constexpr int D4 = D / 4;
@@ -186,11 +187,14 @@ __device__ __forceinline__ void merge_splits_from_workspace(const AttnParams& p,
     }
 }
 
-template <int D, bool WIDE, int ROPE, int STAGES>
-__global__ void __launch_bounds__(THREADS, STAGES == kStages ? 2 : 1) paged_decode_attn_kernel(
+template <int D, bool WIDE, int ROPE, int NW>
+__global__ void __launch_bounds__(NW * 32, NW == kWarps ? 2 : 1) paged_decode_attn_kernel(
     const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
     const AttnParams p) {
-    using L = Smem<D, STAGES>;
+    using L = Smem<D, NW>;
+    constexpr int WARPS = NW;
+    constexpr int THREADS = NW * 32;
+    constexpr int STAGES = kStages;
     constexpr int ROWS = WIDE ? 2 : 1;          // row blocks of 8 query heads held per thread
     constexpr int KSTEPS = D / 16;
     constexpr int NTILES = D / 8;
@@ -873,19 +877,19 @@ __global__ void __launch_bounds__(THREADS, STAGES == kStages ? 2 : 1) paged_deco
     __threadfence();
     const size_t hq0 = static_cast<size_t>(b) * p.Hq + h * G;
     const int items = G * (D / 4);                   // a thread owns up to three of them
-    if (items <= THREADS) merge_splits_from_workspace<D, 1, 16>(p, hq0, items, S, n_active);
-    else if (items <= 2 * THREADS) merge_splits_from_workspace<D, 2, 8>(p, hq0, items, S, n_active);
-    else merge_splits_from_workspace<D, 3, 5>(p, hq0, items, S, n_active);
+    if (items <= THREADS) merge_splits_from_workspace<D, THREADS, 1, 16>(p, hq0, items, S, n_active);
+    else if (items <= 2 * THREADS) merge_splits_from_workspace<D, THREADS, 2, 8>(p, hq0, items, S, n_active);
+    else merge_splits_from_workspace<D, THREADS, 3, 5>(p, hq0, items, S, n_active);
 }
 
-template <int D, bool WIDE, int ROPE, int STAGES>
+template <int D, bool WIDE, int ROPE, int NW>
 cudaError_t launch_one_staged(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnParams& p_in, int B,
                        cudaStream_t stream) {
     AttnParams p = p_in;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.Hkv, B, p.num_splits);
-    cfg.blockDim = dim3(THREADS);
-    cfg.dynamicSmemBytes = Smem<D, STAGES>::TOTAL;
+    cfg.blockDim = dim3(NW * 32);
+    cfg.dynamicSmemBytes = Smem<D, NW>::TOTAL;
     cfg.stream = stream;
     // Programmatic dependent launch: this kernel may start while the preceding kernel of the
     // stream is still running; it calls cudaGridDependencySynchronize() before touching anything
@@ -910,7 +914,7 @@ cudaError_t launch_one_staged(const CUtensorMap& k_map, const CUtensorMap& v_map
         if (known == 0) {
             int n = 0;
             cfg.numAttrs = 2;
-            const cudaError_t qe = cudaOccupancyMaxActiveClusters(&n, paged_decode_attn_kernel<D, WIDE, ROPE, STAGES>, &cfg);
+            const cudaError_t qe = cudaOccupancyMaxActiveClusters(&n, paged_decode_attn_kernel<D, WIDE, ROPE, NW>, &cfg);
             if (qe != cudaSuccess) {
                 cudaGetLastError();
                 n = 0;
@@ -920,29 +924,29 @@ cudaError_t launch_one_staged(const CUtensorMap& k_map, const CUtensorMap& v_map
         if (static_cast<long long>(B) * p.Hkv > known) p.cluster_merge = 0;
     }
     cfg.numAttrs = p.cluster_merge ? 2 : 1;
-    return cudaLaunchKernelEx(&cfg, paged_decode_attn_kernel<D, WIDE, ROPE, STAGES>, k_map, v_map, p);
+    return cudaLaunchKernelEx(&cfg, paged_decode_attn_kernel<D, WIDE, ROPE, NW>, k_map, v_map, p);
 }
 
-// Grids of at most one CTA per SM leave half of each SM's shared memory unused: when a split holds more
-// tiles than the six two-stage rings take at once, they run with rings twice as deep (four tiles in
-// flight per warp), which shortens a latency-bound warp's time per tile (single request of 4096 tokens:
-// 9.3 -> 8.3 us).  Shorter splits keep the small footprint, which lets the next kernel of a chain
-// become resident beside this one.
+// Grids of at most one CTA per SM leave half of each SM's shared memory and warp slots unused: when a
+// split holds more tiles than the six two-stage rings take at once, they run with twelve warps per CTA
+// (the same bytes in flight per SM as two resident CTAs, and twice the warps to hide a warp's
+// latency-bound time per tile).  Shorter splits keep the small footprint, which lets the next kernel of
+// a chain become resident beside this one.
 template <int D, bool WIDE, int ROPE>
 cudaError_t launch_one(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnParams& p, int B,
                        cudaStream_t stream) {
     int dev = 0;
     cudaGetDevice(&dev);
-    const bool deep = static_cast<long long>(B) * p.Hkv * p.num_splits <= device_state(dev).sm_count &&
-                      p.split_tokens > kStages * WARPS * TILE;
-    return deep ? launch_one_staged<D, WIDE, ROPE, kDeepStages>(k_map, v_map, p, B, stream)
-                : launch_one_staged<D, WIDE, ROPE, kStages>(k_map, v_map, p, B, stream);
+    const bool fat = static_cast<long long>(B) * p.Hkv * p.num_splits <= device_state(dev).sm_count &&
+                     p.split_tokens > kStages * kWarps * TILE;
+    return fat ? launch_one_staged<D, WIDE, ROPE, kFatWarps>(k_map, v_map, p, B, stream)
+               : launch_one_staged<D, WIDE, ROPE, kWarps>(k_map, v_map, p, B, stream);
 }
 
 }  // namespace
 
 cudaError_t attn_set_attributes(int smem_optin) {
-    if (Smem<128, kDeepStages>::TOTAL > smem_optin) return cudaErrorInvalidConfiguration;
+    if (Smem<128, kFatWarps>::TOTAL > smem_optin) return cudaErrorInvalidConfiguration;
     cudaError_t e;
 #define AC_SET_STAGED(D_, W_, R_, S_)                                                              \
     e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, R_, S_>,                             \
@@ -951,7 +955,7 @@ cudaError_t attn_set_attributes(int smem_optin) {
     e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, R_, S_>,                             \
                              cudaFuncAttributeNonPortableClusterSizeAllowed, 1);                   \
     if (e != cudaSuccess) return e;
-#define AC_SET_ONE(D_, W_, R_) AC_SET_STAGED(D_, W_, R_, kStages) AC_SET_STAGED(D_, W_, R_, kDeepStages)
+#define AC_SET_ONE(D_, W_, R_) AC_SET_STAGED(D_, W_, R_, kWarps) AC_SET_STAGED(D_, W_, R_, kFatWarps)
 #define AC_SET(D_, W_)                                                                             \
     AC_SET_ONE(D_, W_, ROPE_NONE) AC_SET_ONE(D_, W_, ROPE_PLAIN) AC_SET_ONE(D_, W_, ROPE_VARIANT)
     AC_SET(128, false)
