@@ -589,6 +589,26 @@ def test_sliding_window(rt, window, splits, fused):
     run_and_compare(rt, w, num_splits=splits, fused=fused, window=window)
 
 
+@pytest.mark.parametrize("fused", [False, True, "step"])
+@pytest.mark.parametrize("kw,splits,window", [
+    # Grids of at most one CTA per SM (148 on the target) whose splits are longer than 192 tokens run
+    # twelve-warp CTAs: without a merge, with the merge inside a cluster (2 .. 16 splits), with a window,
+    # with 16 query heads per KV head, head_dim 64, a ragged batch with an inactive row
+    (dict(B=2, Hq=32, Hkv=8, context_lens=[3000, 1500], num_pages=300), 1, 0),
+    (dict(B=2, Hq=32, Hkv=8, context_lens=[3000, 1500], num_pages=300), 4, 0),
+    (dict(B=2, Hq=32, Hkv=8, context_lens=[3000, 1500], num_pages=300), 9, 0),
+    (dict(B=3, Hq=32, Hkv=2, d=64, context_lens=[2500, 700, 1300], num_pages=300), 5, 0),
+    (dict(B=4, Hq=28, Hkv=4, page_size=32, context_lens=[2047, 0, 900, 411], num_pages=120, inactive_rows=(1,)), 3, 0),
+    (dict(B=2, Hq=14, Hkv=2, context_lens=[2600, 1000], num_pages=240), 2, 1000),
+    (dict(B=1, Hq=8, Hkv=8, context_lens=[4095], num_pages=260), 13, 0),
+])
+def test_grids_of_one_cta_per_sm(rt, kw, splits, window, fused):
+    w = small(61, **kw)
+    assert w.B * w.Hkv * splits <= 148
+    st, _ = run_and_compare(rt, w, num_splits=splits, fused=fused, window=window)
+    assert st.split_tokens > 192
+
+
 @pytest.mark.parametrize("fused", [True, "step"])
 @pytest.mark.parametrize("kw", [
     dict(B=2, Hq=16, Hkv=1, d=128, page_size=16, context_lens=[700, 33], num_pages=64),            # multi-query
