@@ -201,7 +201,7 @@ int ac_qkv_rope_kv_append(const void* x, const void* w_qkv, int H, void* q_out,
  * Q/K RMSNorm as an option of the fused prelude; the per-model adaptations mention partial rotary):
  * the projected, bf16-rounded q and k head vectors are normalised, rotated over their first
  * rotary_dim elements with the chosen pairing and stored, still in one launch.  The CTAs that share a
- * head (d/32 of the warp-MMA kernel, two or three overlapping tiles of the tcgen05 kernel) form a
+ * head (d/32 of the warp-MMA kernel, the one or two 32-pair tiles of the tcgen05 kernel) form a
  * thread-block cluster and exchange the sums of squares and the rotation partners through distributed
  * shared memory.  options == NULL (or all defaults) is ac_qkv_rope_kv_append.  The rope tables are
  * [max_position, rotary_dim/2].  Everything else as ac_qkv_rope_kv_append. */
