@@ -74,10 +74,12 @@ class DecodeStep:
         self.rope_cos = torch.from_numpy(w.rope_cos).to(self.device)
         self.rope_sin = torch.from_numpy(w.rope_sin).to(self.device)
         # Scheduling hint: requests by decreasing length (what a scheduler that knows the lengths
-        # hands over with the block table).  "auto": only where the kernel does not rank by itself.
-        if isinstance(row_order, str) and row_order == "auto":
-            row_order = (np.argsort(-w.context_lens.astype(np.int64), kind="stable").astype(np.int32)
-                         if w.B > 128 else None)
+        # hands over with the block table).  "auto": wherever the grid is more than one wave deep -- the
+        # kernel would otherwise rank the requests itself in every CTA (up to 128 rows, ~1 us) or keep
+        # index order (more rows); decided in set_splits, once the grid is known.
+        self._row_order_auto = isinstance(row_order, str) and row_order == "auto"
+        if self._row_order_auto:
+            row_order = None
         self.row_order = None if row_order is None else torch.from_numpy(np.asarray(row_order, np.int32)).to(self.device)
         self.out = torch.zeros((self.B, self.Hq, self.d), dtype=torch.int16, device=self.device)
         self.status_flag = torch.zeros(1, dtype=torch.int32, device=self.device)
@@ -95,6 +97,10 @@ class DecodeStep:
                                                              span, ac.ac_sm_count())
         self.num_splits = int(num_splits)
         self.split_tokens = ac.ac_split_tokens(span, self.num_splits)
+        if self._row_order_auto:
+            deep = self.B > 1 and self.B * self.Hkv * self.num_splits > 2 * (ac.ac_sm_count() or 148)
+            order = np.argsort(-self.w.context_lens.astype(np.int64), kind="stable").astype(np.int32)
+            self.row_order = torch.from_numpy(order).to(self.device) if deep else None
         # sized for either merge flavour: partials, then the fused path's arrival counters
         self.workspace_bytes = ac.ac_fused_workspace_bytes(self.B, self.Hq, self.Hkv, self.d,
                                                            self.num_splits)
