@@ -295,11 +295,14 @@ static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_con
     }
     if (pairs < static_cast<long long>(slots) && pairs * S <= static_cast<long long>(slots) &&
         split_tokens_for(max_context_len, static_cast<int>(S)) >= 8192) {
-        // Very long contexts in a single wave: every CTA ramps up and drains together, so nothing
-        // overlaps the ramp and the next kernel cannot start under the tail.  About 1.75 waves of
-        // still-long chunks measured 4-5 % faster (long-context workload: 316 vs 330 us).
-        const long long more = static_cast<long long>(1.75 * slots / static_cast<double>(pairs) + 0.5);
-        if (more > S && split_tokens_for(max_context_len, static_cast<int>(more)) >= 2048) S = more;
+        // Very long contexts in a single wave.  The launch runs such grids with four warps per CTA
+        // (launch_one in paged_decode_attn.cu: splits of at least 8192 tokens, more than one and at most
+        // two CTAs per SM), which streams fastest when the wave is full: take the most splits that still
+        // fit the slots and stay that long (long-context workload: 309 us; six-warp CTAs in one wave 326-330 us,
+        // in 1.75 waves of shorter chunks 315 us).
+        long long full = static_cast<long long>(slots) / pairs;
+        while (full > S && split_tokens_for(max_context_len, static_cast<int>(full)) < 8192) --full;
+        if (full > S) S = full;
     }
     if (S < 1) S = 1;
     if (S > 65535) S = 65535;

@@ -48,6 +48,8 @@ using namespace acdev;
 
 constexpr int kWarps = 6;                     // warps per CTA, two CTAs per SM
 constexpr int kFatWarps = 12;                 // warps per CTA when the SM holds one CTA (grids of at most one CTA per SM)
+constexpr int kSlimWarps = 4;                 // warps per CTA, two CTAs per SM, for one wave of very long splits
+constexpr int kSlimMinSplitTokens = 8192;
 constexpr int kStages = 2;                    // tiles in flight per warp
 constexpr int TILE = 16;                      // tokens per stage
 constexpr int kLongestFirstMaxBatch = 128;
@@ -188,7 +190,7 @@ __device__ __forceinline__ void merge_splits_from_workspace(const AttnParams& p,
 }
 
 template <int D, bool WIDE, int ROPE, int NW>
-__global__ void __launch_bounds__(NW * 32, NW == kWarps ? 2 : 1) paged_decode_attn_kernel(
+__global__ void __launch_bounds__(NW * 32, NW == kFatWarps ? 1 : 2) paged_decode_attn_kernel(
     const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
     const AttnParams p) {
     using L = Smem<D, NW>;
@@ -937,10 +939,17 @@ cudaError_t launch_one(const CUtensorMap& k_map, const CUtensorMap& v_map, const
                        cudaStream_t stream) {
     int dev = 0;
     cudaGetDevice(&dev);
-    const bool fat = static_cast<long long>(B) * p.Hkv * p.num_splits <= device_state(dev).sm_count &&
-                     p.split_tokens > kStages * kWarps * TILE;
-    return fat ? launch_one_staged<D, WIDE, ROPE, kFatWarps>(k_map, v_map, p, B, stream)
-               : launch_one_staged<D, WIDE, ROPE, kWarps>(k_map, v_map, p, B, stream);
+    const long long ctas = static_cast<long long>(B) * p.Hkv * p.num_splits;
+    const int sms = device_state(dev).sm_count;
+    const bool fat = ctas <= sms && p.split_tokens > kStages * kWarps * TILE;
+    if (fat) return launch_one_staged<D, WIDE, ROPE, kFatWarps>(k_map, v_map, p, B, stream);
+    // One wave of very long splits, two CTAs per SM: every CTA streams for the whole launch, nothing
+    // ramps beside it, and HBM delivers more with fewer requests outstanding per SM (a compute-free
+    // loop with this kernel's loads: 6.59 TB/s at 192 KB in flight per SM, 6.64 at 128 KB, 6.8 at 96 KB).
+    // Four warps per CTA still cover the arithmetic (three do not).
+    const bool slim = ctas > sms && ctas <= 2ll * sms && p.split_tokens >= kSlimMinSplitTokens;
+    return slim ? launch_one_staged<D, WIDE, ROPE, kSlimWarps>(k_map, v_map, p, B, stream)
+                : launch_one_staged<D, WIDE, ROPE, kWarps>(k_map, v_map, p, B, stream);
 }
 
 }  // namespace
@@ -955,7 +964,8 @@ cudaError_t attn_set_attributes(int smem_optin) {
     e = cudaFuncSetAttribute(paged_decode_attn_kernel<D_, W_, R_, S_>,                             \
                              cudaFuncAttributeNonPortableClusterSizeAllowed, 1);                   \
     if (e != cudaSuccess) return e;
-#define AC_SET_ONE(D_, W_, R_) AC_SET_STAGED(D_, W_, R_, kWarps) AC_SET_STAGED(D_, W_, R_, kFatWarps)
+#define AC_SET_ONE(D_, W_, R_)                                                                    \
+    AC_SET_STAGED(D_, W_, R_, kWarps) AC_SET_STAGED(D_, W_, R_, kFatWarps) AC_SET_STAGED(D_, W_, R_, kSlimWarps)
 #define AC_SET(D_, W_)                                                                             \
     AC_SET_ONE(D_, W_, ROPE_NONE) AC_SET_ONE(D_, W_, ROPE_PLAIN) AC_SET_ONE(D_, W_, ROPE_VARIANT)
     AC_SET(128, false)
