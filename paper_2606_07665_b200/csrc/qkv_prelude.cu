@@ -191,6 +191,53 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
         }
     }
 
+    // The plain epilogues likewise: consumer thread t owns item t of the CTA's tile (one rotary pair, or one
+    // output feature, of one batch row).  Its position, destination and angle -- or its residual -- are
+    // fetched here, under the main loop, not behind it.
+    uint16_t* e_dst = nullptr;                        // QKV: the head vector the pair goes to; nullptr: not stored
+    float e_cos = 1.0f, e_sin = 0.0f;
+    float e_res = 0.0f;                               // o_proj: the residual
+    size_t e_idx = 0;
+    bool e_live = false;
+    if (EPI == EPI_QKV_ROPE_APPEND && warp != QKV_WARPS && threadIdx.x < 16 * BT) {
+        const int j = threadIdx.x / BT, n = threadIdx.x % BT;     // pair inside the block, batch row
+        const int b = b0 + n;
+        const int ctx = b < p.B ? p.context_lens[b] : -1;
+        if (ctx >= 0) {                                            // else: no such row, or inactive
+            const int d = p.d, i = 16 * blk + j;                   // pair index inside the head
+            const int page_idx = ctx / p.page_size;
+            if (ctx >= p.max_position || page_idx >= p.max_pages_per_seq) {
+                if (p.status_flag != nullptr && j == 0 && blk == 0) atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
+            } else if (hh < p.Hq) {
+                e_dst = p.q_out + (static_cast<size_t>(b) * p.Hq + hh) * d + i;
+            } else {
+                const int page = p.block_table[static_cast<size_t>(b) * p.max_pages_per_seq + page_idx];
+                if (page < 0 || page >= p.num_pages) {
+                    if (p.status_flag != nullptr && j == 0 && blk == 0) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
+                } else {
+                    const bool is_k = hh < p.Hq + p.Hkv;
+                    const int h = is_k ? hh - p.Hq : hh - p.Hq - p.Hkv;
+                    e_dst = (is_k ? p.k_cache : p.v_cache) + static_cast<size_t>(page) * p.stride_page +
+                            static_cast<size_t>(ctx - page_idx * p.page_size) * p.stride_token +
+                            static_cast<size_t>(h) * p.stride_head + i;
+                }
+            }
+            if (e_dst != nullptr && hh < p.Hq + p.Hkv) {           // q and k features are rotated
+                e_cos = __ldg(p.rope_cos + static_cast<size_t>(ctx) * (d / 2) + i);
+                e_sin = __ldg(p.rope_sin + static_cast<size_t>(ctx) * (d / 2) + i);
+            }
+        }
+    }
+    if (EPI == EPI_RESIDUAL_ADD && warp != QKV_WARPS && threadIdx.x < TROWS * BT) {
+        const int r = threadIdx.x / BT, n = threadIdx.x % BT;     // feature inside the CTA's block, batch row
+        const int b = b0 + n;
+        if (b < p.B) {
+            e_live = true;
+            e_idx = static_cast<size_t>(b) * p.N + TROWS * hh + r;
+            e_res = bf16_bits_to_float(p.residual_in[e_idx]);
+        }
+    }
+
     bool timed_out = false;
     float acc[RB][NT][4];
 #pragma unroll
@@ -308,17 +355,13 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
 
     if (EPI == EPI_RESIDUAL_ADD) {
         // ---- epilogue of the output projection: h = bf16(residual + y), one rounding ----------------
-        for (int item = threadIdx.x; item < TROWS * BT; item += QKV_THREADS) {
-            const int r = item / BT;                   // row inside the CTA's block of features
-            const int n = item - r * BT;
-            const int b = b0 + n;
-            if (b >= p.B) continue;
+        static_assert(EPI != EPI_RESIDUAL_ADD || TROWS * 16 <= QKV_WARPS * 32, "one item per consumer thread");
+        if (e_live) {
+            const int r = threadIdx.x / BT, n = threadIdx.x % BT;
             float y = 0.0f;
 #pragma unroll
             for (int w = 0; w < QKV_WARPS; ++w) y += red[(w * TROWS + r) * BT + n];
-            const size_t idx = static_cast<size_t>(b) * p.N + TROWS * hh + r;
-            const float res = bf16_bits_to_float(p.residual_in[idx]);
-            p.residual_out[idx] = static_cast<uint16_t>(pack_bf16x2(res + y, 0.0f) & 0xFFFFu);
+            p.residual_out[e_idx] = static_cast<uint16_t>(pack_bf16x2(e_res + y, 0.0f) & 0xFFFFu);
         }
         return;
     }
@@ -421,14 +464,8 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
     }
 
     // ---- epilogue: round, rotate, scatter --------------------------------------------------------
-    const int d = p.d, half = d / 2;
-    for (int item = threadIdx.x; item < 16 * BT; item += QKV_THREADS) {
-        const int j = item / BT;                       // pair inside the block
-        const int n = item - j * BT;
-        const int b = b0 + n;
-        if (b >= p.B) continue;
-        const int ctx = p.context_lens[b];
-        if (ctx < 0) continue;                         // inactive row
+    if (e_dst != nullptr) {
+        const int j = threadIdx.x / BT, n = threadIdx.x % BT;
         float y_lo = 0.0f, y_hi = 0.0f;
 #pragma unroll
         for (int w = 0; w < QKV_WARPS; ++w) {
@@ -437,38 +474,14 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
         }
         const uint32_t packed = pack_bf16x2(y_lo, y_hi);
         uint16_t lo = static_cast<uint16_t>(packed & 0xFFFFu), hi = static_cast<uint16_t>(packed >> 16);
-        const int i = 16 * blk + j;                    // pair index inside the head
-        const int page_idx = ctx / p.page_size;
-        if (ctx >= p.max_position || page_idx >= p.max_pages_per_seq) {
-            if (p.status_flag != nullptr && j == 0 && blk == 0) atomicOr(p.status_flag, AC_FLAG_POSITION_OOB);
-            continue;
-        }
         if (hh < p.Hq + p.Hkv) {                       // q and k features are rotated
-            const float c = p.rope_cos[static_cast<size_t>(ctx) * half + i];
-            const float sn = p.rope_sin[static_cast<size_t>(ctx) * half + i];
-            const uint16_t r0 = rope_first_half(lo, hi, c, sn);
-            const uint16_t r1 = rope_second_half(lo, hi, c, sn);
+            const uint16_t r0 = rope_first_half(lo, hi, e_cos, e_sin);
+            const uint16_t r1 = rope_second_half(lo, hi, e_cos, e_sin);
             lo = r0;
             hi = r1;
         }
-        if (hh < p.Hq) {
-            uint16_t* dst = p.q_out + (static_cast<size_t>(b) * p.Hq + hh) * d;
-            dst[i] = lo;
-            dst[i + half] = hi;
-        } else {
-            const int page = p.block_table[static_cast<size_t>(b) * p.max_pages_per_seq + page_idx];
-            if (page < 0 || page >= p.num_pages) {
-                if (p.status_flag != nullptr && j == 0 && blk == 0) atomicOr(p.status_flag, AC_FLAG_PAGE_OOB);
-                continue;
-            }
-            const bool is_k = hh < p.Hq + p.Hkv;
-            const int h = is_k ? hh - p.Hq : hh - p.Hq - p.Hkv;
-            uint16_t* dst = (is_k ? p.k_cache : p.v_cache) + static_cast<size_t>(page) * p.stride_page +
-                            static_cast<size_t>(ctx - page_idx * p.page_size) * p.stride_token +
-                            static_cast<size_t>(h) * p.stride_head;
-            dst[i] = lo;
-            dst[i + half] = hi;
-        }
+        e_dst[0] = lo;
+        e_dst[p.d / 2] = hi;
     }
 }
 
