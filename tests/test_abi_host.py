@@ -68,6 +68,15 @@ def test_plan_properties(ac, B, Hq, Hkv, d, ps, maxlen):
         assert S > 1                                              # small batches are split across SMs
 
 
+def test_plan_fills_one_wave_for_very_long_contexts(ac):
+    # few requests, very long contexts: the most splits of at least 8192 tokens that still fit one wave
+    # of two CTAs per SM -- the shape the launch runs with four warps per CTA
+    for B, Hkv, maxlen, want in [(4, 8, 131073, 9), (2, 8, 131073, 16), (8, 8, 131073, 4), (1, 8, 1000000, 37)]:
+        S, st, _ = ac.ac_decode_plan(B, 8 * Hkv, Hkv, 128, 16, maxlen, 148)
+        assert S == want, (B, Hkv, maxlen, S)
+        assert st >= 8192 and 148 < B * Hkv * S <= 296 and st * (S - 1) < maxlen
+
+
 def test_plan_for_lengths(ac):
     import numpy as np
     # every row at the maximum: the same plan as without lengths
