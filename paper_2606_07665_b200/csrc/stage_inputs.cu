@@ -25,9 +25,23 @@ __global__ void __launch_bounds__(256) stage_inputs_kernel(const StageList list)
     cudaGridDependencySynchronize();
     const unsigned long long tid = blockIdx.x * 256ull + threadIdx.x;
     const unsigned long long stride = gridDim.x * 256ull;
+    // The five buffers are one index space: a thread's pieces come from whichever buffers they fall
+    // in, so every read over the host link is in flight at once (one buffer after the other made the
+    // threads that serve several buffers pay one link round trip per buffer).
+    unsigned long long total = 0;
 #pragma unroll
-    for (int b = 0; b < 5; ++b)
-        for (unsigned long long i = tid; i < list.chunks[b]; i += stride) list.dst[b][i] = list.src[b][i];
+    for (int b = 0; b < 5; ++b) total += list.chunks[b];
+    for (unsigned long long i = tid; i < total; i += stride) {
+        unsigned long long k = i;
+        int b = 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if (b == c && k >= list.chunks[c]) {
+                k -= list.chunks[c];
+                b = c + 1;
+            }
+        list.dst[b][k] = list.src[b][k];
+    }
     for (unsigned long long i = tid; i < list.zero_chunks; i += stride)
         list.zero_dst[i] = make_uint4(0u, 0u, 0u, 0u);
 }
