@@ -341,9 +341,7 @@ __global__ void __launch_bounds__(NW * 32, NW == kFatWarps ? 1 : 2) paged_decode
     const int new_token_tile = p.new_tokens > 0 ? ctx / TILE : -1;
     const int first_dependent_tile = (ctx > 0 ? ctx - 1 : 0) / TILE;
 
-    auto issue = [&](int j, int page) {      // lane 0 only
-        const int tok0 = tile_token0(j);
-        const int slot = tok0 % p.page_size;
+    auto issue_at = [&](int j, int slot, int page) {      // lane 0 only; slot = first token's slot inside its page
         const int stage = j % STAGES;
         const uint32_t bar = bars + stage * 8;
         const uint32_t dst = ring + stage * L::STAGE_BYTES;
@@ -386,11 +384,18 @@ __global__ void __launch_bounds__(NW * 32, NW == kFatWarps ? 1 : 2) paged_decode
                 dependency_sync();
                 dependency_met = true;
             }
-            if (lane == 0) issue(s, page_first[s]);
+            if (lane == 0) issue_at(s, tile_token0(s) % p.page_size, page_first[s]);
             issued = s + 1;
         }
     }
     int page_next = issued < n_my ? load_page_id(issued) : 0;
+    // Where this warp's next tile sits in the row (block-table index, slot inside the page).  A warp's
+    // tiles are WARPS * TILE tokens apart, so from here on the position is stepped, not divided: the two
+    // integer divisions by the run-time page size per refill cost a fifth of a warp's time per tile.
+    const int step_tokens = WARPS * TILE;
+    const int step_pages = step_tokens / p.page_size, step_slots = step_tokens - step_pages * p.page_size;
+    int next_idx = tile_token0(issued) / p.page_size;
+    int next_slot = tile_token0(issued) - next_idx * p.page_size;
     if (!dependency_met) dependency_sync();                    // q was written by the preceding kernel
     uint16_t q_raw_lo[QP], q_raw_hi[QP];
     if (ROPE == ROPE_PLAIN) {
@@ -718,8 +723,15 @@ __global__ void __launch_bounds__(NW * 32, NW == kFatWarps ? 1 : 2) paged_decode
         __syncwarp();
         if (issued < n_my) {
             const int page = page_next;
-            page_next = issued + 1 < n_my ? load_page_id(issued + 1) : 0;
-            if (lane == 0) issue(issued, page);
+            const int slot = next_slot;
+            next_idx += step_pages;
+            next_slot += step_slots;
+            if (next_slot >= p.page_size) {
+                next_slot -= p.page_size;
+                ++next_idx;
+            }
+            page_next = issued + 1 < n_my ? (next_idx < p.max_pages_per_seq ? bt_row[next_idx] : -1) : 0;
+            if (lane == 0) issue_at(issued, slot, page);
             ++issued;
         }
     }
