@@ -365,7 +365,11 @@ int ac_splitkv_merge(const void* workspace, int num_splits, const int32_t* conte
  * memory the GPU can address, the kernel's final stores go to both; otherwise a copy from out follows).  When the host
  * buffers are pinned memory the GPU can address and their sizes are multiples of 16 bytes, the five
  * inputs are gathered (and the counters cleared) by ONE small kernel reading host memory directly
- * instead of five copy-engine transfers; otherwise each buffer gets its own cudaMemcpyAsync.  Everything is asynchronous on `stream`; the caller
+ * instead of five copy-engine transfers; otherwise each buffer gets its own cudaMemcpyAsync.  The
+ * *_host inputs must be complete when the call is made and stay unchanged until the step has
+ * finished: that kernel reads them as soon as it is resident, which may be while earlier work of the
+ * stream is still running (it writes the device buffers only after that work has completed).
+ * Everything is asynchronous on `stream`; the caller
  * synchronises the stream before reading out_host.  The KV cache pools and rope tables stay on the
  * device (they are the layer's resident state, not a per-step input).  No paper counterpart. */
 int ac_decode_step_host(const void* q_host, const void* k_new_host, const void* v_new_host,

@@ -22,7 +22,6 @@ __global__ void __launch_bounds__(256) stage_inputs_kernel(const StageList list)
     // No early launch-completion trigger here: the attention kernel that follows reads context_lens
     // and block_table (written by this kernel) BEFORE it synchronises on its predecessor, so it must
     // not become resident until this grid has finished.
-    cudaGridDependencySynchronize();
     const unsigned long long tid = blockIdx.x * 256ull + threadIdx.x;
     const unsigned long long stride = gridDim.x * 256ull;
     // The five buffers are one index space: a thread's pieces come from whichever buffers they fall
@@ -31,15 +30,33 @@ __global__ void __launch_bounds__(256) stage_inputs_kernel(const StageList list)
     unsigned long long total = 0;
 #pragma unroll
     for (int b = 0; b < 5; ++b) total += list.chunks[b];
-    for (unsigned long long i = tid; i < total; i += stride) {
-        unsigned long long k = i;
-        int b = 0;
+    auto locate = [&](unsigned long long i, int& b, unsigned long long& k) {
+        k = i;
+        b = 0;
 #pragma unroll
         for (int c = 0; c < 4; ++c)
             if (b == c && k >= list.chunks[c]) {
                 k -= list.chunks[c];
                 b = c + 1;
             }
+    };
+    // The host buffers are complete when the call is made; the device buffers may still be read by the
+    // kernel ahead of this one.  So a thread's first piece crosses the host link BEFORE the wait for
+    // that kernel (this grid becomes resident beside it under programmatic stream serialization) and is
+    // stored after it.
+    int b0 = 0;
+    unsigned long long k0 = 0;
+    uint4 first = make_uint4(0u, 0u, 0u, 0u);
+    if (tid < total) {
+        locate(tid, b0, k0);
+        first = list.src[b0][k0];
+    }
+    cudaGridDependencySynchronize();
+    if (tid < total) list.dst[b0][k0] = first;
+    for (unsigned long long i = tid + stride; i < total; i += stride) {
+        int b;
+        unsigned long long k;
+        locate(i, b, k);
         list.dst[b][k] = list.src[b][k];
     }
     for (unsigned long long i = tid; i < list.zero_chunks; i += stride)
