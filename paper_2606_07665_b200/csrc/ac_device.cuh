@@ -147,6 +147,11 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ void cluster_arrive_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 }
+// Arrival that publishes nothing (a pure "I am done with your shared memory"): it does not wait for the
+// thread's earlier stores to become visible, as the releasing form does.
+__device__ __forceinline__ void cluster_arrive_relaxed_all() {
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void cluster_wait_all() {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }

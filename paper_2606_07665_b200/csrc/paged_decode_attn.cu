@@ -317,7 +317,8 @@ __global__ void __launch_bounds__(NW * 32, NW == kFatWarps ? 1 : 2) paged_decode
             // Cluster merge: keep step with the two cluster barriers of the CTAs that have tokens
             // (this CTA stages nothing and nobody reads its shared memory).
             cluster_sync_all();
-            cluster_sync_all();
+            cluster_arrive_relaxed_all();
+            cluster_wait_all();
         }
         return;
     }
@@ -869,7 +870,11 @@ __global__ void __launch_bounds__(NW * 32, NW == kFatWarps ? 1 : 2) paged_decode
                 if (p.out_mirror != nullptr) *reinterpret_cast<uint2*>(p.out_mirror + (hq0 + row) * D + c4 * 4) = bits;
             }
         }
-        cluster_sync_all();                              // nobody's shared memory goes away before it was read
+        // Second barrier, in two halves and without a release: it publishes nothing, it only keeps every
+        // CTA's shared memory alive until split 0 has consumed it (the values are in its registers by
+        // then), so nobody waits for the result stores above to become visible.
+        cluster_arrive_relaxed_all();
+        cluster_wait_all();
         return;
     }
 

@@ -647,7 +647,7 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
         // Sisters read this CTA's partial sums above: it must not exit before they have.  With local
         // partners that is the last remote access, so arrive now and wait at the very end.
         const bool split_barrier = has_norm && !remote_partner;
-        if (split_barrier) cluster_arrive_all();
+        if (split_barrier) cluster_arrive_relaxed_all();      // publishes nothing: no release needed
         // Every sister of the cluster has the same head slot, hence the same answer to "is there a norm":
         // without one the rotation reads the parked features where they are.
         const uint16_t* rot_src = norm_w != nullptr ? valsn : vals;
@@ -694,8 +694,12 @@ __global__ void __launch_bounds__(TcTile<EPI>::THREADS, 1) proj_tc_kernel(const 
                 }
             }
         }
-        if (remote_partner) cluster_sync_all();               // nobody's shared memory goes while a sister reads it
-        else if (split_barrier) cluster_wait_all();
+        if (remote_partner) {                                 // nobody's shared memory goes while a sister reads it;
+            cluster_arrive_relaxed_all();                     // nothing is published, so no wait for the stores above
+            cluster_wait_all();
+        } else if (split_barrier) {
+            cluster_wait_all();
+        }
     }
 
     // ---- release TMEM (every path reaches this point) ----------------------------------------------

@@ -422,7 +422,7 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
         }
         __syncthreads();
         const bool split_barrier = has_norm && !remote_partner;
-        if (split_barrier) cluster_arrive_all();
+        if (split_barrier) cluster_arrive_relaxed_all();      // publishes nothing: no release needed
         const uint16_t* rot_src = has_norm ? valsn : vals;
         if (has_norm && pass_thread) {
 #pragma unroll
@@ -458,8 +458,12 @@ __global__ void __launch_bounds__(QKV_THREADS, 2) qkv_rope_append_kernel(
                 *v_dst[k] = v16;
             }
         }
-        if (remote_partner) cluster_sync_all();
-        else if (split_barrier) cluster_wait_all();
+        if (remote_partner) {                           // nothing is published here: no wait for the stores above
+            cluster_arrive_relaxed_all();
+            cluster_wait_all();
+        } else if (split_barrier) {
+            cluster_wait_all();
+        }
         return;
     }
 
