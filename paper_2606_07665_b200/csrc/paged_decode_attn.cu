@@ -884,17 +884,19 @@ __global__ void __launch_bounds__(NW * 32, NW == kFatWarps ? 1 : 2) paged_decode
     __shared__ int s_is_last;
     // splits with tokens (a row longer than the split grid covers still has S of them)
     const int n_active = min(S, (n_tokens - window_base + p.split_tokens - 1) / p.split_tokens);
-    __threadfence();
+    // One acquire-release atomic by one thread, bracketed by CTA barriers: the release orders the
+    // partials that every thread of this CTA stored before the first barrier ahead of the ticket, the
+    // acquire orders the ticket ahead of the partial loads that follow the second barrier.
     __syncthreads();
     if (threadIdx.x == 0) {
         int32_t* counter = p.arrivals + static_cast<size_t>(b) * p.Hkv + h;
-        const int ticket = atomicAdd(counter, 1);
+        int ticket;
+        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(ticket) : "l"(counter) : "memory");
         s_is_last = ticket == n_active - 1;
         if (s_is_last) *counter = 0;             // leave the counter ready for the next launch
     }
     __syncthreads();
     if (!s_is_last) return;
-    __threadfence();
     const size_t hq0 = static_cast<size_t>(b) * p.Hq + h * G;
     const int items = G * (D / 4);                   // a thread owns up to three of them
     if (items <= THREADS) merge_splits_from_workspace<D, THREADS, 1, 16>(p, hq0, items, S, n_active);
