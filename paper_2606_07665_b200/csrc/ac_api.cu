@@ -186,6 +186,19 @@ size_t ac_workspace_bytes(int B, int Hq, int d, int num_splits) {
 
 // The plan proper.  token_counts == nullptr: every row is taken to attend over max_context_len
 // tokens; otherwise token_counts[b] = tokens row b attends over (<= 0: the row launches no work).
+// How many thread-block clusters of `size` one-per-SM CTAs are resident at once.  A cluster lives inside
+// one GPC, so this is well below sm_count / size for the larger sizes.  For the 148-SM part the figures
+// are what cudaOccupancyMaxActiveClusters reports for the twelve-warp attention kernel (the launch asks
+// the runtime itself and falls back to the ticket merge when a grid has more clusters than that; the
+// plan only needs to know it in advance to price the merge correctly); other parts get a cautious
+// guess.
+static int cluster_capacity(int size, int sm_count) {
+    static const int b200[17] = {0, 148, 74, 45, 33, 26, 22, 15, 15, 15, 11, 7, 7, 7, 7, 7, 7};
+    if (size < 1 || size > 16) return 0;
+    if (sm_count == 148) return b200[size];
+    return (sm_count / size) * 3 / 4;
+}
+
 static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_context_len, int sm_count,
                        const int32_t* token_counts, int* num_splits_out, int* split_tokens_out,
                        size_t* workspace_bytes_out) {
@@ -251,7 +264,8 @@ static int plan_splits(int B, int Hq, int Hkv, int d, int page_size, int max_con
             if (static_cast<long long>(chunk) * (cand - 1) >= max_context_len) continue;   // empty split
             // the launch decides by the grid it is given: all B rows count, active or not
             const bool in_cluster = cand <= kClusterMergeMaxSplits &&
-                                    static_cast<long long>(B) * Hkv * cand <= sm_count;
+                                    static_cast<long long>(B) * Hkv * cand <= sm_count &&
+                                    static_cast<long long>(B) * Hkv <= cluster_capacity(cand, sm_count);
             if (cand > 1 && chunk < (in_cluster ? 128 : 256)) continue;
             const bool fat = static_cast<long long>(B) * Hkv * cand <= sm_count && chunk > 192;
             const double rate = fat ? fat_cta_rate : cta_rate;
